@@ -1,0 +1,149 @@
+/* covspec.h - C ABI of the B200 (sm_100a) visual-token reduction library.
+ *
+ * The library computes CoVSpec's training-free visual token selection (Sec. III-A of the paper):
+ * query-aware score (Eq. 10), token activity score (Eq. 11), normalise + fuse (Eq. 12), preselect
+ * the M best tokens, energy of every preselected token in the top-r singular subspace of the
+ * stacked matrix Z_M (Eq. 13-15), keep the B_vis tokens of largest energy, and gather the
+ * survivors into a dense buffer (the reduced visual context V-hat that the draft model consumes).
+ *
+ * Conventions used by every entry point
+ *  - "device" pointers are CUDA global-memory addresses on the current device; "host" pointers
+ *    are ordinary process memory.  The library never takes ownership of a caller's buffer.
+ *  - Matrices are dense row-major.  X, Q and every Hs[l] hold one token per row of `d` elements
+ *    of `dtype`; requests are packed back to back and delimited by host offset arrays.
+ *  - Wq / Wk are [n_heads*head_dim, d] row-major: one output feature of the embedding map e(.)
+ *    per row (the layout of a linear layer's weight).  Head h owns rows [h*head_dim,(h+1)*head_dim).
+ *  - Token indices written by the library are request-local (0 .. N_b-1) and ascending inside a
+ *    request.
+ *  - Every call is asynchronous on `stream` (a cudaStream_t passed as void*; NULL = the legacy
+ *    default stream) except for the small host->device copy of the launch plan, which is issued on
+ *    the same stream from a pinned staging buffer owned by the context.
+ *  - Return value: COVSPEC_OK or a negative covspec_status.  Argument, shape, capacity and
+ *    unsupported-configuration errors are detected on the host before anything is launched.
+ *    Conditions only the device can see (non-finite scores) are recorded in a device status word,
+ *    read back by covspec_get_device_status(); outputs are then unspecified but in bounds.
+ *  - One context serves one stream at a time; calls on one context must not overlap.
+ */
+#ifndef COVSPEC_H_
+#define COVSPEC_H_
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct covspec_ctx covspec_ctx; /* opaque; owns the device workspace and the plan cache */
+
+typedef enum { COVSPEC_F32 = 0, COVSPEC_BF16 = 1 } covspec_dtype;
+
+typedef enum {
+  COVSPEC_OK = 0,
+  COVSPEC_ERR_ARG = -1,         /* NULL or inconsistent argument                              */
+  COVSPEC_ERR_SHAPE = -2,       /* offsets not monotone, empty request, budget out of range   */
+  COVSPEC_ERR_UNSUPPORTED = -3, /* configuration outside what the kernels implement           */
+  COVSPEC_ERR_WORKSPACE = -4,   /* problem exceeds the capacities given at init               */
+  COVSPEC_ERR_CUDA = -5,        /* a CUDA runtime call failed (see covspec_last_cuda_error)   */
+  COVSPEC_ERR_NONFINITE = -6,   /* device status: a score was NaN or Inf                      */
+  COVSPEC_ERR_NOCONVERGE = -7   /* device status: small eigen-solve hit its sweep limit       */
+} covspec_status;
+
+/* Static configuration.  Fill with covspec_default_config() and override. */
+typedef struct {
+  int dtype;           /* covspec_dtype of X, Q, Wq, Wk, Hs and of the compacted output           */
+  int d;               /* feature width; must be a multiple of 8                                   */
+  int n_heads;         /* 0 = identity embedding e(x)=x (Wq, Wk ignored); else head_dim must be 128 */
+  int head_dim;
+  int act_layers;      /* K of Eq. 11 (number of late-layer differences); 0 = no activity term     */
+  float lambda;        /* lambda of Eq. 12                                                         */
+  int norm_mode;       /* "normalize to the same scale": 0 min-max per request, 1 z-score, 2 none  */
+  int head_reduce;     /* 0 max over (query element, head) pairs, 1 mean over heads then max       */
+  float presel_factor; /* M = min(N, max(B_vis, ceil(presel_factor*B_vis)))                        */
+  float rank_frac;     /* r = clamp(ceil(rank_frac*B_vis), 1, min(rank_cap, M-1, d-1))             */
+  int rank_cap;
+  int eig_iters;       /* subspace-iteration steps used to reach the top-r singular subspace       */
+  int eig_oversample;  /* extra basis vectors carried beyond r; rank_cap + eig_oversample <= 160    */
+  int max_batch;                 /* capacities the workspace is sized for */
+  long long max_total_vis;       /* sum of N_b */
+  long long max_total_txt;       /* sum of T_b */
+  int max_vis_per_req;           /* max N_b */
+  int max_presel_per_req;        /* max M_b   (0: derive from max_vis_per_req) */
+  long long max_total_presel;    /* sum of M_b (0: derive from max_total_vis)  */
+} covspec_config;
+
+/* One batch of requests (Sec. III-A notation in brackets). */
+typedef struct {
+  int batch;
+  const void* X;            /* device [vis_offsets[batch], d]  visual tokens v_i = z_i            */
+  const int* vis_offsets;   /* host   [batch+1] first row of each request in X, vis_offsets[0]=0   */
+  const void* Q;            /* device [txt_offsets[batch], d]  query elements q_j                  */
+  const int* txt_offsets;   /* host   [batch+1]                                                    */
+  const void* Wq;           /* device [n_heads*head_dim, d] or NULL when n_heads == 0              */
+  const void* Wk;           /* device [n_heads*head_dim, d] or NULL when n_heads == 0              */
+  const void* const* Hs;    /* host array of act_layers+1 device pointers h^(L-K) .. h^(L), each
+                               laid out like X; NULL when act_layers == 0                          */
+  const int* keep;          /* host [batch] B_vis per request, or NULL to use keep_ratio           */
+  double keep_ratio;        /* B_vis = max(1, ceil(keep_ratio*N_b - 1e-6)), evaluated in double      */
+} covspec_problem;
+
+/* Defaults: lambda 0.5, min-max, head max, presel_factor 2, rank_frac 0.5, rank_cap 128,
+ * eig_iters 6, eig_oversample 32, act_layers 4; capacities zero (the caller must set them). */
+void covspec_default_config(covspec_config* cfg);
+
+/* Host-only integer logic of the budgets (paper: r < min(M,d), B_vis < M <= N).  `keep` is the
+ * requested B_vis (clamped to n).  Writes B_vis, M, r.  Returns COVSPEC_OK or COVSPEC_ERR_ARG. */
+int covspec_budgets(const covspec_config* cfg, int n, int keep, int* b_vis, int* m, int* r);
+
+/* Budgets of a whole problem: keep_offsets[batch+1] and presel_offsets[batch+1] (host, either may
+ * be NULL) receive the prefix sums of B_vis and M.  Launches nothing. */
+int covspec_plan_sizes(const covspec_config* cfg, const covspec_problem* p, int* keep_offsets,
+                       int* presel_offsets);
+
+/* Allocates the context and its device workspace for the capacities in cfg (the only allocation
+ * the library makes).  *out is NULL on failure.  Must be called with the target device current. */
+int covspec_prune_init(const covspec_config* cfg, covspec_ctx** out);
+int covspec_prune_destroy(covspec_ctx* ctx);
+/* Bytes of device workspace held by the context. */
+long long covspec_workspace_bytes(const covspec_ctx* ctx);
+
+/* Eq. 10-12.  Writes float32 device arrays of vis_offsets[batch] elements: s_query (Eq. 10),
+ * s_act (Eq. 11), s_fused (Eq. 12).  s_query and s_act may be NULL (kept in the workspace);
+ * s_fused is required. */
+int covspec_score(covspec_ctx* ctx, const covspec_problem* p, float* s_query, float* s_act,
+                  float* s_fused, void* stream);
+
+/* Preselection and low-rank redundancy reduction (Eq. 13-15) from a fused score.
+ *  s_fused       device [sum N_b] float32, as written by covspec_score
+ *  keep_idx      device [sum B_vis] int32: kept token indices, request-local, ascending
+ *  keep_offsets  host   [batch+1] (out, may be NULL): prefix sums of B_vis
+ *  presel_idx    device [sum M_b] int32 (out, may be NULL): the M preselected tokens, ascending
+ *  energy        device [sum M_b] float32 (out, may be NULL): c_i of Eq. 15 in presel order;
+ *                requests whose stage 2 is skipped (B_vis >= M) get zeros
+ * Ties in either selection: larger value first, then lower token index. */
+int covspec_select(covspec_ctx* ctx, const covspec_problem* p, const float* s_fused, int* keep_idx,
+                   int* keep_offsets, int* presel_idx, float* energy, void* stream);
+
+/* Gather of the survivors: out_hidden[keep_offsets[b] + k, :] = X[vis_offsets[b] + keep_idx[..], :]
+ * (bit copies, dtype of X), out_pos (device int32, may be NULL) = the same request-local indices.
+ * keep_offsets is the host array returned by covspec_select / covspec_plan_sizes. */
+int covspec_compact(covspec_ctx* ctx, const covspec_problem* p, const int* keep_idx,
+                    const int* keep_offsets, void* out_hidden, int* out_pos, void* stream);
+
+/* The whole path, Eq. 10 through the compacted buffer, in one call.  out_hidden device
+ * [sum B_vis, d]; keep_idx device [sum B_vis]; keep_offsets host [batch+1] (may be NULL). */
+int covspec_prune(covspec_ctx* ctx, const covspec_problem* p, void* out_hidden, int* keep_idx,
+                  int* keep_offsets, void* stream);
+
+/* Synchronises `stream`, returns the device status word (COVSPEC_OK, COVSPEC_ERR_NONFINITE or
+ * COVSPEC_ERR_NOCONVERGE) and clears it. */
+int covspec_get_device_status(covspec_ctx* ctx, void* stream);
+
+/* Number of kernels the last call on this context launched. */
+int covspec_last_launch_count(const covspec_ctx* ctx);
+
+/* Text of a covspec_status; for COVSPEC_ERR_CUDA, covspec_last_cuda_error gives the runtime's. */
+const char* covspec_strerror(int status);
+const char* covspec_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* COVSPEC_H_ */

@@ -1,0 +1,664 @@
+// Host runtime and C ABI of the covspec library: argument validation, budgets, the cached launch
+// plan, workspace carving and the kernel sequence of every entry point (see include/covspec.h).
+#include "covspec.h"
+
+#include <math.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <string>
+#include <vector>
+
+#include "common.cuh"
+#include "eig_kernels.cuh"
+#include "gemm_simt.cuh"
+#include "score_kernels.cuh"
+#include "select_kernels.cuh"
+
+using namespace covspec;
+
+namespace {
+
+thread_local std::string g_cuda_error;
+
+#define CUDA_TRY(expr)                                                                  \
+  do {                                                                                  \
+    cudaError_t e_ = (expr);                                                            \
+    if (e_ != cudaSuccess) {                                                            \
+      g_cuda_error = std::string(#expr) + ": " + cudaGetErrorString(e_);                \
+      return COVSPEC_ERR_CUDA;                                                          \
+    }                                                                                   \
+  } while (0)
+
+inline long long round_up(long long v, long long a) { return (v + a - 1) / a * a; }
+
+// Gemm tables kept on the device for the subspace iteration (one entry per stage-2 request).
+enum TableId {
+  T_GRAM_G = 0,   // G   = Zg Zg^T            (storage dtype operands)
+  T_MULG_01,      // U1  = U0 G
+  T_MULG_10,      // U0  = U1 G
+  T_GRAM_U1,      // B64 = U1 U1^T            (float64)
+  T_GRAM_U0,      // B64 = U0 U0^T
+  T_APPLY_10,     // U0  = Linv U1
+  T_APPLY_01,     // U1  = Linv U0
+  T_RR,           // S32 = U0 U1^T            (Rayleigh-Ritz matrix, U0 = U1 G)
+  T_RITZ,         // U0  = Wr U1              (Ritz vectors)
+  T_COUNT
+};
+
+struct Plan {
+  std::vector<int> vis_off, txt_off, keep;    // key of the cache
+  double keep_ratio = 0.0;
+  bool has_keep = false;
+  std::vector<ReqPlan> req;
+  std::vector<int> keep_offsets, presel_offsets;
+  int n_stage2 = 0;
+  int tiles[T_COUNT] = {0};
+  int t_max = 0, p_max = 0, m_max = 0;
+  long long total_vis = 0, total_txt = 0, total_keep = 0, total_presel = 0;
+  bool valid = false;
+};
+
+}  // namespace
+
+struct covspec_ctx {
+  covspec_config cfg;
+  int P = 0, hd = 0, heads = 0;          // embedding width, head width, head count (identity: 1 head)
+  int esize = 0;
+  char* ws = nullptr;                    // device workspace
+  long long ws_bytes = 0;
+  // carved regions
+  int* status = nullptr;
+  ReqPlan* d_plan = nullptr;
+  GemmProb* d_tables = nullptr;          // [T_COUNT][max_batch]
+  float* Qn = nullptr;
+  float* Kp = nullptr;
+  long long kp_rows = 0;
+  float *sq = nullptr, *sa = nullptr, *sf = nullptr;
+  int* presel = nullptr;
+  float* energy = nullptr;
+  void* Zg = nullptr;
+  float* G = nullptr;
+  long long g_cap = 0, u_cap = 0;
+  float *U0 = nullptr, *U1 = nullptr;
+  double* B64 = nullptr;
+  float *Linv = nullptr, *S32 = nullptr, *Wr = nullptr, *theta = nullptr;
+  // pinned staging for the plan upload
+  char* h_stage = nullptr;
+  long long stage_bytes = 0;
+  cudaEvent_t stage_free = nullptr;      // the previous upload has been consumed
+  Plan plan;
+  int launches = 0;
+};
+
+namespace {
+
+int budgets_impl(const covspec_config* cfg, int n, int keep, int* b, int* m, int* r) {
+  if (n < 1 || keep < 1) return COVSPEC_ERR_ARG;
+  int B = keep < n ? keep : n;
+  long long want = (long long)ceil((double)cfg->presel_factor * (double)B - 1e-9);
+  if (want < B) want = B;
+  int M = (int)(want < n ? want : n);
+  int R = (int)ceil((double)cfg->rank_frac * (double)B - 1e-9);
+  int cap = cfg->rank_cap;
+  if (M - 1 < cap) cap = M - 1;
+  if (cfg->d - 1 < cap) cap = cfg->d - 1;
+  if (R > cap) R = cap;
+  if (R < 1) R = 1;
+  *b = B; *m = M; *r = R;
+  return COVSPEC_OK;
+}
+
+int keep_of(const covspec_problem* p, int b, int n) {
+  if (p->keep) return p->keep[b];
+  int k = (int)ceil(p->keep_ratio * (double)n - 1e-6);
+  return k < 1 ? 1 : k;
+}
+
+int validate_cfg(const covspec_config* c) {
+  if (!c) return COVSPEC_ERR_ARG;
+  if (c->dtype != COVSPEC_F32 && c->dtype != COVSPEC_BF16) return COVSPEC_ERR_ARG;
+  if (c->d < 8 || c->d % 8) return COVSPEC_ERR_UNSUPPORTED;
+  if (c->n_heads < 0) return COVSPEC_ERR_ARG;
+  if (c->n_heads > 0 && c->head_dim != 128) return COVSPEC_ERR_UNSUPPORTED;
+  if (c->act_layers < 0 || c->act_layers + 1 > kMaxLayers) return COVSPEC_ERR_UNSUPPORTED;
+  if (!(c->lambda >= 0.f && c->lambda <= 1.f)) return COVSPEC_ERR_ARG;
+  if (c->norm_mode < 0 || c->norm_mode > 2 || c->head_reduce < 0 || c->head_reduce > 1)
+    return COVSPEC_ERR_ARG;
+  if (!(c->presel_factor >= 1.f) || !(c->rank_frac > 0.f) || c->rank_cap < 1) return COVSPEC_ERR_ARG;
+  if (c->eig_iters < 1 || c->eig_oversample < 0) return COVSPEC_ERR_ARG;
+  if (c->rank_cap + c->eig_oversample > kPMax) return COVSPEC_ERR_UNSUPPORTED;
+  return COVSPEC_OK;
+}
+
+int validate_problem(const covspec_config* c, const covspec_problem* p) {
+  if (!p || p->batch < 1 || !p->vis_offsets || !p->txt_offsets) return COVSPEC_ERR_ARG;
+  if (!p->keep && !(p->keep_ratio > 0.0 && p->keep_ratio <= 1.0)) return COVSPEC_ERR_ARG;
+  if (p->vis_offsets[0] != 0 || p->txt_offsets[0] != 0) return COVSPEC_ERR_SHAPE;
+  for (int b = 0; b < p->batch; ++b) {
+    if (p->vis_offsets[b + 1] <= p->vis_offsets[b]) return COVSPEC_ERR_SHAPE;   // N_b >= 1
+    if (p->txt_offsets[b + 1] <= p->txt_offsets[b]) return COVSPEC_ERR_SHAPE;   // T_b >= 1
+    if (p->keep && p->keep[b] < 1) return COVSPEC_ERR_SHAPE;
+  }
+  (void)c;
+  return COVSPEC_OK;
+}
+
+// Builds (or reuses) the launch plan and uploads it on `stream`.
+int get_plan(covspec_ctx* ctx, const covspec_problem* p, cudaStream_t stream) {
+  const covspec_config& cfg = ctx->cfg;
+  int st = validate_problem(&cfg, p);
+  if (st) return st;
+  Plan& pl = ctx->plan;
+  int B = p->batch;
+  bool same = pl.valid && (int)pl.req.size() == B && pl.has_keep == (p->keep != nullptr) &&
+              !memcmp(pl.vis_off.data(), p->vis_offsets, sizeof(int) * (B + 1)) &&
+              !memcmp(pl.txt_off.data(), p->txt_offsets, sizeof(int) * (B + 1)) &&
+              (p->keep ? !memcmp(pl.keep.data(), p->keep, sizeof(int) * B)
+                       : pl.keep_ratio == p->keep_ratio);
+  if (same) return COVSPEC_OK;
+  if (B > cfg.max_batch) return COVSPEC_ERR_WORKSPACE;
+  pl.valid = false;
+  pl.vis_off.assign(p->vis_offsets, p->vis_offsets + B + 1);
+  pl.txt_off.assign(p->txt_offsets, p->txt_offsets + B + 1);
+  pl.has_keep = p->keep != nullptr;
+  if (p->keep) pl.keep.assign(p->keep, p->keep + B);
+  pl.keep_ratio = p->keep_ratio;
+  pl.req.assign(B, ReqPlan{});
+  pl.keep_offsets.assign(B + 1, 0);
+  pl.presel_offsets.assign(B + 1, 0);
+  pl.n_stage2 = 0; pl.t_max = 0; pl.p_max = 0; pl.m_max = 0;
+  long long g_off = 0, u_off = 0;
+  int n_max = 0;
+  for (int b = 0; b < B; ++b) {
+    ReqPlan& r = pl.req[b];
+    r.vis_off = p->vis_offsets[b]; r.n = p->vis_offsets[b + 1] - r.vis_off;
+    r.txt_off = p->txt_offsets[b]; r.t = p->txt_offsets[b + 1] - r.txt_off;
+    st = budgets_impl(&cfg, r.n, keep_of(p, b, r.n), &r.b_vis, &r.m, &r.r);
+    if (st) return COVSPEC_ERR_SHAPE;
+    r.stage2 = r.b_vis < r.m;
+    r.p = 0;
+    if (r.stage2) {
+      r.p = r.r + cfg.eig_oversample;
+      if (r.p > r.m) r.p = r.m;
+      ++pl.n_stage2;
+    }
+    r.ldm = (int)round_up(r.m, 4);
+    r.keep_off = pl.keep_offsets[b]; r.presel_off = pl.presel_offsets[b];
+    pl.keep_offsets[b + 1] = r.keep_off + r.b_vis;
+    pl.presel_offsets[b + 1] = r.presel_off + r.m;
+    r.g_off = g_off; r.u_off = u_off;
+    if (r.stage2) { g_off += (long long)r.m * r.ldm; u_off += (long long)r.p * r.ldm; }
+    if (r.t > pl.t_max) pl.t_max = r.t;
+    if (r.p > pl.p_max) pl.p_max = r.p;
+    if (r.m > pl.m_max) pl.m_max = r.m;
+    if (r.n > n_max) n_max = r.n;
+  }
+  pl.total_vis = p->vis_offsets[B]; pl.total_txt = p->txt_offsets[B];
+  pl.total_keep = pl.keep_offsets[B]; pl.total_presel = pl.presel_offsets[B];
+  if (pl.total_vis > cfg.max_total_vis || pl.total_txt > cfg.max_total_txt ||
+      n_max > cfg.max_vis_per_req || g_off > ctx->g_cap || u_off > ctx->u_cap ||
+      pl.total_presel > ctx->cfg.max_total_presel)
+    return COVSPEC_ERR_WORKSPACE;
+
+  // Stage plan + gemm tables in pinned memory and upload.
+  if (ctx->stage_free) CUDA_TRY(cudaEventSynchronize(ctx->stage_free));
+  ReqPlan* h_plan = reinterpret_cast<ReqPlan*>(ctx->h_stage);
+  GemmProb* h_tab = reinterpret_cast<GemmProb*>(ctx->h_stage + round_up(sizeof(ReqPlan) * cfg.max_batch, 256));
+  memcpy(h_plan, pl.req.data(), sizeof(ReqPlan) * B);
+  int mb = cfg.max_batch;
+  for (int t = 0; t < T_COUNT; ++t) pl.tiles[t] = 0;
+  int s2 = 0;
+  char* Zg = reinterpret_cast<char*>(ctx->Zg);
+  for (int b = 0; b < B; ++b) {
+    const ReqPlan& r = pl.req[b];
+    if (!r.stage2) continue;
+    auto tiles_of = [](int m, int n, int* tn) {
+      *tn = (n + kGemmBN - 1) / kGemmBN;
+      return ((m + kGemmBM - 1) / kGemmBM) * *tn;
+    };
+    auto put = [&](int t, const void* A, const void* Bp, void* C, int m, int n, int k, int lda,
+                   int ldb, int ldc) {
+      GemmProb& g = h_tab[(size_t)t * mb + s2];
+      g.A = A; g.B = Bp; g.C = C; g.m = m; g.n = n; g.k = k; g.lda = lda; g.ldb = ldb; g.ldc = ldc;
+      g.tile_start = pl.tiles[t];
+      pl.tiles[t] += tiles_of(m, n, &g.tiles_n);
+    };
+    const void* zg = Zg + (size_t)r.presel_off * cfg.d * ctx->esize;
+    float* G = ctx->G + r.g_off;
+    float *U0 = ctx->U0 + r.u_off, *U1 = ctx->U1 + r.u_off;
+    double* B64 = ctx->B64 + (size_t)b * kPMax * kPMax;
+    float* Linv = ctx->Linv + (size_t)b * kPMax * kPMax;
+    float* S32 = ctx->S32 + (size_t)b * kPMax * kPMax;
+    float* Wr = ctx->Wr + (size_t)b * kPMax * kPMax;
+    int ldp = (int)round_up(r.p, 4);
+    put(T_GRAM_G, zg, zg, G, r.m, r.m, cfg.d, cfg.d, cfg.d, r.ldm);
+    put(T_MULG_01, U0, G, U1, r.p, r.m, r.m, r.ldm, r.ldm, r.ldm);
+    put(T_MULG_10, U1, G, U0, r.p, r.m, r.m, r.ldm, r.ldm, r.ldm);
+    put(T_GRAM_U1, U1, U1, B64, r.p, r.p, r.m, r.ldm, r.ldm, kPMax);
+    put(T_GRAM_U0, U0, U0, B64, r.p, r.p, r.m, r.ldm, r.ldm, kPMax);
+    put(T_APPLY_10, Linv, U1, U0, r.p, r.m, r.p, ldp, r.ldm, r.ldm);
+    put(T_APPLY_01, Linv, U0, U1, r.p, r.m, r.p, ldp, r.ldm, r.ldm);
+    put(T_RR, U0, U1, S32, r.p, r.p, r.m, r.ldm, r.ldm, ldp);
+    put(T_RITZ, Wr, U1, U0, r.r, r.m, r.p, ldp, r.ldm, r.ldm);
+    ++s2;
+  }
+  CUDA_TRY(cudaMemcpyAsync(ctx->d_plan, h_plan, sizeof(ReqPlan) * B, cudaMemcpyHostToDevice, stream));
+  if (s2 > 0)
+    CUDA_TRY(cudaMemcpyAsync(ctx->d_tables, h_tab, sizeof(GemmProb) * (size_t)T_COUNT * mb,
+                             cudaMemcpyHostToDevice, stream));
+  CUDA_TRY(cudaEventRecord(ctx->stage_free, stream));
+  pl.valid = true;
+  return COVSPEC_OK;
+}
+
+#define LAUNCH_CHECK(ctx)                               \
+  do {                                                  \
+    ++(ctx)->launches;                                  \
+    CUDA_TRY(cudaGetLastError());                       \
+  } while (0)
+
+template <typename TA, typename TB, typename AccT, typename TC, bool B_KN>
+int launch_table(covspec_ctx* ctx, int table, int lower_only, cudaStream_t s) {
+  int tiles = ctx->plan.tiles[table];
+  if (tiles == 0) return COVSPEC_OK;
+  gemm_simt_kernel<TA, TB, AccT, TC, B_KN><<<tiles, 256, 0, s>>>(
+      ctx->d_tables + (size_t)table * ctx->cfg.max_batch, ctx->plan.n_stage2, GemmProb{}, lower_only);
+  LAUNCH_CHECK(ctx);
+  return COVSPEC_OK;
+}
+
+template <typename T>
+int launch_single_nt(covspec_ctx* ctx, const T* A, const T* B, float* C, int m, int n, int k, int lda,
+                     int ldb, int ldc, cudaStream_t s) {
+  GemmProb g{};
+  g.A = A; g.B = B; g.C = C; g.m = m; g.n = n; g.k = k; g.lda = lda; g.ldb = ldb; g.ldc = ldc;
+  g.tile_start = 0;
+  g.tiles_n = (n + kGemmBN - 1) / kGemmBN;
+  int tiles = ((m + kGemmBM - 1) / kGemmBM) * g.tiles_n;
+  gemm_simt_kernel<T, T, float, float, false><<<tiles, 256, 0, s>>>(nullptr, 0, g, 0);
+  LAUNCH_CHECK(ctx);
+  return COVSPEC_OK;
+}
+
+// ---- Eq. 10-12 -------------------------------------------------------------------------------
+template <typename T>
+int score_impl(covspec_ctx* ctx, const covspec_problem* p, float* s_query, float* s_act,
+               float* s_fused, bool do_fuse, cudaStream_t s) {
+  const covspec_config& cfg = ctx->cfg;
+  const Plan& pl = ctx->plan;
+  int B = p->batch;
+  int rowsQ = (int)pl.total_txt;
+  long long rowsX = pl.total_vis;
+  const T* X = reinterpret_cast<const T*>(p->X);
+  const T* Q = reinterpret_cast<const T*>(p->Q);
+  int P = ctx->P, hd = ctx->hd, H = ctx->heads;
+  if (!s_query) s_query = ctx->sq;
+  if (!s_act) s_act = ctx->sa;
+  bool identity = cfg.n_heads == 0;
+  if (identity) {
+    int warps = rowsQ * H;
+    qnorm_kernel<T><<<(warps + 7) / 8, 256, 0, s>>>(Q, ctx->Qn, rowsQ, H, hd);
+    LAUNCH_CHECK(ctx);
+  } else {
+    int st = launch_single_nt<T>(ctx, Q, reinterpret_cast<const T*>(p->Wq), ctx->Qn, rowsQ, P, cfg.d,
+                                 cfg.d, cfg.d, P, s);
+    if (st) return st;
+    int warps = rowsQ * H;
+    qnorm_kernel<float><<<(warps + 7) / 8, 256, 0, s>>>(ctx->Qn, ctx->Qn, rowsQ, H, hd);
+    LAUNCH_CHECK(ctx);
+  }
+  int mean = cfg.head_reduce == 1;
+  size_t smem = mean ? (size_t)8 * pl.t_max * sizeof(float) : 0;
+  if (smem > 48 * 1024) return COVSPEC_ERR_UNSUPPORTED;
+  if (identity) {
+    cosmax_kernel<T><<<(unsigned)((rowsX + 7) / 8), 256, smem, s>>>(
+        X, ctx->Qn, ctx->d_plan, B, 0, (int)rowsX, H, hd, mean, pl.t_max, s_query);
+    LAUNCH_CHECK(ctx);
+  } else {
+    for (long long r0 = 0; r0 < rowsX; r0 += ctx->kp_rows) {
+      int rows = (int)((rowsX - r0) < ctx->kp_rows ? (rowsX - r0) : ctx->kp_rows);
+      int st = launch_single_nt<T>(ctx, X + (size_t)r0 * cfg.d, reinterpret_cast<const T*>(p->Wk),
+                                   ctx->Kp, rows, P, cfg.d, cfg.d, cfg.d, P, s);
+      if (st) return st;
+      cosmax_kernel<float><<<(rows + 7) / 8, 256, smem, s>>>(ctx->Kp, ctx->Qn, ctx->d_plan, B, (int)r0,
+                                                             rows, H, hd, mean, pl.t_max, s_query);
+      LAUNCH_CHECK(ctx);
+    }
+  }
+  if (cfg.act_layers > 0) {
+    LayerPtrs lp{};
+    for (int l = 0; l <= cfg.act_layers; ++l) lp.h[l] = p->Hs[l];
+    unsigned grid = (unsigned)((rowsX + 7) / 8);
+    if (cfg.act_layers <= 4)
+      activity_kernel<T, 4><<<grid, 256, 0, s>>>(lp, cfg.act_layers, rowsX, cfg.d, s_act);
+    else if (cfg.act_layers <= 8)
+      activity_kernel<T, 8><<<grid, 256, 0, s>>>(lp, cfg.act_layers, rowsX, cfg.d, s_act);
+    else
+      activity_kernel<T, 16><<<grid, 256, 0, s>>>(lp, cfg.act_layers, rowsX, cfg.d, s_act);
+    LAUNCH_CHECK(ctx);
+  }
+  if (do_fuse) {
+    fuse_kernel<<<B, 1024, 0, s>>>(s_query, cfg.act_layers > 0 ? s_act : nullptr, ctx->d_plan,
+                                   cfg.lambda, cfg.norm_mode, s_fused, ctx->status);
+    LAUNCH_CHECK(ctx);
+  }
+  return COVSPEC_OK;
+}
+
+// ---- preselect, Eq. 13-15, final select ---------------------------------------------------------
+template <typename T>
+int select_impl(covspec_ctx* ctx, const covspec_problem* p, const float* s_fused, int* keep_idx,
+                int* presel_out, float* energy_out, cudaStream_t s) {
+  const covspec_config& cfg = ctx->cfg;
+  const Plan& pl = ctx->plan;
+  int B = p->batch;
+  int* presel = presel_out ? presel_out : ctx->presel;
+  float* energy = energy_out ? energy_out : ctx->energy;
+  preselect_kernel<<<B, 1024, 0, s>>>(s_fused, ctx->d_plan, presel, ctx->status);
+  LAUNCH_CHECK(ctx);
+  if (pl.n_stage2 > 0) {
+    int vec16 = cfg.d * ctx->esize / 16;
+    gather_rows_kernel<<<(unsigned)pl.total_presel, 256, 0, s>>>(
+        reinterpret_cast<const uint4*>(p->X), presel, ctx->d_plan, B, 1, vec16,
+        reinterpret_cast<uint4*>(ctx->Zg), nullptr);
+    LAUNCH_CHECK(ctx);
+    int st = launch_table<T, T, float, float, false>(ctx, T_GRAM_G, 1, s);
+    if (st) return st;
+    int init_blocks = (pl.p_max * (pl.m_max + 3) + 255) / 256;
+    dim3 gi(init_blocks > 64 ? 64 : init_blocks, B);
+    eig_init_kernel<<<gi, 256, 0, s>>>(ctx->d_plan, ctx->U0);
+    LAUNCH_CHECK(ctx);
+    size_t chol_smem = ((size_t)pl.p_max * pl.p_max + 2 * pl.p_max) * sizeof(double);
+    size_t jac_smem = (size_t)2 * pl.p_max * (pl.p_max + 1) * sizeof(float) +
+                      (size_t)4 * ((pl.p_max + 1) / 2 + 1) * sizeof(float);
+    for (int it = 0; it < cfg.eig_iters; ++it) {
+      // U1 = U0 G ; orthonormalise rows of U1 into U0
+      if ((st = launch_table<float, float, float, float, false>(ctx, T_MULG_01, 0, s))) return st;
+      if ((st = launch_table<float, float, double, double, false>(ctx, T_GRAM_U1, 0, s))) return st;
+      chol_inv_kernel<<<B, 1024, chol_smem, s>>>(ctx->d_plan, ctx->B64, ctx->Linv);
+      LAUNCH_CHECK(ctx);
+      if ((st = launch_table<float, float, float, float, true>(ctx, T_APPLY_10, 0, s))) return st;
+    }
+    // second Cholesky-QR pass for an orthonormal basis: U1 = orth(U0)
+    if ((st = launch_table<float, float, double, double, false>(ctx, T_GRAM_U0, 0, s))) return st;
+    chol_inv_kernel<<<B, 1024, chol_smem, s>>>(ctx->d_plan, ctx->B64, ctx->Linv);
+    LAUNCH_CHECK(ctx);
+    if ((st = launch_table<float, float, float, float, true>(ctx, T_APPLY_01, 0, s))) return st;
+    // Rayleigh-Ritz: U0 = U1 G, S = U0 U1^T, eig(S), Ritz vectors U0 = Wr U1
+    if ((st = launch_table<float, float, float, float, false>(ctx, T_MULG_10, 0, s))) return st;
+    if ((st = launch_table<float, float, float, float, false>(ctx, T_RR, 0, s))) return st;
+    jacobi_kernel<<<B, 1024, jac_smem, s>>>(ctx->d_plan, ctx->S32, ctx->Wr, ctx->theta, 30, ctx->status);
+    LAUNCH_CHECK(ctx);
+    if ((st = launch_table<float, float, float, float, true>(ctx, T_RITZ, 0, s))) return st;
+  }
+  dim3 ge((pl.m_max + 255) / 256, B);
+  energy_kernel<<<ge, 256, 0, s>>>(ctx->d_plan, ctx->U0, ctx->theta, energy);
+  LAUNCH_CHECK(ctx);
+  final_select_kernel<<<B, 1024, 0, s>>>(energy, presel, ctx->d_plan, keep_idx, ctx->status);
+  LAUNCH_CHECK(ctx);
+  return COVSPEC_OK;
+}
+
+int compact_impl(covspec_ctx* ctx, const covspec_problem* p, const int* keep_idx, void* out,
+                 int* out_pos, cudaStream_t s) {
+  const Plan& pl = ctx->plan;
+  int vec16 = ctx->cfg.d * ctx->esize / 16;
+  gather_rows_kernel<<<(unsigned)pl.total_keep, 256, 0, s>>>(
+      reinterpret_cast<const uint4*>(p->X), keep_idx, ctx->d_plan, p->batch, 0, vec16,
+      reinterpret_cast<uint4*>(out), out_pos);
+  LAUNCH_CHECK(ctx);
+  return COVSPEC_OK;
+}
+
+int check_score_args(const covspec_ctx* ctx, const covspec_problem* p) {
+  if (!p->X || !p->Q) return COVSPEC_ERR_ARG;
+  if (ctx->cfg.n_heads > 0 && (!p->Wq || !p->Wk)) return COVSPEC_ERR_ARG;
+  if (ctx->cfg.act_layers > 0) {
+    if (!p->Hs) return COVSPEC_ERR_ARG;
+    for (int l = 0; l <= ctx->cfg.act_layers; ++l) if (!p->Hs[l]) return COVSPEC_ERR_ARG;
+  }
+  return COVSPEC_OK;
+}
+
+void copy_offsets(const Plan& pl, int* keep_offsets) {
+  if (keep_offsets) memcpy(keep_offsets, pl.keep_offsets.data(), sizeof(int) * pl.keep_offsets.size());
+}
+
+}  // namespace
+
+// ================================================================================================
+extern "C" {
+
+void covspec_default_config(covspec_config* c) {
+  if (!c) return;
+  memset(c, 0, sizeof(*c));
+  c->dtype = COVSPEC_BF16;
+  c->head_dim = 128;
+  c->act_layers = 4;
+  c->lambda = 0.5f;
+  c->norm_mode = 0;
+  c->head_reduce = 0;
+  c->presel_factor = 2.0f;
+  c->rank_frac = 0.5f;
+  c->rank_cap = 128;
+  c->eig_iters = 6;
+  c->eig_oversample = 32;
+}
+
+int covspec_budgets(const covspec_config* cfg, int n, int keep, int* b_vis, int* m, int* r) {
+  if (!cfg || !b_vis || !m || !r) return COVSPEC_ERR_ARG;
+  return budgets_impl(cfg, n, keep, b_vis, m, r);
+}
+
+int covspec_plan_sizes(const covspec_config* cfg, const covspec_problem* p, int* keep_offsets,
+                       int* presel_offsets) {
+  if (!cfg) return COVSPEC_ERR_ARG;
+  int st = validate_problem(cfg, p);
+  if (st) return st;
+  int ko = 0, po = 0;
+  if (keep_offsets) keep_offsets[0] = 0;
+  if (presel_offsets) presel_offsets[0] = 0;
+  for (int b = 0; b < p->batch; ++b) {
+    int n = p->vis_offsets[b + 1] - p->vis_offsets[b], B, M, R;
+    if (budgets_impl(cfg, n, keep_of(p, b, n), &B, &M, &R)) return COVSPEC_ERR_SHAPE;
+    ko += B; po += M;
+    if (keep_offsets) keep_offsets[b + 1] = ko;
+    if (presel_offsets) presel_offsets[b + 1] = po;
+  }
+  return COVSPEC_OK;
+}
+
+int covspec_prune_init(const covspec_config* cfg, covspec_ctx** out) {
+  if (!out) return COVSPEC_ERR_ARG;
+  *out = nullptr;
+  int st = validate_cfg(cfg);
+  if (st) return st;
+  if (cfg->max_batch < 1 || cfg->max_total_vis < 1 || cfg->max_total_txt < 1 || cfg->max_vis_per_req < 1)
+    return COVSPEC_ERR_ARG;
+  covspec_ctx* ctx = new covspec_ctx();
+  ctx->cfg = *cfg;
+  covspec_config& c = ctx->cfg;
+  if (c.max_presel_per_req <= 0) c.max_presel_per_req = c.max_vis_per_req;
+  if (c.max_total_presel <= 0) c.max_total_presel = c.max_total_vis;
+  ctx->esize = c.dtype == COVSPEC_BF16 ? 2 : 4;
+  ctx->heads = c.n_heads > 0 ? c.n_heads : 1;
+  ctx->hd = c.n_heads > 0 ? c.head_dim : c.d;
+  ctx->P = ctx->heads * ctx->hd;
+  // projection chunk: keep the float32 embedding of a chunk within ~64 MB so it stays in L2
+  long long rows = (64ll << 20) / ((long long)ctx->P * 4);
+  rows = rows < 256 ? 256 : rows / 64 * 64;
+  if (rows > c.max_total_vis) rows = round_up(c.max_total_vis, 64);
+  ctx->kp_rows = c.n_heads > 0 ? rows : 0;
+  long long ldm_max = round_up(c.max_presel_per_req, 4);
+  ctx->g_cap = (c.max_total_presel + 4ll * c.max_batch) * ldm_max;
+  ctx->u_cap = (long long)kPMax * (c.max_total_presel + 4ll * c.max_batch);
+
+  long long off = 0;
+  auto carve = [&](long long bytes) { long long o = off; off += round_up(bytes, 256); return o; };
+  long long o_status = carve(256);
+  long long o_plan = carve(sizeof(ReqPlan) * c.max_batch);
+  long long o_tab = carve(sizeof(GemmProb) * (long long)T_COUNT * c.max_batch);
+  long long o_qn = carve(4ll * c.max_total_txt * ctx->P);
+  long long o_kp = carve(4ll * ctx->kp_rows * ctx->P);
+  long long o_sq = carve(4ll * c.max_total_vis), o_sa = carve(4ll * c.max_total_vis);
+  long long o_sf = carve(4ll * c.max_total_vis);
+  long long o_presel = carve(4ll * c.max_total_presel), o_energy = carve(4ll * c.max_total_presel);
+  long long o_zg = carve((long long)ctx->esize * c.max_total_presel * c.d);
+  long long o_g = carve(4ll * ctx->g_cap);
+  long long o_u0 = carve(4ll * ctx->u_cap), o_u1 = carve(4ll * ctx->u_cap);
+  long long small = (long long)c.max_batch * kPMax * kPMax;
+  long long o_b64 = carve(8ll * small), o_linv = carve(4ll * small), o_s32 = carve(4ll * small);
+  long long o_wr = carve(4ll * small), o_theta = carve(4ll * c.max_batch * kPMax);
+  ctx->ws_bytes = off;
+  cudaError_t e = cudaMalloc(&ctx->ws, (size_t)off);
+  if (e != cudaSuccess) {
+    g_cuda_error = std::string("cudaMalloc workspace: ") + cudaGetErrorString(e);
+    delete ctx;
+    return COVSPEC_ERR_CUDA;
+  }
+  char* w = ctx->ws;
+  ctx->status = reinterpret_cast<int*>(w + o_status);
+  ctx->d_plan = reinterpret_cast<ReqPlan*>(w + o_plan);
+  ctx->d_tables = reinterpret_cast<GemmProb*>(w + o_tab);
+  ctx->Qn = reinterpret_cast<float*>(w + o_qn);
+  ctx->Kp = reinterpret_cast<float*>(w + o_kp);
+  ctx->sq = reinterpret_cast<float*>(w + o_sq);
+  ctx->sa = reinterpret_cast<float*>(w + o_sa);
+  ctx->sf = reinterpret_cast<float*>(w + o_sf);
+  ctx->presel = reinterpret_cast<int*>(w + o_presel);
+  ctx->energy = reinterpret_cast<float*>(w + o_energy);
+  ctx->Zg = w + o_zg;
+  ctx->G = reinterpret_cast<float*>(w + o_g);
+  ctx->U0 = reinterpret_cast<float*>(w + o_u0);
+  ctx->U1 = reinterpret_cast<float*>(w + o_u1);
+  ctx->B64 = reinterpret_cast<double*>(w + o_b64);
+  ctx->Linv = reinterpret_cast<float*>(w + o_linv);
+  ctx->S32 = reinterpret_cast<float*>(w + o_s32);
+  ctx->Wr = reinterpret_cast<float*>(w + o_wr);
+  ctx->theta = reinterpret_cast<float*>(w + o_theta);
+  ctx->stage_bytes = round_up(sizeof(ReqPlan) * c.max_batch, 256) +
+                     sizeof(GemmProb) * (long long)T_COUNT * c.max_batch;
+  bool ok = cudaMemset(ctx->status, 0, 256) == cudaSuccess &&
+            cudaMallocHost(&ctx->h_stage, (size_t)ctx->stage_bytes) == cudaSuccess &&
+            cudaEventCreateWithFlags(&ctx->stage_free, cudaEventDisableTiming) == cudaSuccess;
+  // the small dense kernels need more than the default 48 KB of dynamic shared memory
+  ok = ok && cudaFuncSetAttribute(chol_inv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                  (int)(((size_t)kPMax * kPMax + 2 * kPMax) * sizeof(double))) == cudaSuccess;
+  ok = ok && cudaFuncSetAttribute(jacobi_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                  (int)((size_t)2 * kPMax * (kPMax + 1) * 4 + 4 * (kPMax / 2 + 2) * 4)) == cudaSuccess;
+  if (!ok) {
+    g_cuda_error = std::string("context set-up: ") + cudaGetErrorString(cudaGetLastError());
+    covspec_prune_destroy(ctx);
+    return COVSPEC_ERR_CUDA;
+  }
+  *out = ctx;
+  return COVSPEC_OK;
+}
+
+int covspec_prune_destroy(covspec_ctx* ctx) {
+  if (!ctx) return COVSPEC_ERR_ARG;
+  if (ctx->ws) cudaFree(ctx->ws);
+  if (ctx->h_stage) cudaFreeHost(ctx->h_stage);
+  if (ctx->stage_free) cudaEventDestroy(ctx->stage_free);
+  delete ctx;
+  return COVSPEC_OK;
+}
+
+long long covspec_workspace_bytes(const covspec_ctx* ctx) { return ctx ? ctx->ws_bytes : 0; }
+
+int covspec_score(covspec_ctx* ctx, const covspec_problem* p, float* s_query, float* s_act,
+                  float* s_fused, void* stream) {
+  if (!ctx || !p || !s_fused) return COVSPEC_ERR_ARG;
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  int st = validate_problem(&ctx->cfg, p);
+  if (st) return st;
+  if ((st = check_score_args(ctx, p))) return st;
+  ctx->launches = 0;
+  if ((st = get_plan(ctx, p, s))) return st;
+  return ctx->cfg.dtype == COVSPEC_BF16
+             ? score_impl<__nv_bfloat16>(ctx, p, s_query, s_act, s_fused, true, s)
+             : score_impl<float>(ctx, p, s_query, s_act, s_fused, true, s);
+}
+
+int covspec_select(covspec_ctx* ctx, const covspec_problem* p, const float* s_fused, int* keep_idx,
+                   int* keep_offsets, int* presel_idx, float* energy, void* stream) {
+  if (!ctx || !p || !s_fused || !keep_idx || !p->X) return COVSPEC_ERR_ARG;
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  ctx->launches = 0;
+  int st = get_plan(ctx, p, s);
+  if (st) return st;
+  copy_offsets(ctx->plan, keep_offsets);
+  return ctx->cfg.dtype == COVSPEC_BF16
+             ? select_impl<__nv_bfloat16>(ctx, p, s_fused, keep_idx, presel_idx, energy, s)
+             : select_impl<float>(ctx, p, s_fused, keep_idx, presel_idx, energy, s);
+}
+
+int covspec_compact(covspec_ctx* ctx, const covspec_problem* p, const int* keep_idx,
+                    const int* keep_offsets, void* out_hidden, int* out_pos, void* stream) {
+  if (!ctx || !p || !keep_idx || !keep_offsets || !out_hidden || !p->X) return COVSPEC_ERR_ARG;
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  ctx->launches = 0;
+  int st = get_plan(ctx, p, s);
+  if (st) return st;
+  if (memcmp(keep_offsets, ctx->plan.keep_offsets.data(), sizeof(int) * (p->batch + 1)))
+    return COVSPEC_ERR_SHAPE;
+  return compact_impl(ctx, p, keep_idx, out_hidden, out_pos, s);
+}
+
+int covspec_prune(covspec_ctx* ctx, const covspec_problem* p, void* out_hidden, int* keep_idx,
+                  int* keep_offsets, void* stream) {
+  if (!ctx || !p || !out_hidden || !keep_idx) return COVSPEC_ERR_ARG;
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  int st = validate_problem(&ctx->cfg, p);
+  if (st) return st;
+  if ((st = check_score_args(ctx, p))) return st;
+  ctx->launches = 0;
+  if ((st = get_plan(ctx, p, s))) return st;
+  copy_offsets(ctx->plan, keep_offsets);
+  bool bf = ctx->cfg.dtype == COVSPEC_BF16;
+  float* fused = ctx->sf;
+  st = bf ? score_impl<__nv_bfloat16>(ctx, p, nullptr, nullptr, fused, false, s)
+          : score_impl<float>(ctx, p, nullptr, nullptr, fused, false, s);
+  if (st) return st;
+  fuse_kernel<<<p->batch, 1024, 0, s>>>(ctx->sq, ctx->cfg.act_layers > 0 ? ctx->sa : nullptr,
+                                        ctx->d_plan, ctx->cfg.lambda, ctx->cfg.norm_mode, fused,
+                                        ctx->status);
+  LAUNCH_CHECK(ctx);
+  st = bf ? select_impl<__nv_bfloat16>(ctx, p, fused, keep_idx, nullptr, nullptr, s)
+          : select_impl<float>(ctx, p, fused, keep_idx, nullptr, nullptr, s);
+  if (st) return st;
+  return compact_impl(ctx, p, keep_idx, out_hidden, nullptr, s);
+}
+
+int covspec_get_device_status(covspec_ctx* ctx, void* stream) {
+  if (!ctx) return COVSPEC_ERR_ARG;
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  int h = 0;
+  CUDA_TRY(cudaMemcpyAsync(&h, ctx->status, sizeof(int), cudaMemcpyDeviceToHost, s));
+  CUDA_TRY(cudaMemsetAsync(ctx->status, 0, sizeof(int), s));
+  CUDA_TRY(cudaStreamSynchronize(s));
+  if (h & kStatusNonFinite) return COVSPEC_ERR_NONFINITE;
+  if (h & kStatusNoConverge) return COVSPEC_ERR_NOCONVERGE;
+  return COVSPEC_OK;
+}
+
+int covspec_last_launch_count(const covspec_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+const char* covspec_strerror(int status) {
+  switch (status) {
+    case COVSPEC_OK: return "ok";
+    case COVSPEC_ERR_ARG: return "invalid argument";
+    case COVSPEC_ERR_SHAPE: return "invalid shape (offsets, empty request or budget)";
+    case COVSPEC_ERR_UNSUPPORTED: return "unsupported configuration";
+    case COVSPEC_ERR_WORKSPACE: return "problem exceeds the workspace capacities given at init";
+    case COVSPEC_ERR_CUDA: return "CUDA runtime error";
+    case COVSPEC_ERR_NONFINITE: return "non-finite score on the device";
+    case COVSPEC_ERR_NOCONVERGE: return "small eigen-solve did not converge";
+    default: return "unknown status";
+  }
+}
+
+const char* covspec_last_cuda_error(void) { return g_cuda_error.c_str(); }
+
+}  // extern "C"

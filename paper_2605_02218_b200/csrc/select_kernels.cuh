@@ -1,0 +1,145 @@
+// Segmented top-k selection (preselect the M best fused scores; keep the B_vis largest energies)
+// and the row gather used for Z_M (Eq. 13) and for the compacted output.
+#pragma once
+#include "common.cuh"
+
+namespace covspec {
+
+// Monotone map float -> uint32 (larger float = larger key).  -0 is folded onto +0 so that equal
+// values share a key; NaN maps to the smallest key.
+__device__ __forceinline__ unsigned order_key(float v) {
+  if (v != v) return 0u;
+  v += 0.0f;
+  unsigned u = __float_as_uint(v);
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+// Block-wide exclusive scan of a small packed counter (blockDim.x multiple of 32, <= 1024).
+// Returns the exclusive prefix; *total receives the block sum.
+__device__ __forceinline__ unsigned block_exclusive_scan(unsigned v, unsigned* warp_tot,
+                                                         unsigned* total) {
+  int lane = threadIdx.x & 31, w = threadIdx.x >> 5, nw = blockDim.x >> 5;
+  unsigned inc = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    unsigned t = __shfl_up_sync(0xffffffffu, inc, o);
+    if (lane >= o) inc += t;
+  }
+  __syncthreads();
+  if (lane == 31) warp_tot[w] = inc;
+  __syncthreads();
+  if (w == 0) {
+    unsigned t = lane < nw ? warp_tot[lane] : 0u, ti = t;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      unsigned u = __shfl_up_sync(0xffffffffu, ti, o);
+      if (lane >= o) ti += u;
+    }
+    if (lane < nw) warp_tot[lane] = ti - t;   // exclusive warp offsets
+    if (lane == 31) warp_tot[32] = ti;        // block total
+  }
+  __syncthreads();
+  *total = warp_tot[32];
+  return warp_tot[w] + inc - v;
+}
+
+// Top-k of keys[0..n) by an 8-bit-per-pass radix select on the ordered keys, then an ordered
+// emission: every element above the k-th value, plus the lowest-index elements equal to it until k
+// are taken.  out[0..k) receives the selected positions in ascending order, mapped through `remap`
+// when given.  `all_equal` treats every key as equal (selects the first k positions).
+__device__ void block_topk(const float* __restrict__ keys, int n, int k, bool all_equal,
+                           const int* __restrict__ remap, int* __restrict__ out, int* status) {
+  __shared__ unsigned hist[256];
+  __shared__ unsigned sel_prefix, sel_k;
+  __shared__ unsigned warp_tot[33];
+  unsigned prefix = 0u, mask = 0u, kk = (unsigned)k;
+  if (!all_equal) {
+    bool bad = false;
+    for (int shift = 24; shift >= 0; shift -= 8) {
+      for (int i = threadIdx.x; i < 256; i += blockDim.x) hist[i] = 0u;
+      __syncthreads();
+      for (int i = threadIdx.x; i < n; i += blockDim.x) {
+        float v = keys[i];
+        if (shift == 24) bad |= !(fabsf(v) <= 3.402823466e38f);
+        unsigned key = order_key(v);
+        if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
+      }
+      __syncthreads();
+      if (threadIdx.x == 0) {
+        unsigned c = 0u;
+        int bin = 255;
+        for (; bin > 0; --bin) {
+          if (c + hist[bin] >= kk) break;
+          c += hist[bin];
+        }
+        sel_prefix = prefix | ((unsigned)bin << shift);
+        sel_k = kk - c;
+      }
+      __syncthreads();
+      prefix = sel_prefix;
+      kk = sel_k;
+      mask |= 255u << shift;
+    }
+    if (bad) atomicOr(status, kStatusNonFinite);
+  }
+  // Ordered emission.  kk = how many elements equal to the threshold are taken.
+  unsigned run_gt = 0u, run_eq = 0u;
+  for (int base = 0; base < n; base += blockDim.x) {
+    int i = base + threadIdx.x;
+    unsigned gt = 0u, eq = 0u;
+    if (i < n) {
+      if (all_equal) eq = 1u;
+      else {
+        unsigned key = order_key(keys[i]);
+        gt = key > prefix; eq = key == prefix;
+      }
+    }
+    unsigned tot;
+    unsigned ex = block_exclusive_scan(gt | (eq << 16), warp_tot, &tot);
+    unsigned gt_before = run_gt + (ex & 0xffffu), eq_before = run_eq + (ex >> 16);
+    if (gt || (eq && eq_before < kk)) {
+      unsigned pos = gt_before + min(eq_before, kk);
+      out[pos] = remap ? remap[i] : i;
+    }
+    run_gt += tot & 0xffffu;
+    run_eq += tot >> 16;
+  }
+}
+
+// Preselection: one block per request, the M best fused scores -> presel (ascending token index).
+__global__ void __launch_bounds__(1024)
+preselect_kernel(const float* __restrict__ s_fused, const ReqPlan* __restrict__ plan,
+                 int* __restrict__ presel, int* status) {
+  ReqPlan rp = plan[blockIdx.x];
+  block_topk(s_fused + rp.vis_off, rp.n, rp.m, false, nullptr, presel + rp.presel_off, status);
+}
+
+// Final selection: one block per request, the B_vis largest energies among the M preselected
+// tokens -> keep_idx (token indices, ascending).  Requests whose stage 2 is skipped keep their
+// whole preselected set (B_vis == M).
+__global__ void __launch_bounds__(1024)
+final_select_kernel(const float* __restrict__ energy, const int* __restrict__ presel,
+                    const ReqPlan* __restrict__ plan, int* __restrict__ keep_idx, int* status) {
+  ReqPlan rp = plan[blockIdx.x];
+  block_topk(energy + rp.presel_off, rp.m, rp.b_vis, rp.stage2 == 0, presel + rp.presel_off,
+             keep_idx + rp.keep_off, status);
+}
+
+// out[row, :] = src[vis_off(b) + idx[row], :] as 16-byte vectors; one block per output row.
+// `use_presel` selects which plan offsets delimit the rows of a request (presel_off / keep_off).
+__global__ void __launch_bounds__(256)
+gather_rows_kernel(const uint4* __restrict__ src, const int* __restrict__ idx,
+                   const ReqPlan* __restrict__ plan, int batch, int use_presel, int row_vec16,
+                   uint4* __restrict__ dst, int* __restrict__ out_pos) {
+  int row = blockIdx.x;
+  int b = find_request(row, batch, [&](int q) {
+    return use_presel ? plan[q].presel_off : plan[q].keep_off;
+  });
+  int tok = idx[row];
+  const uint4* s = src + ((size_t)plan[b].vis_off + tok) * row_vec16;
+  uint4* d = dst + (size_t)row * row_vec16;
+  for (int v = threadIdx.x; v < row_vec16; v += blockDim.x) d[v] = s[v];
+  if (out_pos != nullptr && threadIdx.x == 0) out_pos[row] = tok;
+}
+
+}  // namespace covspec

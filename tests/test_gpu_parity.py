@@ -1,0 +1,142 @@
+"""Parity of the CUDA path (through the C ABI) with the CPU oracle, element by element on seeded
+inputs: small shapes that span several tiles with ragged tails, the degenerate cases, and the
+named configurations."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2605_02218_b200 import workloads
+from tests import parity
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    from paper_2605_02218_b200 import build
+    build.build()
+
+
+def _report(name, stats):
+    print(f"\n[parity] {name}: " + ", ".join(f"{k}={v:.3g}" if isinstance(v, float) else f"{k}={v}"
+                                             for k, v in sorted(stats.items())))
+
+
+SMALL = [
+    # identity embedding, fp32 and bf16, odd sizes
+    dict(seed=11, dtype=torch.float32, batch=3, n_vis=(50, 300), n_txt=(1, 9), d=72, n_heads=0,
+         rank=8, keep_ratio=0.3),
+    dict(seed=12, dtype=torch.bfloat16, batch=4, n_vis=(100, 700), n_txt=(3, 40), d=264, n_heads=0,
+         rank=16, keep_ratio=0.2),
+    # projection heads, ragged, tails that are not multiples of any tile
+    dict(seed=13, dtype=torch.bfloat16, batch=5, n_vis=(65, 900), n_txt=(1, 70), d=136, n_heads=3,
+         rank=12, keep_ratio=0.25),
+    dict(seed=14, dtype=torch.float32, batch=2, n_vis=(129, 257), n_txt=(2, 33), d=200, n_heads=2,
+         rank=10, keep=40),
+    # many late layers / no activity term
+    dict(seed=15, dtype=torch.bfloat16, batch=2, n_vis=333, n_txt=7, d=128, n_heads=1, rank=8,
+         keep_ratio=0.1, act_layers=9),
+    dict(seed=16, dtype=torch.bfloat16, batch=2, n_vis=333, n_txt=7, d=128, n_heads=1, rank=8,
+         keep_ratio=0.1, act_layers=0),
+    # video-like near-duplicate frames: low-rank dependency dominates
+    dict(seed=17, dtype=torch.bfloat16, batch=2, n_vis=1536, n_txt=16, d=256, n_heads=2, rank=16,
+         kind="video", keep=128),
+]
+
+
+@pytest.mark.parametrize("kw", SMALL, ids=lambda kw: f"seed{kw['seed']}")
+def test_small_shapes(kw):
+    wl = workloads.make_workload(f"small{kw['seed']}", **kw)
+    _report(wl.name, parity.run_gpu(wl))
+
+
+def test_degenerate_requests():
+    # N = 1; B_vis >= N (keep everything); B_vis = N - 1; B_vis = 1; T = 1
+    wl = workloads.make_workload("degenerate", seed=21, dtype=torch.bfloat16, batch=6,
+                                 n_vis=(2, 40), n_txt=1, d=64, n_heads=0, rank=4, keep=1)
+    n = np.diff(wl.vis_offsets)
+    wl.keep[:] = [1, n[1], n[2] - 1, 1, n[4] + 5, max(1, n[5] // 2)]
+    _report(wl.name, parity.run_gpu(wl))
+    one = workloads.make_workload("single-token", seed=22, dtype=torch.float32, batch=2, n_vis=1,
+                                  n_txt=3, d=32, n_heads=0, rank=2, keep=1)
+    _report(one.name, parity.run_gpu(one))
+
+
+@pytest.mark.parametrize("mode", ["zscore", "none"])
+def test_norm_modes(mode):
+    wl = workloads.make_workload("norm-" + mode, seed=23, dtype=torch.bfloat16, batch=2, n_vis=400,
+                                 n_txt=12, d=128, n_heads=2, rank=8, keep_ratio=0.2)
+    _report(wl.name, parity.run_gpu(wl, pruner_kw=dict(norm_mode=mode), norm_mode=mode))
+
+
+def test_head_mean_and_lambda_extremes():
+    wl = workloads.make_workload("head-mean", seed=24, dtype=torch.bfloat16, batch=2, n_vis=300,
+                                 n_txt=(4, 20), d=128, n_heads=4, rank=8, keep_ratio=0.2)
+    _report(wl.name, parity.run_gpu(wl, pruner_kw=dict(head_reduce="mean"), head_reduce="mean"))
+    for lam in (0.0, 1.0):
+        wl.lam = lam
+        _report(f"lambda={lam}", parity.run_gpu(wl))
+
+
+def test_budget_knobs():
+    wl = workloads.make_workload("knobs", seed=25, dtype=torch.bfloat16, batch=3, n_vis=(200, 500),
+                                 n_txt=8, d=128, n_heads=1, rank=24, keep_ratio=0.15)
+    kn = dict(presel_factor=3.0, rank_frac=0.25, rank_cap=16)
+    _report(wl.name, parity.run_gpu(wl, pruner_kw=kn, **kn))
+    kn = dict(presel_factor=1.0)          # M == B_vis: stage 2 is skipped
+    _report(wl.name + " M=B", parity.run_gpu(wl, pruner_kw=kn, **kn))
+
+
+def test_config_c1():
+    _report("c1", parity.run_gpu(workloads.make_config("c1")))
+
+
+def test_config_c2():
+    wl = workloads.make_config("c2")
+    _report("c2", parity.run_gpu(wl))
+
+
+def test_determinism_and_plan_cache():
+    from paper_2605_02218_b200 import api
+    wl = workloads.make_workload("det", seed=31, dtype=torch.bfloat16, batch=3, n_vis=(100, 400),
+                                 n_txt=10, d=128, n_heads=2, rank=8, keep_ratio=0.2).to("cuda:0")
+    pr = api.Pruner.for_workload(wl)
+    m = pr.marshal(wl)
+    a = pr.prune(m)
+    b = pr.prune(m)                       # cached plan
+    assert torch.equal(a[0], b[0]) and torch.equal(a[1], b[1])
+    # a different shape on the same context rebuilds the plan
+    wl2 = wl.request(1).to("cuda:0")
+    m2 = pr.marshal(wl2)
+    c = pr.prune(m2)
+    k1 = a[1][a[2][1]:a[2][2]]
+    assert torch.equal(c[1], k1)
+    pr.check_device_status()
+
+
+def test_device_status_reports_nonfinite():
+    from paper_2605_02218_b200 import api
+    wl = workloads.make_workload("nan", seed=32, dtype=torch.float32, batch=1, n_vis=64, n_txt=4,
+                                 d=32, n_heads=0, rank=4, keep=8).to("cuda:0")
+    wl.X[5, 3] = float("nan")
+    pr = api.Pruner.for_workload(wl)
+    out, keep, ko = pr.prune(pr.marshal(wl))
+    assert pr.device_status() == -6
+    assert pr.device_status() == 0        # reading clears it
+    k = keep.cpu().numpy()
+    assert len(np.unique(k)) == 8 and k.min() >= 0 and k.max() < 64
+
+
+def test_capacity_and_argument_errors():
+    from paper_2605_02218_b200 import api
+    wl = workloads.make_workload("cap", seed=33, dtype=torch.bfloat16, batch=2, n_vis=100, n_txt=4,
+                                 d=64, n_heads=0, rank=4, keep=10).to("cuda:0")
+    pr = api.Pruner.for_workload(wl.request(0).to("cuda:0"))
+    with pytest.raises(api.CovspecError) as e:
+        pr.prune(pr.marshal(wl))          # batch 2 on a context sized for 1
+    assert e.value.status == -4
+    m = pr.marshal(wl.request(0).to("cuda:0"))
+    m.problem.X = None
+    with pytest.raises(api.CovspecError) as e:
+        pr.prune(m)
+    assert e.value.status == -1
