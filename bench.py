@@ -1,0 +1,322 @@
+#!/usr/bin/env python
+"""Benchmark of the fused visual-token reduction (covspec_prune) on synthetic inputs.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--config c2] [--impl ours|reference]
+
+One step = one pass of the whole hot path (Eq. 10 through the compacted buffer) over one batch.
+`value` is whole-job visual tokens pruned per second with inputs resident in HBM; `e2e` repeats the
+measurement with host (pinned) inputs copied in and the results copied out inside the timed region.
+N > 1 (launched with torch.distributed.run): requests are independent, so every rank prunes its own
+batch of the same shape (different seed) with no collective on the data path (weak scaling); the
+time is the maximum over ranks.
+
+--impl reference times the CPU oracle (oracle/) on the host cores on a bounded sample of the same
+workload; it is a deliberately plain program, reported for context.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+from paper_2605_02218_b200 import workloads
+
+METRIC = "visual_tokens_pruned_per_s"
+UNIT = "tokens/s"
+
+
+def _peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return dict(hbm=p["hbm_gbs"], tf_burst=p["bf16_tflops"], tf_sust=p["bf16_tflops_sustained"],
+                    source="measured")
+    return dict(hbm=6650.0, tf_burst=1590.0, tf_sust=1400.0, source="fallback")
+
+
+def _describe(wl):
+    n = np.diff(wl.vis_offsets)
+    t = np.diff(wl.txt_offsets)
+    return dict(batch=wl.batch, n_vis=[int(n.min()), int(n.max())], n_txt=[int(t.min()), int(t.max())],
+                d=wl.d, n_heads=wl.n_heads, head_dim=wl.head_dim, act_layers=wl.act_layers,
+                keep=[int(wl.keep.min()), int(wl.keep.max())],
+                dtype=str(wl.dtype).replace("torch.", ""))
+
+
+def algorithmic_work(wl):
+    """Algorithmic flops of the relevance stage and bytes of the whole path (per step)."""
+    n = np.diff(wl.vis_offsets).astype(np.float64)
+    t = np.diff(wl.txt_offsets).astype(np.float64)
+    P = wl.n_heads * wl.head_dim if wl.n_heads else wl.d
+    e = 2 if wl.dtype == torch.bfloat16 else 4
+    proj = 2.0 * n.sum() * wl.d * P if wl.n_heads else 0.0
+    qproj = 2.0 * t.sum() * wl.d * P if wl.n_heads else 0.0
+    logits = 2.0 * (n * t).sum() * P
+    in_bytes = (n.sum() * wl.d * e * (1 + (wl.act_layers + 1 if wl.act_layers else 0))
+                + t.sum() * wl.d * e + (2 * P * wl.d * e if wl.n_heads else 0))
+    return dict(relevance_flops=proj + logits, qembed_flops=qproj, input_bytes=in_bytes,
+                activity_bytes=n.sum() * wl.d * e * (wl.act_layers + 1 if wl.act_layers else 0))
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML (read-only) while the timed region runs."""
+
+    def __init__(self, index):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def _run(self):
+        nv = self.nv
+        names = {
+            "hw_slowdown": getattr(nv, "nvmlClocksThrottleReasonHwSlowdown", 0x8),
+            "hw_thermal_slowdown": getattr(nv, "nvmlClocksThrottleReasonHwThermalSlowdown", 0x40),
+            "sw_thermal_slowdown": getattr(nv, "nvmlClocksThrottleReasonSwThermalSlowdown", 0x20),
+            "sw_power_cap": getattr(nv, "nvmlClocksThrottleReasonSwPowerCap", 0x4),
+        }
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for k, bit in names.items():
+                    if mask & bit:
+                        self.reasons.add(k)
+            except Exception:
+                pass
+            self._stop.wait(0.02)
+
+    def __enter__(self):
+        if self.nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+
+    def summary(self):
+        if not self.samples:
+            return dict(sm_mhz=None, sm_max_mhz=self.max_mhz, reasons=sorted(self.reasons), samples=0)
+        return dict(sm_mhz=float(np.median(self.samples)), sm_max_mhz=self.max_mhz,
+                    reasons=sorted(self.reasons), samples=len(self.samples))
+
+
+def cpu_baseline(wl_cpu, budget_s=20.0):
+    """Times the oracle as it stands on a bounded sample (whole requests) of the workload."""
+    from oracle import covspec_oracle as oracle
+    n = np.diff(wl_cpu.vis_offsets)
+    done_tokens, reqs = 0, 0
+    t0 = time.perf_counter()
+    for b in range(wl_cpu.batch):
+        oracle.prune_batch(wl_cpu, requests=[b])
+        done_tokens += int(n[b])
+        reqs += 1
+        if time.perf_counter() - t0 > budget_s:
+            break
+    dt = time.perf_counter() - t0
+    cores = len(os.sched_getaffinity(0))
+    return dict(value=done_tokens / dt, unit=UNIT, cores=cores, kind="oracle",
+                sample=f"{reqs} of {wl_cpu.batch} requests ({done_tokens} tokens), one pass, {dt:.2f} s",
+                seconds=dt)
+
+
+def run_reference(args, rank):
+    if rank != 0:
+        return
+    wl = workloads.make_config(args.config, batch=min(args.ref_batch, workloads.CONFIGS[args.config]["batch"]))
+    for _ in range(args.warmup):
+        cpu_baseline(wl.request(0), budget_s=0)
+    t_total, tok_total, samples = 0.0, 0, []
+    for _ in range(args.steps):
+        r = cpu_baseline(wl, budget_s=args.ref_budget)
+        t_total += r["seconds"]
+        tok_total += r["value"] * r["seconds"]
+        samples.append(r["sample"])
+    value = tok_total / t_total
+    line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=args.gpus, steps=args.steps,
+                warmup=args.warmup, ms_per_step=1e3 * t_total / args.steps, higher_is_better=True,
+                scaling="weak", vs_baseline=None, dtype="f64", data="synthetic", impl="reference",
+                config=dict(workload=f"{args.config}: " + json.dumps(_describe(wl)),
+                            note="CPU oracle on a bounded sample of the workload"),
+                cpu_baseline=dict(value=value, unit=UNIT, cores=len(os.sched_getaffinity(0)),
+                                  kind="oracle", sample=samples[-1]),
+                e2e=dict(value=value, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0),
+                gpu_launches=0)
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--config", default="c2", choices=sorted(workloads.CONFIGS))
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--copies", type=int, default=0, help="independent input sets to rotate through")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--ref-batch", type=int, default=16)
+    ap.add_argument("--ref-budget", type=float, default=20.0)
+    args = ap.parse_args()
+
+    rank = int(os.environ.get("RANK", 0))
+    local_rank = int(os.environ.get("LOCAL_RANK", 0))
+    world = int(os.environ.get("WORLD_SIZE", 1))
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+
+    from paper_2605_02218_b200 import api, build
+    build.build()
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU path)"
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # Input sets: rotate through enough independent copies that the working set of consecutive
+    # steps exceeds twice the 126 MB L2.
+    base_seed = workloads.CONFIGS[args.config]["seed"]
+    wl0 = workloads.make_config(args.config, device=dev, seed=base_seed + 1000 * rank)
+    work = algorithmic_work(wl0)
+    copies = args.copies or max(2, int(np.ceil(2 * 126e6 * 2 / work["input_bytes"])))
+    copies = min(copies, 8)
+    sets = [wl0] + [workloads.make_config(args.config, device=dev, seed=base_seed + 1000 * rank + 17 * (i + 1))
+                    for i in range(copies - 1)]
+    pr = api.Pruner.for_workload(wl0)
+    ms = [pr.marshal(w) for w in sets]
+    ko, _ = pr.plan_sizes(ms[0])
+    n_keep = int(ko[-1])
+    outs = [torch.empty((n_keep, wl0.d), dtype=wl0.dtype, device=dev) for _ in sets]
+    keeps = [torch.empty(n_keep, dtype=torch.int32, device=dev) for _ in sets]
+    tokens = wl0.total_vis
+
+    def step(i):
+        j = i % copies
+        pr.prune(ms[j], outs[j], keeps[j])
+
+    # ---- device-resident timing ---------------------------------------------------------------
+    for i in range(max(args.warmup, 3)):
+        step(i)
+    pr.check_device_status()
+    launches_per_step = pr.last_launch_count
+    barrier()
+    pr.profile_begin(args.steps)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(local_rank) as clk:
+        ev0.record()
+        for i in range(args.steps):
+            step(i)
+        ev1.record()
+        barrier()
+    ms_total = ev0.elapsed_time(ev1)
+    stage_ms, prof_calls = pr.profile_end()
+    pr.check_device_status()
+
+    # ---- end to end: pinned host inputs in, results out, every step -----------------------------
+    host = wl0.to("cpu")
+    pin = lambda t: t.pin_memory()
+    hX, hQ, hHs = pin(host.X), pin(host.Q), [pin(h) for h in host.Hs]
+    dX, dQ, dHs = torch.empty_like(wl0.X), torch.empty_like(wl0.Q), [torch.empty_like(h) for h in wl0.Hs]
+    m_e2e = pr.marshal(X=dX, Q=dQ, vis_offsets=wl0.vis_offsets, txt_offsets=wl0.txt_offsets,
+                       Wq=wl0.Wq, Wk=wl0.Wk, Hs=dHs, keep=wl0.keep)
+    h_out = torch.empty((n_keep, wl0.d), dtype=wl0.dtype).pin_memory()
+    h_keep = torch.empty(n_keep, dtype=torch.int32).pin_memory()
+    h2d = hX.nbytes + hQ.nbytes + sum(h.nbytes for h in hHs)
+    d2h = h_out.nbytes + h_keep.nbytes
+
+    def step_e2e():
+        dX.copy_(hX, non_blocking=True)
+        dQ.copy_(hQ, non_blocking=True)
+        for a, b in zip(dHs, hHs):
+            a.copy_(b, non_blocking=True)
+        pr.prune(m_e2e, outs[0], keeps[0])
+        h_out.copy_(outs[0], non_blocking=True)
+        h_keep.copy_(keeps[0], non_blocking=True)
+
+    e2e_steps = max(3, min(args.steps, 20))
+    for _ in range(3):
+        step_e2e()
+    barrier()
+    ev0.record()
+    for _ in range(e2e_steps):
+        step_e2e()
+    ev1.record()
+    barrier()
+    ms_e2e = ev0.elapsed_time(ev1) / e2e_steps
+
+    # ---- reduce over ranks ------------------------------------------------------------------
+    ms_step = ms_total / args.steps
+    if dist is not None:
+        t = torch.tensor([ms_step, ms_e2e], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_step, ms_e2e = t.tolist()
+    if rank == 0:
+        peaks = _peaks()
+        rel_ms = stage_ms["relevance"] / max(prof_calls, 1)
+        long_region = ms_total > 1000.0
+        peak_tf = peaks["tf_sust"] if long_region else peaks["tf_burst"]
+        if wl0.dtype != torch.bfloat16:
+            peak_tf *= 0.5            # tf32 / fp32 path: nominal ratio to the bf16 peak
+        achieved = work["relevance_flops"] / (rel_ms * 1e-3) / 1e12 if rel_ms > 0 else 0.0
+        traffic = None
+        tpath = os.path.join(ROOT, "profiles", "traffic.json")
+        if os.path.exists(tpath):
+            traffic = json.load(open(tpath)).get(args.config, {}).get("relevance_dram_bytes_per_step")
+        line = dict(
+            metric=METRIC, value=world * tokens / (ms_step * 1e-3), unit=UNIT, n_gpus=world,
+            steps=args.steps, warmup=max(args.warmup, 3), ms_per_step=ms_step, higher_is_better=True,
+            scaling="weak", vs_baseline=None,
+            dtype="bf16" if wl0.dtype == torch.bfloat16 else "f32", data="synthetic",
+            config=dict(workload=f"{args.config}: " + json.dumps(_describe(wl0)),
+                        l2="rotating %d independent input sets (%.0f MB) between steps" %
+                           (copies, copies * work["input_bytes"] / 1e6),
+                        us_per_request=1e3 * ms_step / wl0.batch, parallelism=f"dp{world} (requests sharded)"),
+            e2e=dict(value=world * tokens / (ms_e2e * 1e-3), unit=UNIT, h2d_bytes_per_step=int(h2d),
+                     d2h_bytes_per_step=int(d2h), ms_per_step=ms_e2e),
+            gpu_launches=launches_per_step * args.steps,
+            clocks=clk.summary(),
+            roofline=dict(bound="tensor", achieved=achieved, peak=peak_tf, unit="TFLOP/s",
+                          frac=achieved / peak_tf, traffic=traffic,
+                          kernel="relevance stage (projection + cosine max, Eq. 10)",
+                          peak_source=("sustained" if long_region else "burst") + " bf16, " + peaks["source"],
+                          flops_per_step=work["relevance_flops"], ms_per_launch=rel_ms),
+            stages_ms={k: v / max(prof_calls, 1) for k, v in stage_ms.items()},
+        )
+        if not args.no_cpu_baseline and world == 1:
+            cb = cpu_baseline(host)
+            cb.pop("seconds")
+            line["cpu_baseline"] = cb
+        print(json.dumps(line))
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

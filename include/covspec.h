@@ -136,6 +136,16 @@ int covspec_prune(covspec_ctx* ctx, const covspec_problem* p, void* out_hidden, 
  * COVSPEC_ERR_NOCONVERGE) and clears it. */
 int covspec_get_device_status(covspec_ctx* ctx, void* stream);
 
+/* Optional per-stage timing of covspec_prune with CUDA events recorded on the call's stream.
+ * covspec_profile_begin reserves events for up to max_calls prune calls; covspec_profile_end
+ * waits for them, writes the summed milliseconds of each stage into stage_ms[n_stages] (stage
+ * names from covspec_profile_stage_name, count from covspec_profile_stage_count), the number of
+ * profiled calls into *calls, and releases the events. */
+int covspec_profile_begin(covspec_ctx* ctx, int max_calls);
+int covspec_profile_end(covspec_ctx* ctx, double* stage_ms, int n_stages, int* calls);
+int covspec_profile_stage_count(void);
+const char* covspec_profile_stage_name(int stage);
+
 /* Number of kernels the last call on this context launched. */
 int covspec_last_launch_count(const covspec_ctx* ctx);
 

@@ -24,6 +24,8 @@ EXPORTS = [
     "covspec_prune_destroy", "covspec_workspace_bytes", "covspec_score", "covspec_select",
     "covspec_compact", "covspec_prune", "covspec_get_device_status",
     "covspec_last_launch_count", "covspec_strerror", "covspec_last_cuda_error",
+    "covspec_profile_begin", "covspec_profile_end", "covspec_profile_stage_count",
+    "covspec_profile_stage_name",
 ]
 
 
@@ -90,6 +92,11 @@ def load_library():
     lib.covspec_strerror.restype = C.c_char_p
     lib.covspec_last_cuda_error.argtypes = []
     lib.covspec_last_cuda_error.restype = C.c_char_p
+    lib.covspec_profile_begin.argtypes = [vp, C.c_int]
+    lib.covspec_profile_end.argtypes = [vp, C.POINTER(C.c_double), C.c_int, ip]
+    lib.covspec_profile_stage_count.argtypes = []
+    lib.covspec_profile_stage_name.argtypes = [C.c_int]
+    lib.covspec_profile_stage_name.restype = C.c_char_p
     _lib = lib
     return lib
 
@@ -283,6 +290,22 @@ class Pruner:
         if st:
             raise CovspecError(st, "covspec_prune")
         return out, keep_idx, ko
+
+    def profile_begin(self, max_calls: int):
+        st = self.lib.covspec_profile_begin(self._ctx, int(max_calls))
+        if st:
+            raise CovspecError(st, "covspec_profile_begin")
+
+    def profile_end(self):
+        """Returns ({stage name: summed milliseconds}, number of profiled prune calls)."""
+        n = self.lib.covspec_profile_stage_count()
+        ms = (C.c_double * n)()
+        calls = C.c_int()
+        st = self.lib.covspec_profile_end(self._ctx, ms, n, C.byref(calls))
+        if st:
+            raise CovspecError(st, "covspec_profile_end")
+        names = [self.lib.covspec_profile_stage_name(i).decode() for i in range(n)]
+        return dict(zip(names, list(ms))), calls.value
 
     def device_status(self) -> int:
         return int(self.lib.covspec_get_device_status(self._ctx, _stream()))

@@ -46,6 +46,12 @@ enum TableId {
   T_COUNT
 };
 
+// Stages reported by the optional event timing.
+enum StageId { ST_QEMBED = 0, ST_RELEVANCE, ST_ACTIVITY, ST_FUSE, ST_PRESELECT, ST_GRAM, ST_EIG,
+               ST_FINAL, ST_COUNT };
+const char* const kStageNames[ST_COUNT] = {"query_embed", "relevance", "activity", "fuse",
+                                            "preselect", "gram", "subspace", "final_select_compact"};
+
 struct Plan {
   std::vector<int> vis_off, txt_off, keep;    // key of the cache
   double keep_ratio = 0.0;
@@ -89,6 +95,10 @@ struct covspec_ctx {
   cudaEvent_t stage_free = nullptr;      // the previous upload has been consumed
   Plan plan;
   int launches = 0;
+  // optional per-stage timing (CUDA events on the call's stream)
+  std::vector<cudaEvent_t> prof_events;  // [prof_cap][ST_COUNT][2]
+  std::vector<unsigned char> prof_set;
+  int prof_cap = 0, prof_calls = 0;
 };
 
 namespace {
@@ -258,6 +268,13 @@ int get_plan(covspec_ctx* ctx, const covspec_problem* p, cudaStream_t stream) {
     CUDA_TRY(cudaGetLastError());                       \
   } while (0)
 
+// Records the begin (edge 0) or end (edge 1) event of a stage for the current profiled call.
+inline void prof_mark(covspec_ctx* ctx, int stage, int edge, cudaStream_t s) {
+  if (ctx->prof_cap == 0 || ctx->prof_calls >= ctx->prof_cap) return;
+  size_t i = ((size_t)ctx->prof_calls * ST_COUNT + stage) * 2 + edge;
+  if (cudaEventRecord(ctx->prof_events[i], s) == cudaSuccess) ctx->prof_set[i] = 1;
+}
+
 template <typename TA, typename TB, typename AccT, typename TC, bool B_KN>
 int launch_table(covspec_ctx* ctx, int table, int lower_only, cudaStream_t s) {
   int tiles = ctx->plan.tiles[table];
@@ -296,6 +313,7 @@ int score_impl(covspec_ctx* ctx, const covspec_problem* p, float* s_query, float
   if (!s_query) s_query = ctx->sq;
   if (!s_act) s_act = ctx->sa;
   bool identity = cfg.n_heads == 0;
+  prof_mark(ctx, ST_QEMBED, 0, s);
   if (identity) {
     int warps = rowsQ * H;
     qnorm_kernel<T><<<(warps + 7) / 8, 256, 0, s>>>(Q, ctx->Qn, rowsQ, H, hd);
@@ -308,9 +326,11 @@ int score_impl(covspec_ctx* ctx, const covspec_problem* p, float* s_query, float
     qnorm_kernel<float><<<(warps + 7) / 8, 256, 0, s>>>(ctx->Qn, ctx->Qn, rowsQ, H, hd);
     LAUNCH_CHECK(ctx);
   }
+  prof_mark(ctx, ST_QEMBED, 1, s);
   int mean = cfg.head_reduce == 1;
   size_t smem = mean ? (size_t)8 * pl.t_max * sizeof(float) : 0;
   if (smem > 48 * 1024) return COVSPEC_ERR_UNSUPPORTED;
+  prof_mark(ctx, ST_RELEVANCE, 0, s);
   if (identity) {
     cosmax_kernel<T><<<(unsigned)((rowsX + 7) / 8), 256, smem, s>>>(
         X, ctx->Qn, ctx->d_plan, B, 0, (int)rowsX, H, hd, mean, pl.t_max, s_query);
@@ -326,7 +346,9 @@ int score_impl(covspec_ctx* ctx, const covspec_problem* p, float* s_query, float
       LAUNCH_CHECK(ctx);
     }
   }
+  prof_mark(ctx, ST_RELEVANCE, 1, s);
   if (cfg.act_layers > 0) {
+    prof_mark(ctx, ST_ACTIVITY, 0, s);
     LayerPtrs lp{};
     for (int l = 0; l <= cfg.act_layers; ++l) lp.h[l] = p->Hs[l];
     unsigned grid = (unsigned)((rowsX + 7) / 8);
@@ -337,11 +359,14 @@ int score_impl(covspec_ctx* ctx, const covspec_problem* p, float* s_query, float
     else
       activity_kernel<T, 16><<<grid, 256, 0, s>>>(lp, cfg.act_layers, rowsX, cfg.d, s_act);
     LAUNCH_CHECK(ctx);
+    prof_mark(ctx, ST_ACTIVITY, 1, s);
   }
   if (do_fuse) {
+    prof_mark(ctx, ST_FUSE, 0, s);
     fuse_kernel<<<B, 1024, 0, s>>>(s_query, cfg.act_layers > 0 ? s_act : nullptr, ctx->d_plan,
                                    cfg.lambda, cfg.norm_mode, s_fused, ctx->status);
     LAUNCH_CHECK(ctx);
+    prof_mark(ctx, ST_FUSE, 1, s);
   }
   return COVSPEC_OK;
 }
@@ -355,9 +380,12 @@ int select_impl(covspec_ctx* ctx, const covspec_problem* p, const float* s_fused
   int B = p->batch;
   int* presel = presel_out ? presel_out : ctx->presel;
   float* energy = energy_out ? energy_out : ctx->energy;
+  prof_mark(ctx, ST_PRESELECT, 0, s);
   preselect_kernel<<<B, 1024, 0, s>>>(s_fused, ctx->d_plan, presel, ctx->status);
   LAUNCH_CHECK(ctx);
+  prof_mark(ctx, ST_PRESELECT, 1, s);
   if (pl.n_stage2 > 0) {
+    prof_mark(ctx, ST_GRAM, 0, s);
     int vec16 = cfg.d * ctx->esize / 16;
     gather_rows_kernel<<<(unsigned)pl.total_presel, 256, 0, s>>>(
         reinterpret_cast<const uint4*>(p->X), presel, ctx->d_plan, B, 1, vec16,
@@ -365,6 +393,8 @@ int select_impl(covspec_ctx* ctx, const covspec_problem* p, const float* s_fused
     LAUNCH_CHECK(ctx);
     int st = launch_table<T, T, float, float, false>(ctx, T_GRAM_G, 1, s);
     if (st) return st;
+    prof_mark(ctx, ST_GRAM, 1, s);
+    prof_mark(ctx, ST_EIG, 0, s);
     int init_blocks = (pl.p_max * (pl.m_max + 3) + 255) / 256;
     dim3 gi(init_blocks > 64 ? 64 : init_blocks, B);
     eig_init_kernel<<<gi, 256, 0, s>>>(ctx->d_plan, ctx->U0);
@@ -395,6 +425,8 @@ int select_impl(covspec_ctx* ctx, const covspec_problem* p, const float* s_fused
   dim3 ge((pl.m_max + 255) / 256, B);
   energy_kernel<<<ge, 256, 0, s>>>(ctx->d_plan, ctx->U0, ctx->theta, energy);
   LAUNCH_CHECK(ctx);
+  if (pl.n_stage2 > 0) prof_mark(ctx, ST_EIG, 1, s);
+  prof_mark(ctx, ST_FINAL, 0, s);
   final_select_kernel<<<B, 1024, 0, s>>>(energy, presel, ctx->d_plan, keep_idx, ctx->status);
   LAUNCH_CHECK(ctx);
   return COVSPEC_OK;
@@ -408,6 +440,7 @@ int compact_impl(covspec_ctx* ctx, const covspec_problem* p, const int* keep_idx
       reinterpret_cast<const uint4*>(p->X), keep_idx, ctx->d_plan, p->batch, 0, vec16,
       reinterpret_cast<uint4*>(out), out_pos);
   LAUNCH_CHECK(ctx);
+  prof_mark(ctx, ST_FINAL, 1, s);
   return COVSPEC_OK;
 }
 
@@ -621,14 +654,58 @@ int covspec_prune(covspec_ctx* ctx, const covspec_problem* p, void* out_hidden, 
   st = bf ? score_impl<__nv_bfloat16>(ctx, p, nullptr, nullptr, fused, false, s)
           : score_impl<float>(ctx, p, nullptr, nullptr, fused, false, s);
   if (st) return st;
+  prof_mark(ctx, ST_FUSE, 0, s);
   fuse_kernel<<<p->batch, 1024, 0, s>>>(ctx->sq, ctx->cfg.act_layers > 0 ? ctx->sa : nullptr,
                                         ctx->d_plan, ctx->cfg.lambda, ctx->cfg.norm_mode, fused,
                                         ctx->status);
   LAUNCH_CHECK(ctx);
+  prof_mark(ctx, ST_FUSE, 1, s);
   st = bf ? select_impl<__nv_bfloat16>(ctx, p, fused, keep_idx, nullptr, nullptr, s)
           : select_impl<float>(ctx, p, fused, keep_idx, nullptr, nullptr, s);
   if (st) return st;
-  return compact_impl(ctx, p, keep_idx, out_hidden, nullptr, s);
+  st = compact_impl(ctx, p, keep_idx, out_hidden, nullptr, s);
+  if (ctx->prof_cap && ctx->prof_calls < ctx->prof_cap) ++ctx->prof_calls;
+  return st;
+}
+
+int covspec_profile_begin(covspec_ctx* ctx, int max_calls) {
+  if (!ctx || max_calls < 1 || ctx->prof_cap) return COVSPEC_ERR_ARG;
+  size_t n = (size_t)max_calls * ST_COUNT * 2;
+  ctx->prof_events.assign(n, nullptr);
+  ctx->prof_set.assign(n, 0);
+  for (size_t i = 0; i < n; ++i) CUDA_TRY(cudaEventCreate(&ctx->prof_events[i]));
+  ctx->prof_cap = max_calls;
+  ctx->prof_calls = 0;
+  return COVSPEC_OK;
+}
+
+int covspec_profile_end(covspec_ctx* ctx, double* stage_ms, int n_stages, int* calls) {
+  if (!ctx || !ctx->prof_cap) return COVSPEC_ERR_ARG;
+  int st = COVSPEC_OK;
+  for (int g = 0; g < n_stages; ++g) if (stage_ms) stage_ms[g] = 0.0;
+  for (int c = 0; c < ctx->prof_calls; ++c)
+    for (int g = 0; g < ST_COUNT; ++g) {
+      size_t i = ((size_t)c * ST_COUNT + g) * 2;
+      if (!ctx->prof_set[i] || !ctx->prof_set[i + 1]) continue;
+      float ms = 0.f;
+      if (cudaEventSynchronize(ctx->prof_events[i + 1]) != cudaSuccess ||
+          cudaEventElapsedTime(&ms, ctx->prof_events[i], ctx->prof_events[i + 1]) != cudaSuccess) {
+        st = COVSPEC_ERR_CUDA;
+        continue;
+      }
+      if (stage_ms && g < n_stages) stage_ms[g] += ms;
+    }
+  if (calls) *calls = ctx->prof_calls;
+  for (cudaEvent_t e : ctx->prof_events) if (e) cudaEventDestroy(e);
+  ctx->prof_events.clear();
+  ctx->prof_set.clear();
+  ctx->prof_cap = ctx->prof_calls = 0;
+  return st;
+}
+
+int covspec_profile_stage_count(void) { return ST_COUNT; }
+const char* covspec_profile_stage_name(int stage) {
+  return stage >= 0 && stage < ST_COUNT ? kStageNames[stage] : "";
 }
 
 int covspec_get_device_status(covspec_ctx* ctx, void* stream) {

@@ -51,6 +51,7 @@ cosmax_kernel(const TE* __restrict__ E, const float* __restrict__ Qn, const ReqP
   float* acc = smem_mean + (size_t)wib * t_max;
   if (head_mean) for (int j = lane; j < T; j += 32) acc[j] = 0.f;
   float best = -FLT_MAX;
+  bool nonfinite = false;   // fmaxf drops NaN operands, so non-finite inputs are tracked explicitly
   for (int h = 0; h < n_heads; ++h) {
     const TE* eh = e + (size_t)h * hd;
     float ss = 0.f;
@@ -59,6 +60,7 @@ cosmax_kernel(const TE* __restrict__ E, const float* __restrict__ Qn, const ReqP
       ss += v[0] * v[0] + v[1] * v[1] + v[2] * v[2] + v[3] * v[3];
     }
     ss = warp_sum(ss);
+    nonfinite |= !(ss <= FLT_MAX);
     float inv = 0.f;
     if (ss > FLT_MIN) { inv = rsqrtf(ss); inv = inv * (1.5f - 0.5f * ss * inv * inv); }
     for (int j = 0; j < T; ++j) {
@@ -70,6 +72,7 @@ cosmax_kernel(const TE* __restrict__ E, const float* __restrict__ Qn, const ReqP
         dot += v[0] * w.x + v[1] * w.y + v[2] * w.z + v[3] * w.w;
       }
       dot = warp_sum(dot) * inv;
+      nonfinite |= dot != dot;
       if (head_mean) { if (lane == 0) acc[j] += dot; }
       else best = fmaxf(best, dot);
     }
@@ -80,7 +83,7 @@ cosmax_kernel(const TE* __restrict__ E, const float* __restrict__ Qn, const ReqP
     for (int j = lane; j < T; j += 32) m = fmaxf(m, acc[j] / (float)n_heads);
     best = warp_max(m);
   }
-  if (lane == 0) s_query[row] = best;
+  if (lane == 0) s_query[row] = nonfinite ? __int_as_float(0x7fc00000) : best;
 }
 
 // Eq. 11.  One warp per token streams the token's row of all act_layers+1 snapshots once, 16 bytes
