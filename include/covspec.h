@@ -43,7 +43,8 @@ typedef enum {
   COVSPEC_ERR_WORKSPACE = -4,   /* problem exceeds the capacities given at init               */
   COVSPEC_ERR_CUDA = -5,        /* a CUDA runtime call failed (see covspec_last_cuda_error)   */
   COVSPEC_ERR_NONFINITE = -6,   /* device status: a score was NaN or Inf                      */
-  COVSPEC_ERR_NOCONVERGE = -7   /* device status: small eigen-solve hit its sweep limit       */
+  COVSPEC_ERR_NOCONVERGE = -7,  /* device status: small eigen-solve hit its sweep limit       */
+  COVSPEC_ERR_STATIC_CAPACITY = -8 /* covspec_query_score_static: beyond its fixed scratch size */
 } covspec_status;
 
 /* Static configuration.  Fill with covspec_default_config() and override. */
@@ -145,6 +146,35 @@ int covspec_profile_begin(covspec_ctx* ctx, int max_calls);
 int covspec_profile_end(covspec_ctx* ctx, double* stage_ms, int n_stages, int* calls);
 int covspec_profile_stage_count(void);
 const char* covspec_profile_stage_name(int stage);
+
+/* Allocation-free variant of the query-aware score.  (The paper has no counterpart of this entry
+ * point: it computes Eq. 10 exactly as covspec_score does with the identity embedding, but is
+ * packaged for callers that cannot allocate.)
+ *
+ * Who needs it: code that runs where device allocation is off limits - inside a serving loop whose
+ * memory pool is fully handed out at start-up, in a process whose allocator is owned by another
+ * framework and must not see foreign cudaMalloc calls, or in a latency path where an allocation's
+ * implicit device synchronisation is unacceptable.  Such callers cannot create a covspec_ctx
+ * (covspec_prune_init allocates the workspace).  This entry point needs no context: its scratch
+ * (the unit-length query elements and the per-request plan) lives in a fixed device array inside
+ * the library, which every GPU that loads the library holds until the process exits.  The call
+ * issues no cudaMalloc, cudaFree or other allocating routine.
+ *
+ *  dtype, d      as in covspec_config (d a multiple of 8); identity embedding, max over elements
+ *  X, Q          device, laid out as in covspec_problem; vis_offsets, txt_offsets host [batch+1]
+ *  s_query       device [vis_offsets[batch]] float32 (out): Eq. 10 per visual token
+ * Limits: batch <= COVSPEC_STATIC_MAX_BATCH and txt_offsets[batch] * d <=
+ * COVSPEC_STATIC_MAX_QUERY_ELEMS; larger problems are rejected with COVSPEC_ERR_STATIC_CAPACITY
+ * and nothing is launched.
+ * The first call on a device looks up the scratch array's device address (once per device, with
+ * that device current) and should therefore be made before any stream capture begins.
+ * Every call on a device shares the one scratch array and leaves its contents behind.  Nothing in
+ * it has to start at zero (each call rewrites the part it reads), but two calls that overlap on
+ * the GPU - different streams, or different host threads - race on it: serialise them. */
+#define COVSPEC_STATIC_MAX_BATCH 256
+#define COVSPEC_STATIC_MAX_QUERY_ELEMS (1 << 20)   /* 4 MiB of float32 scratch */
+int covspec_query_score_static(int dtype, int d, int batch, const void* X, const int* vis_offsets,
+                               const void* Q, const int* txt_offsets, float* s_query, void* stream);
 
 /* Number of kernels the last call on this context launched. */
 int covspec_last_launch_count(const covspec_ctx* ctx);

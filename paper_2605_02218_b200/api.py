@@ -25,8 +25,10 @@ EXPORTS = [
     "covspec_compact", "covspec_prune", "covspec_get_device_status",
     "covspec_last_launch_count", "covspec_strerror", "covspec_last_cuda_error",
     "covspec_profile_begin", "covspec_profile_end", "covspec_profile_stage_count",
-    "covspec_profile_stage_name",
+    "covspec_profile_stage_name", "covspec_query_score_static",
 ]
+STATIC_MAX_BATCH = 256
+STATIC_MAX_QUERY_ELEMS = 1 << 20
 
 
 class Config(C.Structure):
@@ -92,6 +94,7 @@ def load_library():
     lib.covspec_strerror.restype = C.c_char_p
     lib.covspec_last_cuda_error.argtypes = []
     lib.covspec_last_cuda_error.restype = C.c_char_p
+    lib.covspec_query_score_static.argtypes = [C.c_int, C.c_int, C.c_int, vp, ip, vp, ip, fp, vp]
     lib.covspec_profile_begin.argtypes = [vp, C.c_int]
     lib.covspec_profile_end.argtypes = [vp, C.POINTER(C.c_double), C.c_int, ip]
     lib.covspec_profile_stage_count.argtypes = []
@@ -314,3 +317,23 @@ class Pruner:
         st = self.device_status()
         if st:
             raise CovspecError(st, "device status")
+
+
+def query_score_static(X: torch.Tensor, Q: torch.Tensor, vis_offsets, txt_offsets,
+                       out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """covspec_query_score_static: Eq. 10 with the identity embedding for callers that must not
+    allocate device memory (a serving loop with a fully committed memory pool, a process whose
+    allocator belongs to another framework).  The library call itself allocates nothing; pass
+    `out` (float32, one element per visual token) to keep this wrapper allocation-free as well."""
+    lib = load_library()
+    assert X.is_cuda and Q.is_cuda and X.is_contiguous() and Q.is_contiguous() and X.dtype == Q.dtype
+    vis, vis_p = _i32(vis_offsets)
+    txt, txt_p = _i32(txt_offsets)
+    if out is None:
+        out = torch.empty(int(vis[-1]), dtype=torch.float32, device=X.device)
+    dtype = COVSPEC_BF16 if X.dtype == torch.bfloat16 else COVSPEC_F32
+    st = lib.covspec_query_score_static(dtype, X.shape[1], len(vis) - 1, _ptr(X), vis_p, _ptr(Q),
+                                        txt_p, _ptr(out), _stream())
+    if st:
+        raise CovspecError(st, "covspec_query_score_static")
+    return out

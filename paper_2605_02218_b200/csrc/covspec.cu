@@ -6,6 +6,7 @@
 #include <stdio.h>
 #include <string.h>
 
+#include <mutex>
 #include <string>
 #include <vector>
 
@@ -732,6 +733,8 @@ const char* covspec_strerror(int status) {
     case COVSPEC_ERR_CUDA: return "CUDA runtime error";
     case COVSPEC_ERR_NONFINITE: return "non-finite score on the device";
     case COVSPEC_ERR_NOCONVERGE: return "small eigen-solve did not converge";
+    case COVSPEC_ERR_STATIC_CAPACITY:
+      return "problem exceeds the fixed scratch capacity of the allocation-free entry point";
     default: return "unknown status";
   }
 }
@@ -739,3 +742,82 @@ const char* covspec_strerror(int status) {
 const char* covspec_last_cuda_error(void) { return g_cuda_error.c_str(); }
 
 }  // extern "C"
+
+// ================================================================================================
+// Allocation-free query score.  The scratch the cosine kernel needs (the unit-length query
+// elements and the per-request plan) lives in this fixed device array instead of a context
+// workspace, so the entry point below never calls an allocator.
+namespace {
+
+constexpr int kStaticMaxBatch = COVSPEC_STATIC_MAX_BATCH;
+constexpr long long kStaticMaxQueryElems = COVSPEC_STATIC_MAX_QUERY_ELEMS;
+constexpr size_t kStaticPlanBytes = (sizeof(ReqPlan) * kStaticMaxBatch + 255) / 256 * 256;
+constexpr size_t kStaticScratchBytes = kStaticPlanBytes + sizeof(float) * kStaticMaxQueryElems;
+
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+constexpr int kStaticMaxDevices = 64;
+std::mutex g_static_mutex;
+void* g_static_ptr[kStaticMaxDevices] = {nullptr};
+
+// Device address of g_static_scratch on the current device.  In host code the array's name is only
+// a handle for the runtime, not an address a kernel can use; the address is looked up once per
+// device, with that device current, and cached.
+int static_scratch_ptr(unsigned char** out) {
+  int dev = 0;
+  CUDA_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kStaticMaxDevices) return COVSPEC_ERR_UNSUPPORTED;
+  std::lock_guard<std::mutex> lock(g_static_mutex);
+  if (g_static_ptr[dev] == nullptr) {
+    void* ptr = nullptr;
+    CUDA_TRY(cudaGetSymbolAddress((void**)&ptr, g_static_scratch));
+    g_static_ptr[dev] = ptr;
+  }
+  *out = reinterpret_cast<unsigned char*>(g_static_ptr[dev]);
+  return COVSPEC_OK;
+}
+
+template <typename T>
+int query_score_static_impl(int d, int batch, const ReqPlan* h_plan, const void* X, const void* Q,
+                            long long rows_x, int rows_q, float* s_query, cudaStream_t s) {
+  unsigned char* scratch = nullptr;
+  int st = static_scratch_ptr(&scratch);
+  if (st) return st;
+  ReqPlan* d_plan = reinterpret_cast<ReqPlan*>(scratch);
+  float* Qn = reinterpret_cast<float*>(scratch + kStaticPlanBytes);
+  // The copy source is ordinary host memory: the runtime stages it before the call returns.
+  CUDA_TRY(cudaMemcpyAsync(d_plan, h_plan, sizeof(ReqPlan) * batch, cudaMemcpyHostToDevice, s));
+  qnorm_kernel<T><<<(rows_q + 7) / 8, 256, 0, s>>>(reinterpret_cast<const T*>(Q), Qn, rows_q, 1, d);
+  CUDA_TRY(cudaGetLastError());
+  cosmax_kernel<T><<<(unsigned)((rows_x + 7) / 8), 256, 0, s>>>(
+      reinterpret_cast<const T*>(X), Qn, d_plan, batch, 0, (int)rows_x, 1, d, 0, 0, s_query);
+  CUDA_TRY(cudaGetLastError());
+  return COVSPEC_OK;
+}
+
+}  // namespace
+
+extern "C" int covspec_query_score_static(int dtype, int d, int batch, const void* X,
+                                          const int* vis_offsets, const void* Q,
+                                          const int* txt_offsets, float* s_query, void* stream) {
+  if (!X || !Q || !vis_offsets || !txt_offsets || !s_query || batch < 1) return COVSPEC_ERR_ARG;
+  if (dtype != COVSPEC_F32 && dtype != COVSPEC_BF16) return COVSPEC_ERR_ARG;
+  if (d < 8 || d % 8) return COVSPEC_ERR_UNSUPPORTED;
+  if (vis_offsets[0] != 0 || txt_offsets[0] != 0) return COVSPEC_ERR_SHAPE;
+  if (batch > kStaticMaxBatch) return COVSPEC_ERR_STATIC_CAPACITY;
+  ReqPlan h_plan[kStaticMaxBatch];
+  memset(h_plan, 0, sizeof(ReqPlan) * batch);
+  for (int b = 0; b < batch; ++b) {
+    if (vis_offsets[b + 1] <= vis_offsets[b] || txt_offsets[b + 1] <= txt_offsets[b])
+      return COVSPEC_ERR_SHAPE;
+    h_plan[b].vis_off = vis_offsets[b]; h_plan[b].n = vis_offsets[b + 1] - vis_offsets[b];
+    h_plan[b].txt_off = txt_offsets[b]; h_plan[b].t = txt_offsets[b + 1] - txt_offsets[b];
+  }
+  if ((long long)txt_offsets[batch] * d > kStaticMaxQueryElems) return COVSPEC_ERR_STATIC_CAPACITY;
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  return dtype == COVSPEC_BF16
+             ? query_score_static_impl<__nv_bfloat16>(d, batch, h_plan, X, Q, vis_offsets[batch],
+                                                      txt_offsets[batch], s_query, s)
+             : query_score_static_impl<float>(d, batch, h_plan, X, Q, vis_offsets[batch],
+                                              txt_offsets[batch], s_query, s);
+}
