@@ -44,7 +44,8 @@ typedef enum {
   COVSPEC_ERR_CUDA = -5,        /* a CUDA runtime call failed (see covspec_last_cuda_error)   */
   COVSPEC_ERR_NONFINITE = -6,   /* device status: a score was NaN or Inf                      */
   COVSPEC_ERR_NOCONVERGE = -7,  /* device status: small eigen-solve hit its sweep limit       */
-  COVSPEC_ERR_STATIC_CAPACITY = -8 /* covspec_query_score_static: beyond its fixed scratch size */
+  COVSPEC_ERR_STATIC_CAPACITY = -8, /* covspec_query_score_static: beyond its fixed scratch size */
+  COVSPEC_ERR_TIMEOUT = -9      /* device status: a bounded wait inside a kernel expired      */
 } covspec_status;
 
 /* Static configuration.  Fill with covspec_default_config() and override. */
@@ -68,6 +69,9 @@ typedef struct {
   int max_vis_per_req;           /* max N_b */
   int max_presel_per_req;        /* max M_b   (0: derive from max_vis_per_req) */
   long long max_total_presel;    /* sum of M_b (0: derive from max_total_vis)  */
+  int relevance_path;  /* 0: Eq. 10 on the tensor cores (tcgen05) whenever the configuration allows
+                          (bf16, 128-wide heads, max over heads, d >= 64), else the CUDA-core path;
+                          1: always the CUDA-core path                                            */
 } covspec_config;
 
 /* One batch of requests (Sec. III-A notation in brackets). */
@@ -133,7 +137,7 @@ int covspec_compact(covspec_ctx* ctx, const covspec_problem* p, const int* keep_
 int covspec_prune(covspec_ctx* ctx, const covspec_problem* p, void* out_hidden, int* keep_idx,
                   int* keep_offsets, void* stream);
 
-/* Synchronises `stream`, returns the device status word (COVSPEC_OK, COVSPEC_ERR_NONFINITE or
+/* Synchronises `stream`, returns the device status word (COVSPEC_OK, COVSPEC_ERR_TIMEOUT, COVSPEC_ERR_NONFINITE or
  * COVSPEC_ERR_NOCONVERGE) and clears it. */
 int covspec_get_device_status(covspec_ctx* ctx, void* stream);
 

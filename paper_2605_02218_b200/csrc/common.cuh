@@ -21,6 +21,8 @@ struct ReqPlan {
   int keep_off, presel_off;
   int ldm;                 // m rounded up to a multiple of 4 (row stride of G and of the bases)
   int stage2;              // 1 when b_vis < m (Eq. 13-15 are evaluated)
+  int tile_off;            // first 128-token tile of the request in the tensor-core relevance kernel
+  int pad_;
   long long g_off;         // float offset of the request's Gram matrix
   long long u_off;         // float offset of the request's basis buffers (p x ldm)
 };

@@ -13,6 +13,7 @@
 #include "common.cuh"
 #include "eig_kernels.cuh"
 #include "gemm_simt.cuh"
+#include "relevance_tc.cuh"
 #include "score_kernels.cuh"
 #include "select_kernels.cuh"
 
@@ -62,6 +63,7 @@ struct Plan {
   int n_stage2 = 0;
   int tiles[T_COUNT] = {0};
   int t_max = 0, p_max = 0, m_max = 0;
+  int n_tiles = 0;                            // 128-token tiles over all requests
   long long total_vis = 0, total_txt = 0, total_keep = 0, total_presel = 0;
   bool valid = false;
 };
@@ -95,6 +97,8 @@ struct covspec_ctx {
   long long stage_bytes = 0;
   cudaEvent_t stage_free = nullptr;      // the previous upload has been consumed
   Plan plan;
+  int num_sms = 148;
+  bool tc_ready = false;                 // tensor-core relevance kernel configured on this device
   int launches = 0;
   // optional per-stage timing (CUDA events on the call's stream)
   std::vector<cudaEvent_t> prof_events;  // [prof_cap][ST_COUNT][2]
@@ -178,7 +182,7 @@ int get_plan(covspec_ctx* ctx, const covspec_problem* p, cudaStream_t stream) {
   pl.req.assign(B, ReqPlan{});
   pl.keep_offsets.assign(B + 1, 0);
   pl.presel_offsets.assign(B + 1, 0);
-  pl.n_stage2 = 0; pl.t_max = 0; pl.p_max = 0; pl.m_max = 0;
+  pl.n_stage2 = 0; pl.t_max = 0; pl.p_max = 0; pl.m_max = 0; pl.n_tiles = 0;
   long long g_off = 0, u_off = 0;
   int n_max = 0;
   for (int b = 0; b < B; ++b) {
@@ -195,6 +199,8 @@ int get_plan(covspec_ctx* ctx, const covspec_problem* p, cudaStream_t stream) {
       ++pl.n_stage2;
     }
     r.ldm = (int)round_up(r.m, 4);
+    r.tile_off = pl.n_tiles;
+    pl.n_tiles += (r.n + tc::kTileM - 1) / tc::kTileM;
     r.keep_off = pl.keep_offsets[b]; r.presel_off = pl.presel_offsets[b];
     pl.keep_offsets[b + 1] = r.keep_off + r.b_vis;
     pl.presel_offsets[b + 1] = r.presel_off + r.m;
@@ -299,6 +305,92 @@ int launch_single_nt(covspec_ctx* ctx, const T* A, const T* B, float* C, int m, 
   return COVSPEC_OK;
 }
 
+// ---- tensor-core relevance path ----------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
+                                  const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
+                                  const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+  static EncodeTiledFn fn = [] {
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess)
+      ptr = nullptr;
+    return reinterpret_cast<EncodeTiledFn>(ptr);
+  }();
+  return fn;
+}
+
+// Tensor map of a row-major bf16 matrix [rows, cols] with boxes of 64 columns (one 128-byte
+// swizzle row) by box_rows rows; out-of-range elements read as zero.
+int make_map_bf16(CUtensorMap* map, const void* base, long long rows, long long cols, int box_rows) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (!fn) { g_cuda_error = "cuTensorMapEncodeTiled is not available"; return COVSPEC_ERR_CUDA; }
+  cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+  cuuint32_t box[2] = {(cuuint32_t)tc::kBK, (cuuint32_t)box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box,
+                  estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    g_cuda_error = "cuTensorMapEncodeTiled failed with code " + std::to_string((int)r);
+    return COVSPEC_ERR_CUDA;
+  }
+  return COVSPEC_OK;
+}
+
+bool tc_supported(const covspec_ctx* ctx) {
+  const covspec_config& c = ctx->cfg;
+  return ctx->tc_ready && c.relevance_path == 0 && c.dtype == COVSPEC_BF16 && c.n_heads > 0 &&
+         c.head_dim == tc::kHeadDim && c.head_reduce == 0 && c.d >= tc::kBK;
+}
+
+// Eq. 10 on the tensor cores: query embedding (MODE 1), -inf fill, fused projection + cosine max.
+int relevance_tc(covspec_ctx* ctx, const covspec_problem* p, float* s_query, cudaStream_t s) {
+  const covspec_config& cfg = ctx->cfg;
+  const Plan& pl = ctx->plan;
+  int P = ctx->P, d = cfg.d;
+  __nv_bfloat16* qn = reinterpret_cast<__nv_bfloat16*>(ctx->Qn);
+  CUtensorMap map_x, map_wk, map_q, map_wq, map_qn, map_qnl;
+  long long lo_off = (long long)cfg.max_total_txt * P;   // lo parts follow the hi parts
+  int st;
+  if ((st = make_map_bf16(&map_x, p->X, pl.total_vis, d, tc::kTileM))) return st;
+  if ((st = make_map_bf16(&map_wk, p->Wk, P, d, tc::kTileN))) return st;
+  if ((st = make_map_bf16(&map_q, p->Q, pl.total_txt, d, tc::kTileM))) return st;
+  if ((st = make_map_bf16(&map_wq, p->Wq, P, d, tc::kTileN))) return st;
+  if ((st = make_map_bf16(&map_qn, qn, pl.total_txt, P, tc::kTT))) return st;
+  if ((st = make_map_bf16(&map_qnl, qn + lo_off, pl.total_txt, P, tc::kTT))) return st;
+  int n_hp = (cfg.n_heads + 1) / 2;
+  tc::Params prm{};
+  prm.plan = ctx->d_plan; prm.batch = p->batch;
+  prm.n_groups = n_hp; prm.hp_per_group = 1;
+  prm.n_heads = cfg.n_heads; prm.k_chunks = (d + tc::kBK - 1) / tc::kBK; prm.P = P;
+  prm.status = ctx->status;
+  // query side
+  prof_mark(ctx, ST_QEMBED, 0, s);
+  prm.rows_total = pl.total_txt;
+  prm.n_items = (int)((pl.total_txt + tc::kTileM - 1) / tc::kTileM) * prm.n_groups;
+  prm.qn_out = qn; prm.qn_lo_off = lo_off; prm.s_query = nullptr;
+  int grid = prm.n_items < ctx->num_sms ? prm.n_items : ctx->num_sms;
+  tc::relevance_tc_kernel<1><<<grid, 192, tc::kSmemBytes, s>>>(map_q, map_wq, map_qn, map_qnl, prm);
+  LAUNCH_CHECK(ctx);
+  prof_mark(ctx, ST_QEMBED, 1, s);
+  // visual side
+  prof_mark(ctx, ST_RELEVANCE, 0, s);
+  tc::fill_neg_inf_kernel<<<(unsigned)((pl.total_vis + 255) / 256), 256, 0, s>>>(s_query, pl.total_vis);
+  LAUNCH_CHECK(ctx);
+  prm.n_items = pl.n_tiles * prm.n_groups;
+  prm.qn_out = nullptr; prm.s_query = s_query;
+  grid = prm.n_items < ctx->num_sms ? prm.n_items : ctx->num_sms;
+  tc::relevance_tc_kernel<0><<<grid, 192, tc::kSmemBytes, s>>>(map_x, map_wk, map_qn, map_qnl, prm);
+  LAUNCH_CHECK(ctx);
+  prof_mark(ctx, ST_RELEVANCE, 1, s);
+  return COVSPEC_OK;
+}
+
 // ---- Eq. 10-12 -------------------------------------------------------------------------------
 template <typename T>
 int score_impl(covspec_ctx* ctx, const covspec_problem* p, float* s_query, float* s_act,
@@ -314,6 +406,11 @@ int score_impl(covspec_ctx* ctx, const covspec_problem* p, float* s_query, float
   if (!s_query) s_query = ctx->sq;
   if (!s_act) s_act = ctx->sa;
   bool identity = cfg.n_heads == 0;
+  bool use_tc = tc_supported(ctx);
+  if (use_tc) {
+    int st = relevance_tc(ctx, p, s_query, s);
+    if (st) return st;
+  } else {
   prof_mark(ctx, ST_QEMBED, 0, s);
   if (identity) {
     int warps = rowsQ * H;
@@ -348,6 +445,7 @@ int score_impl(covspec_ctx* ctx, const covspec_problem* p, float* s_query, float
     }
   }
   prof_mark(ctx, ST_RELEVANCE, 1, s);
+  }
   if (cfg.act_layers > 0) {
     prof_mark(ctx, ST_ACTIVITY, 0, s);
     LayerPtrs lp{};
@@ -478,6 +576,7 @@ void covspec_default_config(covspec_config* c) {
   c->rank_cap = 128;
   c->eig_iters = 6;
   c->eig_oversample = 32;
+  c->relevance_path = 0;
 }
 
 int covspec_budgets(const covspec_config* cfg, int n, int keep, int* b_vis, int* m, int* r) {
@@ -581,6 +680,18 @@ int covspec_prune_init(const covspec_config* cfg, covspec_ctx** out) {
                                   (int)(((size_t)kPMax * kPMax + 2 * kPMax) * sizeof(double))) == cudaSuccess;
   ok = ok && cudaFuncSetAttribute(jacobi_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                   (int)((size_t)2 * kPMax * (kPMax + 1) * 4 + 4 * (kPMax / 2 + 2) * 4)) == cudaSuccess;
+  int dev = 0, cc_major = 0;
+  ok = ok && cudaGetDevice(&dev) == cudaSuccess &&
+       cudaDeviceGetAttribute(&ctx->num_sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess &&
+       cudaDeviceGetAttribute(&cc_major, cudaDevAttrComputeCapabilityMajor, dev) == cudaSuccess;
+  if (ok && cc_major == 10 && encode_tiled_fn() != nullptr) {
+    ctx->tc_ready =
+        cudaFuncSetAttribute(tc::relevance_tc_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             tc::kSmemBytes) == cudaSuccess &&
+        cudaFuncSetAttribute(tc::relevance_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             tc::kSmemBytes) == cudaSuccess;
+    ok = ctx->tc_ready;
+  }
   if (!ok) {
     g_cuda_error = std::string("context set-up: ") + cudaGetErrorString(cudaGetLastError());
     covspec_prune_destroy(ctx);
@@ -716,6 +827,7 @@ int covspec_get_device_status(covspec_ctx* ctx, void* stream) {
   CUDA_TRY(cudaMemcpyAsync(&h, ctx->status, sizeof(int), cudaMemcpyDeviceToHost, s));
   CUDA_TRY(cudaMemsetAsync(ctx->status, 0, sizeof(int), s));
   CUDA_TRY(cudaStreamSynchronize(s));
+  if (h & kStatusTimeout) return COVSPEC_ERR_TIMEOUT;
   if (h & kStatusNonFinite) return COVSPEC_ERR_NONFINITE;
   if (h & kStatusNoConverge) return COVSPEC_ERR_NOCONVERGE;
   return COVSPEC_OK;
@@ -733,6 +845,7 @@ const char* covspec_strerror(int status) {
     case COVSPEC_ERR_CUDA: return "CUDA runtime error";
     case COVSPEC_ERR_NONFINITE: return "non-finite score on the device";
     case COVSPEC_ERR_NOCONVERGE: return "small eigen-solve did not converge";
+    case COVSPEC_ERR_TIMEOUT: return "a bounded wait inside a kernel expired";
     case COVSPEC_ERR_STATIC_CAPACITY:
       return "problem exceeds the fixed scratch capacity of the allocation-free entry point";
     default: return "unknown status";

@@ -1,0 +1,480 @@
+// Fused tensor-core kernel for the query-aware score (Eq. 10) with per-head linear embeddings, bf16.
+//
+// Per work item (one 128-token tile of one request, a group of head pairs) the kernel computes
+//   Kp = X_tile * Wk[heads]^T           tcgen05.mma kind::f16, 128 x 256 accumulator in TMEM,
+//                                       operands streamed by TMA through a shared-memory ring
+//   per token and head: ||Kp||^2        epilogue warps read TMEM, keep the norm in float32 and
+//                                       restage Kp as bf16 hi + lo K-major tiles in shared memory
+//   logits = Kp * Qn[head]^T            second tcgen05.mma against the unit-length query elements,
+//                                       as hi*hi + lo*hi + hi*lo so that bf16 staging costs ~2^-16
+//   S^query = max_j,h logits / ||Kp||   row max in registers, atomic max into the score array
+// so the projected embeddings never leave the SM.  MODE 1 reuses the main loop for the query side:
+// Qp = Q * Wq^T, normalised per head and written as bf16 for MODE 0 to consume.
+//
+// Warp roles (192 threads): warps 0-3 epilogue (one TMEM lane = one token each), warp 4 TMA
+// producer, warp 5 MMA issuer and TMEM owner.  Every mbarrier wait is bounded; on expiry the CTA
+// raises a status bit, leaves its loops, frees TMEM and exits.
+#pragma once
+#include <cuda.h>
+
+#include "common.cuh"
+
+namespace covspec {
+
+constexpr int kStatusTimeout = 4;
+
+namespace tc {
+
+constexpr int kTileM = 128;            // tokens per tile (UMMA M)
+constexpr int kTileN = 256;            // projected features per pass: one pair of heads (UMMA N)
+constexpr int kHeadDim = 128;
+constexpr int kBK = 64;                // bf16 elements per k-chunk = one 128-byte swizzle row
+constexpr int kStages = 3;
+constexpr int kTT = 64;                // query elements per logits tile (UMMA N of the 2nd product)
+constexpr int kBytesA = kTileM * kBK * 2;          // 16 KB
+constexpr int kBytesB = kTileN * kBK * 2;          // 32 KB
+constexpr int kBytesStage = kBytesA + kBytesB;
+constexpr int kBytesKp = kTileM * kHeadDim * 2;    // 32 KB: two k-blocks of [128 x 64]; hi and lo
+constexpr int kBytesQ = kTT * kHeadDim * 2;        // 16 KB: two k-blocks of [64 x 64]; hi and lo
+// The query tiles (hi + lo = 32 KB) travel through the same ring slots as the main-loop chunks.
+constexpr int kSmemBytes = kStages * kBytesStage + 2 * kBytesKp + 1024 /*barriers*/ +
+                           1024 /*alignment slack*/;
+constexpr int kTmemCols = 512;
+constexpr int kLogitCol = 256;         // logits tiles live at columns 256 + 64 * buffer
+constexpr uint32_t kSpinLimit = 1u << 22;
+
+struct Params {
+  const ReqPlan* plan;
+  int batch;
+  int n_items;          // (tile, group) pairs
+  int n_groups;         // head-pair groups per tile
+  int hp_per_group;     // head pairs handled by one item
+  int n_heads;
+  int k_chunks;         // ceil(d / 64)
+  int P;                // n_heads * 128
+  long long rows_total; // MODE 1: number of query rows
+  float* s_query;       // MODE 0 out (pre-filled with -inf)
+  __nv_bfloat16* qn_out;// MODE 1 out: hi [rows_total, P] followed by lo at qn_out + qn_lo_off
+  long long qn_lo_off;
+  int* status;
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return (uint32_t)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)),
+               "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+      "selp.u32 %0, 1, 0, p;\n"
+      "}\n"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait.  Returns false when the limit expired or another role already gave up.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+  for (uint32_t i = 0; i < kSpinLimit; ++i) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((i & 255u) == 255u && *abort_flag) return false;
+  }
+  *abort_flag = 1;
+  return false;
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t smem_dst, const CUtensorMap* map, int x, int y,
+                                            uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(smem_dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(smem_u32(bar))
+      : "memory");
+}
+
+// Shared-memory matrix descriptor of a K-major bf16 tile stored as 128-byte rows with the 128-byte
+// swizzle (8-row groups of 1024 bytes): start address, stride between 8-row groups = 1024 bytes,
+// descriptor version 1, layout type 2 (128-byte swizzle).
+__device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((smem_addr & 0x3FFFFu) >> 4);
+  d |= (uint64_t)(1024u >> 4) << 32;
+  d |= (uint64_t)1 << 46;
+  d |= (uint64_t)2 << 61;
+  return d;
+}
+// Instruction descriptor: D float32, A and B bf16, both K-major, tile M x N.
+__device__ __forceinline__ uint32_t umma_idesc(int M, int N) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc,
+                                          uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "setp.ne.b32 p, %4, 0;\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n"
+      "}\n" ::"r"(d_tmem),
+      "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(
+                   smem_u32(bar))
+               : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() {
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void tc_fence_after() {
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+}
+// 32 lanes x 32 consecutive columns of float32 -> 32 registers per thread (thread = lane = row).
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
+  uint32_t r[32];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]),
+        "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]),
+        "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]),
+        "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]),
+        "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr));
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&t);
+}
+
+// Float atomic max through the sign-split integer trick (the target starts at -inf).
+__device__ __forceinline__ void atomic_max_float(float* addr, float v) {
+  if (v >= 0.f) atomicMax(reinterpret_cast<int*>(addr), __float_as_int(v));
+  else atomicMin(reinterpret_cast<unsigned*>(addr), __float_as_uint(v));
+}
+
+template <int MODE>
+__global__ void __launch_bounds__(192, 1)
+relevance_tc_kernel(const __grid_constant__ CUtensorMap map_a,   // X (MODE 0) or Q (MODE 1): [rows, d]
+                    const __grid_constant__ CUtensorMap map_b,   // Wk or Wq: [P, d]
+                    const __grid_constant__ CUtensorMap map_q,   // Qn hi: [sum T, P] (MODE 0 only)
+                    const __grid_constant__ CUtensorMap map_ql,  // Qn lo
+                    const Params prm) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint8_t* stage_base = smem;
+  uint8_t* kp_smem = smem + kStages * kBytesStage;       // hi tile, then lo tile
+  uint64_t* bars = reinterpret_cast<uint64_t*>(kp_smem + 2 * kBytesKp);
+  uint64_t* full = bars;                 // [kStages]
+  uint64_t* empty = bars + kStages;      // [kStages]
+  uint64_t* acc_full = bars + 2 * kStages;
+  uint64_t* acc_empty = acc_full + 1;
+  uint64_t* kp_ready = acc_full + 2;
+  uint64_t* kp_free = acc_full + 3;
+  uint64_t* logit_full = acc_full + 8;   // [2]
+  uint64_t* logit_empty = acc_full + 10; // [2]
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_full + 12);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+    mbar_init(acc_full, 1);
+    mbar_init(acc_empty, 128);
+    mbar_init(kp_ready, 128);
+    mbar_init(kp_free, 1);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&logit_full[i], 1); mbar_init(&logit_empty[i], 128);
+    }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 5) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
+                     smem_u32(tmem_slot)),
+                 "r"(kTmemCols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  const int n_hp = (prm.n_heads + 1) >> 1;
+
+  // Work-item decode shared by all roles.
+  auto decode = [&](int item, int& row0, int& nrows, int& txt0, int& T, int& hp_begin, int& hp_end) {
+    int tile = item / prm.n_groups, g = item % prm.n_groups;
+    hp_begin = g * prm.hp_per_group;
+    hp_end = min(n_hp, hp_begin + prm.hp_per_group);
+    if (MODE == 0) {
+      int b = find_request(tile, prm.batch, [&](int q) { return prm.plan[q].tile_off; });
+      ReqPlan rp = prm.plan[b];
+      int t = tile - rp.tile_off;
+      row0 = rp.vis_off + t * kTileM;
+      nrows = min(kTileM, rp.n - t * kTileM);
+      txt0 = rp.txt_off;
+      T = rp.t;
+    } else {
+      row0 = tile * kTileM;
+      long long rem = prm.rows_total - row0;
+      nrows = rem < kTileM ? (int)rem : kTileM;
+      txt0 = 0; T = 0;
+    }
+  };
+
+  if (warp == 4) {
+    // ---------------------------------------------------------------- TMA producer
+    if (lane == 0) {
+      uint32_t it = 0;
+      bool ok = true;
+      for (int item = blockIdx.x; item < prm.n_items && ok; item += gridDim.x) {
+        int row0, nrows, txt0, T, hp_begin, hp_end;
+        decode(item, row0, nrows, txt0, T, hp_begin, hp_end);
+        for (int hp = hp_begin; hp < hp_end && ok; ++hp) {
+          for (int kc = 0; kc < prm.k_chunks; ++kc, ++it) {
+            int s = it % kStages;
+            uint32_t ph = (it / kStages) & 1u;
+            if (!(ok = mbar_wait(&empty[s], ph ^ 1u, abort_flag))) break;
+            mbar_expect_tx(&full[s], kBytesStage);
+            uint32_t dst = smem_u32(stage_base + s * kBytesStage);
+            tma_load_2d(dst, &map_a, kc * kBK, row0, &full[s]);
+            tma_load_2d(dst + kBytesA, &map_b, kc * kBK, hp * kTileN, &full[s]);
+          }
+          if (MODE == 0 && ok) {
+            // query tiles of this head pair use the next ring slots: [hi kb0][hi kb1][lo kb0][lo kb1]
+            int heads = min(2, prm.n_heads - 2 * hp);
+            int ntt = (T + kTT - 1) / kTT;
+            for (int h = 0; h < heads && ok; ++h)
+              for (int tt = 0; tt < ntt; ++tt, ++it) {
+                int s = it % kStages;
+                uint32_t ph = (it / kStages) & 1u;
+                if (!(ok = mbar_wait(&empty[s], ph ^ 1u, abort_flag))) break;
+                mbar_expect_tx(&full[s], 2 * kBytesQ);
+                uint32_t dst = smem_u32(stage_base + s * kBytesStage);
+                int col = (2 * hp + h) * kHeadDim, y = txt0 + tt * kTT;
+                tma_load_2d(dst, &map_q, col, y, &full[s]);
+                tma_load_2d(dst + kBytesQ / 2, &map_q, col + kBK, y, &full[s]);
+                tma_load_2d(dst + kBytesQ, &map_ql, col, y, &full[s]);
+                tma_load_2d(dst + kBytesQ + kBytesQ / 2, &map_ql, col + kBK, y, &full[s]);
+              }
+          }
+        }
+      }
+    }
+    __syncwarp();
+  } else if (warp == 5) {
+    // ---------------------------------------------------------------- MMA issuer
+    if (lane == 0) {
+      const uint32_t idesc1 = umma_idesc(kTileM, kTileN);
+      const uint32_t idesc2 = umma_idesc(kTileM, kTT);
+      uint32_t it = 0, acc_it = 0, kp_it = 0, qi = 0;
+      bool ok = true;
+      for (int item = blockIdx.x; item < prm.n_items && ok; item += gridDim.x) {
+        int row0, nrows, txt0, T, hp_begin, hp_end;
+        decode(item, row0, nrows, txt0, T, hp_begin, hp_end);
+        for (int hp = hp_begin; hp < hp_end && ok; ++hp, ++acc_it) {
+          if (!(ok = mbar_wait(acc_empty, (acc_it & 1u) ^ 1u, abort_flag))) break;
+          tc_fence_after();
+          for (int kc = 0; kc < prm.k_chunks; ++kc, ++it) {
+            int s = it % kStages;
+            uint32_t ph = (it / kStages) & 1u;
+            if (!(ok = mbar_wait(&full[s], ph, abort_flag))) break;
+            tc_fence_after();
+            uint32_t a_addr = smem_u32(stage_base + s * kBytesStage);
+            uint64_t adesc = umma_desc(a_addr), bdesc = umma_desc(a_addr + kBytesA);
+#pragma unroll
+            for (int k = 0; k < kBK / 16; ++k)
+              umma_bf16(tmem_base, adesc + 2 * k, bdesc + 2 * k, idesc1, (kc | k) != 0);
+            umma_commit(&empty[s]);
+          }
+          if (!ok) break;
+          umma_commit(acc_full);
+          if (MODE == 0) {
+            int heads = min(2, prm.n_heads - 2 * hp);
+            int ntt = (T + kTT - 1) / kTT;
+            for (int h = 0; h < heads && ok; ++h, ++kp_it) {
+              if (!(ok = mbar_wait(kp_ready, kp_it & 1u, abort_flag))) break;
+              for (int tt = 0; tt < ntt; ++tt, ++qi, ++it) {
+                int s = it % kStages;
+                int buf = qi & 1;
+                if (!(ok = mbar_wait(&full[s], (it / kStages) & 1u, abort_flag))) break;
+                if (!(ok = mbar_wait(&logit_empty[buf], ((qi >> 1) & 1u) ^ 1u, abort_flag))) break;
+                tc_fence_after();
+                uint32_t kp_addr = smem_u32(kp_smem), q_addr = smem_u32(stage_base + s * kBytesStage);
+                // logits = Kp_hi Qn_hi^T + Kp_lo Qn_hi^T + Kp_hi Qn_lo^T
+#pragma unroll
+                for (int term = 0; term < 3; ++term) {
+                  uint32_t a0 = kp_addr + (term == 1 ? kBytesKp : 0);
+                  uint32_t b0 = q_addr + (term == 2 ? kBytesQ : 0);
+#pragma unroll
+                  for (int ks = 0; ks < kHeadDim / 16; ++ks) {
+                    uint64_t adesc = umma_desc(a0 + (ks >> 2) * (kBytesKp / 2)) + 2 * (ks & 3);
+                    uint64_t bdesc = umma_desc(b0 + (ks >> 2) * (kBytesQ / 2)) + 2 * (ks & 3);
+                    umma_bf16(tmem_base + kLogitCol + buf * kTT, adesc, bdesc, idesc2, (term | ks) != 0);
+                  }
+                }
+                umma_commit(&empty[s]);
+                umma_commit(&logit_full[buf]);
+              }
+              if (!ok) break;
+              umma_commit(kp_free);
+            }
+          }
+        }
+      }
+    }
+    __syncwarp();
+  } else {
+    // ---------------------------------------------------------------- epilogue (warps 0-3)
+    const int r = warp * 32 + lane;                        // token row inside the tile = TMEM lane
+    const uint32_t t_lane = tmem_base + ((uint32_t)(warp * 32) << 16);
+    uint32_t acc_it = 0, kp_it = 0, qi = 0;
+    bool ok = true;
+    for (int item = blockIdx.x; item < prm.n_items && ok; item += gridDim.x) {
+      int row0, nrows, txt0, T, hp_begin, hp_end;
+      decode(item, row0, nrows, txt0, T, hp_begin, hp_end);
+      float best = -INFINITY;
+      bool nonfinite = false;
+      for (int hp = hp_begin; hp < hp_end && ok; ++hp, ++acc_it) {
+        if (!(ok = mbar_wait(acc_full, acc_it & 1u, abort_flag))) break;
+        tc_fence_after();
+        int heads = min(2, prm.n_heads - 2 * hp);
+        for (int h = 0; h < heads && ok; ++h, ++kp_it) {
+          float ss = 0.f;
+          if (MODE == 0) {
+            if (!(ok = mbar_wait(kp_free, (kp_it & 1u) ^ 1u, abort_flag))) break;
+#pragma unroll 1
+            for (int c4 = 0; c4 < 4; ++c4) {
+              float v[32];
+              tmem_ld32(t_lane + h * kHeadDim + c4 * 32, v);
+              uint32_t pk[16], pl[16];
+#pragma unroll
+              for (int e = 0; e < 16; ++e) {
+                float a = v[2 * e], b = v[2 * e + 1];
+                ss += a * a + b * b;
+                __nv_bfloat162 hi = __floats2bfloat162_rn(a, b);
+                pk[e] = *reinterpret_cast<uint32_t*>(&hi);
+                pl[e] = pack_bf16(a - __low2float(hi), b - __high2float(hi));
+              }
+              uint8_t* rowp = kp_smem + (c4 >> 1) * (kBytesKp / 2) + r * 128;
+#pragma unroll
+              for (int q = 0; q < 4; ++q) {
+                int chunk = ((c4 & 1) * 4 + q) ^ (r & 7);
+                *reinterpret_cast<uint4*>(rowp + chunk * 16) =
+                    make_uint4(pk[4 * q], pk[4 * q + 1], pk[4 * q + 2], pk[4 * q + 3]);
+                *reinterpret_cast<uint4*>(rowp + kBytesKp + chunk * 16) =
+                    make_uint4(pl[4 * q], pl[4 * q + 1], pl[4 * q + 2], pl[4 * q + 3]);
+              }
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            tc_fence_before();
+            mbar_arrive(kp_ready);
+            if (h == heads - 1) mbar_arrive(acc_empty);    // the accumulator is fully drained
+            nonfinite |= !(ss <= 3.402823466e38f);
+            float inv = 0.f;
+            if (ss > 1.17549435e-38f) { inv = rsqrtf(ss); inv = inv * (1.5f - 0.5f * ss * inv * inv); }
+            int ntt = (T + kTT - 1) / kTT;
+            for (int tt = 0; tt < ntt; ++tt, ++qi) {
+              int buf = qi & 1;
+              if (!(ok = mbar_wait(&logit_full[buf], (qi >> 1) & 1u, abort_flag))) break;
+              tc_fence_after();
+#pragma unroll 1
+              for (int c2 = 0; c2 < 2; ++c2) {
+                float v[32];
+                tmem_ld32(t_lane + kLogitCol + buf * kTT + c2 * 32, v);
+                int jbase = tt * kTT + c2 * 32;
+#pragma unroll
+                for (int e = 0; e < 32; ++e)
+                  if (jbase + e < T) {
+                    nonfinite |= v[e] != v[e];
+                    best = fmaxf(best, v[e] * inv);
+                  }
+              }
+              tc_fence_before();
+              mbar_arrive(&logit_empty[buf]);
+            }
+          } else {
+            // MODE 1: unit-length bf16 head slice of the projected query element to global memory.
+#pragma unroll 1
+            for (int c4 = 0; c4 < 4; ++c4) {
+              float v[32];
+              tmem_ld32(t_lane + h * kHeadDim + c4 * 32, v);
+#pragma unroll
+              for (int e = 0; e < 32; ++e) ss += v[e] * v[e];
+            }
+            float inv = 0.f;
+            if (ss > 1.17549435e-38f) { inv = rsqrtf(ss); inv = inv * (1.5f - 0.5f * ss * inv * inv); }
+            if (!(ss <= 3.402823466e38f)) inv = __int_as_float(0x7fc00000);
+#pragma unroll 1
+            for (int c4 = 0; c4 < 4; ++c4) {
+              float v[32];
+              tmem_ld32(t_lane + h * kHeadDim + c4 * 32, v);
+              if (r < nrows) {
+                __nv_bfloat16* dst = prm.qn_out + (size_t)(row0 + r) * prm.P +
+                                     (size_t)(2 * hp + h) * kHeadDim + c4 * 32;
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                  uint32_t ph[4], pw[4];
+#pragma unroll
+                  for (int e = 0; e < 4; ++e) {
+                    float a = v[8 * q + 2 * e] * inv, b = v[8 * q + 2 * e + 1] * inv;
+                    __nv_bfloat162 hi = __floats2bfloat162_rn(a, b);
+                    ph[e] = *reinterpret_cast<uint32_t*>(&hi);
+                    pw[e] = pack_bf16(a - __low2float(hi), b - __high2float(hi));
+                  }
+                  *reinterpret_cast<uint4*>(dst + q * 8) = make_uint4(ph[0], ph[1], ph[2], ph[3]);
+                  *reinterpret_cast<uint4*>(dst + prm.qn_lo_off + q * 8) =
+                      make_uint4(pw[0], pw[1], pw[2], pw[3]);
+                }
+              }
+            }
+            if (h == heads - 1) { tc_fence_before(); mbar_arrive(acc_empty); }
+          }
+        }
+      }
+      if (MODE == 0 && ok && r < nrows) {
+        if (nonfinite) atomicOr(prm.status, kStatusNonFinite);
+        else atomic_max_float(prm.s_query + row0 + r, best);
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 5) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
+                 "r"(kTmemCols)
+                 : "memory");
+  }
+  if (threadIdx.x == 0 && *abort_flag) atomicOr(prm.status, kStatusTimeout);
+}
+
+// Fills the score array with -inf so that the relevance kernel can combine head groups with an
+// atomic max.
+__global__ void fill_neg_inf_kernel(float* __restrict__ s, long long n) {
+  long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) s[i] = -INFINITY;
+}
+
+}  // namespace tc
+}  // namespace covspec
