@@ -19,12 +19,13 @@ struct ReqPlan {
   int txt_off, t;          // rows of Q
   int b_vis, m, r, p;      // keep budget, preselect size, rank, basis size (p = 0: stage 2 skipped)
   int keep_off, presel_off;
-  int ldm;                 // m rounded up to a multiple of 4 (row stride of G and of the bases)
+  int ldm;                 // m rounded up to a multiple of 4 (row stride of the float32 Gram matrix)
   int stage2;              // 1 when b_vis < m (Eq. 13-15 are evaluated)
   int tile_off;            // first 128-token tile of the request in the tensor-core relevance kernel
+  int gram_tile_off;       // first lower-triangle 128 x 128 tile of the request's Gram matrix
+  int ptile_off;           // first 128-row tile of the request's subspace-iteration block
   int pad_;
-  long long g_off;         // float offset of the request's Gram matrix
-  long long u_off;         // float offset of the request's basis buffers (p x ldm)
+  long long g_off;         // float offset of the request's float32 Gram matrix (float32 inputs only)
 };
 
 // One dense product C[m x n] = A[m x k] * op(B) handled by the tiled SIMT kernel.

@@ -6,6 +6,7 @@
 #include <stdio.h>
 #include <string.h>
 
+#include <algorithm>
 #include <mutex>
 #include <string>
 #include <vector>
@@ -14,6 +15,7 @@
 #include "eig_kernels.cuh"
 #include "gemm_simt.cuh"
 #include "relevance_tc.cuh"
+#include "subspace_tc.cuh"
 #include "score_kernels.cuh"
 #include "select_kernels.cuh"
 
@@ -34,17 +36,10 @@ thread_local std::string g_cuda_error;
 
 inline long long round_up(long long v, long long a) { return (v + a - 1) / a * a; }
 
-// Gemm tables kept on the device for the subspace iteration (one entry per stage-2 request).
+// Gemm tables kept on the device (one entry per stage-2 request); only the float32 configuration
+// still forms its Gram matrix on the CUDA cores.
 enum TableId {
-  T_GRAM_G = 0,   // G   = Zg Zg^T            (storage dtype operands)
-  T_MULG_01,      // U1  = U0 G
-  T_MULG_10,      // U0  = U1 G
-  T_GRAM_U1,      // B64 = U1 U1^T            (float64)
-  T_GRAM_U0,      // B64 = U0 U0^T
-  T_APPLY_10,     // U0  = Linv U1
-  T_APPLY_01,     // U1  = Linv U0
-  T_RR,           // S32 = U0 U1^T            (Rayleigh-Ritz matrix, U0 = U1 G)
-  T_RITZ,         // U0  = Wr U1              (Ritz vectors)
+  T_GRAM_G = 0,   // G = Zg Zg^T (float32 operands)
   T_COUNT
 };
 
@@ -62,8 +57,9 @@ struct Plan {
   std::vector<int> keep_offsets, presel_offsets;
   int n_stage2 = 0;
   int tiles[T_COUNT] = {0};
-  int t_max = 0, p_max = 0, m_max = 0;
+  int t_max = 0, p_max = 0, m_max = 0, r_max = 0;
   int n_tiles = 0;                            // 128-token tiles over all requests
+  int n_gram_tiles = 0, n_ptiles = 0;         // lower-triangle Gram tiles / 128-row block tiles (stage 2)
   long long total_vis = 0, total_txt = 0, total_keep = 0, total_presel = 0;
   bool valid = false;
 };
@@ -87,11 +83,17 @@ struct covspec_ctx {
   int* presel = nullptr;
   float* energy = nullptr;
   void* Zg = nullptr;
-  float* G = nullptr;
-  long long g_cap = 0, u_cap = 0;
-  float *U0 = nullptr, *U1 = nullptr;
-  double* B64 = nullptr;
-  float *Linv = nullptr, *S32 = nullptr, *Wr = nullptr, *theta = nullptr;
+  float* G = nullptr;                    // float32 Gram matrices (float32 inputs only)
+  long long g_cap = 0;
+  // subspace iteration (see subspace_tc.cuh for the layouts)
+  int ld = 0;                            // row stride of the G and Y planes
+  long long cap_rows = 0, cap_ptiles = 0;
+  __nv_bfloat16 *Ghi = nullptr, *Glo = nullptr;
+  __nv_bfloat16* Yp[2][2] = {{nullptr, nullptr}, {nullptr, nullptr}};   // [buffer][hi / lo]
+  float* Yf = nullptr;
+  double* partial = nullptr;
+  float *Lbuf = nullptr, *Ut = nullptr, *theta = nullptr;
+  CUtensorMap map_zg, map_gh, map_gl, map_y[2][2];
   // pinned staging for the plan upload
   char* h_stage = nullptr;
   long long stage_bytes = 0;
@@ -183,8 +185,11 @@ int get_plan(covspec_ctx* ctx, const covspec_problem* p, cudaStream_t stream) {
   pl.keep_offsets.assign(B + 1, 0);
   pl.presel_offsets.assign(B + 1, 0);
   pl.n_stage2 = 0; pl.t_max = 0; pl.p_max = 0; pl.m_max = 0; pl.n_tiles = 0;
-  long long g_off = 0, u_off = 0;
+  pl.n_gram_tiles = 0; pl.n_ptiles = 0;
+  pl.r_max = 0;
+  long long g_off = 0;
   int n_max = 0;
+  bool f32 = cfg.dtype == COVSPEC_F32;
   for (int b = 0; b < B; ++b) {
     ReqPlan& r = pl.req[b];
     r.vis_off = p->vis_offsets[b]; r.n = p->vis_offsets[b + 1] - r.vis_off;
@@ -193,19 +198,25 @@ int get_plan(covspec_ctx* ctx, const covspec_problem* p, cudaStream_t stream) {
     if (st) return COVSPEC_ERR_SHAPE;
     r.stage2 = r.b_vis < r.m;
     r.p = 0;
+    r.ldm = (int)round_up(r.m, 4);
+    r.tile_off = pl.n_tiles;
+    pl.n_tiles += (r.n + tc::kTileM - 1) / tc::kTileM;
+    r.gram_tile_off = pl.n_gram_tiles;
+    r.ptile_off = pl.n_ptiles;
+    r.g_off = g_off;
     if (r.stage2) {
       r.p = r.r + cfg.eig_oversample;
       if (r.p > r.m) r.p = r.m;
       ++pl.n_stage2;
+      int nt = (r.m + sub::kTile - 1) / sub::kTile;
+      pl.n_gram_tiles += nt * (nt + 1) / 2;
+      pl.n_ptiles += nt;
+      if (f32) g_off += (long long)r.m * r.ldm;
+      if (r.r > pl.r_max) pl.r_max = r.r;
     }
-    r.ldm = (int)round_up(r.m, 4);
-    r.tile_off = pl.n_tiles;
-    pl.n_tiles += (r.n + tc::kTileM - 1) / tc::kTileM;
     r.keep_off = pl.keep_offsets[b]; r.presel_off = pl.presel_offsets[b];
     pl.keep_offsets[b + 1] = r.keep_off + r.b_vis;
     pl.presel_offsets[b + 1] = r.presel_off + r.m;
-    r.g_off = g_off; r.u_off = u_off;
-    if (r.stage2) { g_off += (long long)r.m * r.ldm; u_off += (long long)r.p * r.ldm; }
     if (r.t > pl.t_max) pl.t_max = r.t;
     if (r.p > pl.p_max) pl.p_max = r.p;
     if (r.m > pl.m_max) pl.m_max = r.m;
@@ -214,11 +225,11 @@ int get_plan(covspec_ctx* ctx, const covspec_problem* p, cudaStream_t stream) {
   pl.total_vis = p->vis_offsets[B]; pl.total_txt = p->txt_offsets[B];
   pl.total_keep = pl.keep_offsets[B]; pl.total_presel = pl.presel_offsets[B];
   if (pl.total_vis > cfg.max_total_vis || pl.total_txt > cfg.max_total_txt ||
-      n_max > cfg.max_vis_per_req || g_off > ctx->g_cap || u_off > ctx->u_cap ||
-      pl.total_presel > ctx->cfg.max_total_presel)
+      n_max > cfg.max_vis_per_req || g_off > ctx->g_cap || pl.m_max > ctx->cfg.max_presel_per_req ||
+      pl.total_presel > ctx->cfg.max_total_presel || pl.n_ptiles > ctx->cap_ptiles)
     return COVSPEC_ERR_WORKSPACE;
 
-  // Stage plan + gemm tables in pinned memory and upload.
+  // Stage plan + gemm table in pinned memory and upload.
   if (ctx->stage_free) CUDA_TRY(cudaEventSynchronize(ctx->stage_free));
   ReqPlan* h_plan = reinterpret_cast<ReqPlan*>(ctx->h_stage);
   GemmProb* h_tab = reinterpret_cast<GemmProb*>(ctx->h_stage + round_up(sizeof(ReqPlan) * cfg.max_batch, 256));
@@ -226,39 +237,20 @@ int get_plan(covspec_ctx* ctx, const covspec_problem* p, cudaStream_t stream) {
   int mb = cfg.max_batch;
   for (int t = 0; t < T_COUNT; ++t) pl.tiles[t] = 0;
   int s2 = 0;
-  char* Zg = reinterpret_cast<char*>(ctx->Zg);
-  for (int b = 0; b < B; ++b) {
-    const ReqPlan& r = pl.req[b];
-    if (!r.stage2) continue;
-    auto tiles_of = [](int m, int n, int* tn) {
-      *tn = (n + kGemmBN - 1) / kGemmBN;
-      return ((m + kGemmBM - 1) / kGemmBM) * *tn;
-    };
-    auto put = [&](int t, const void* A, const void* Bp, void* C, int m, int n, int k, int lda,
-                   int ldb, int ldc) {
-      GemmProb& g = h_tab[(size_t)t * mb + s2];
-      g.A = A; g.B = Bp; g.C = C; g.m = m; g.n = n; g.k = k; g.lda = lda; g.ldb = ldb; g.ldc = ldc;
-      g.tile_start = pl.tiles[t];
-      pl.tiles[t] += tiles_of(m, n, &g.tiles_n);
-    };
-    const void* zg = Zg + (size_t)r.presel_off * cfg.d * ctx->esize;
-    float* G = ctx->G + r.g_off;
-    float *U0 = ctx->U0 + r.u_off, *U1 = ctx->U1 + r.u_off;
-    double* B64 = ctx->B64 + (size_t)b * kPMax * kPMax;
-    float* Linv = ctx->Linv + (size_t)b * kPMax * kPMax;
-    float* S32 = ctx->S32 + (size_t)b * kPMax * kPMax;
-    float* Wr = ctx->Wr + (size_t)b * kPMax * kPMax;
-    int ldp = (int)round_up(r.p, 4);
-    put(T_GRAM_G, zg, zg, G, r.m, r.m, cfg.d, cfg.d, cfg.d, r.ldm);
-    put(T_MULG_01, U0, G, U1, r.p, r.m, r.m, r.ldm, r.ldm, r.ldm);
-    put(T_MULG_10, U1, G, U0, r.p, r.m, r.m, r.ldm, r.ldm, r.ldm);
-    put(T_GRAM_U1, U1, U1, B64, r.p, r.p, r.m, r.ldm, r.ldm, kPMax);
-    put(T_GRAM_U0, U0, U0, B64, r.p, r.p, r.m, r.ldm, r.ldm, kPMax);
-    put(T_APPLY_10, Linv, U1, U0, r.p, r.m, r.p, ldp, r.ldm, r.ldm);
-    put(T_APPLY_01, Linv, U0, U1, r.p, r.m, r.p, ldp, r.ldm, r.ldm);
-    put(T_RR, U0, U1, S32, r.p, r.p, r.m, r.ldm, r.ldm, ldp);
-    put(T_RITZ, Wr, U1, U0, r.r, r.m, r.p, ldp, r.ldm, r.ldm);
-    ++s2;
+  if (f32) {
+    char* Zg = reinterpret_cast<char*>(ctx->Zg);
+    for (int b = 0; b < B; ++b) {
+      const ReqPlan& r = pl.req[b];
+      if (!r.stage2) continue;
+      GemmProb& g = h_tab[(size_t)T_GRAM_G * mb + s2];
+      const void* zg = Zg + (size_t)r.presel_off * cfg.d * ctx->esize;
+      g.A = zg; g.B = zg; g.C = ctx->G + r.g_off;
+      g.m = r.m; g.n = r.m; g.k = cfg.d; g.lda = cfg.d; g.ldb = cfg.d; g.ldc = r.ldm;
+      g.tile_start = pl.tiles[T_GRAM_G];
+      g.tiles_n = (r.m + kGemmBN - 1) / kGemmBN;
+      pl.tiles[T_GRAM_G] += ((r.m + kGemmBM - 1) / kGemmBM) * g.tiles_n;
+      ++s2;
+    }
   }
   CUDA_TRY(cudaMemcpyAsync(ctx->d_plan, h_plan, sizeof(ReqPlan) * B, cudaMemcpyHostToDevice, stream));
   if (s2 > 0)
@@ -490,39 +482,52 @@ int select_impl(covspec_ctx* ctx, const covspec_problem* p, const float* s_fused
         reinterpret_cast<const uint4*>(p->X), presel, ctx->d_plan, B, 1, vec16,
         reinterpret_cast<uint4*>(ctx->Zg), nullptr);
     LAUNCH_CHECK(ctx);
-    int st = launch_table<T, T, float, float, false>(ctx, T_GRAM_G, 1, s);
-    if (st) return st;
+    int st;
+    dim3 gb(std::min(64, (pl.p_max * pl.m_max + 255) / 256 + 1), B);
+    if (cfg.dtype == COVSPEC_BF16) {
+      sub::GramParams gp{};
+      gp.plan = ctx->d_plan; gp.batch = B; gp.n_items = pl.n_gram_tiles;
+      gp.k_chunks = (cfg.d + sub::kBK - 1) / sub::kBK;
+      gp.g_hi = ctx->Ghi; gp.g_lo = ctx->Glo; gp.ld = ctx->ld; gp.status = ctx->status;
+      int grid = std::min(pl.n_gram_tiles, ctx->num_sms);
+      sub::gram_tc_kernel<<<grid, 192, sub::kGramSmem, s>>>(ctx->map_zg, gp);
+      LAUNCH_CHECK(ctx);
+    } else {
+      if ((st = launch_table<T, T, float, float, false>(ctx, T_GRAM_G, 1, s))) return st;
+      dim3 gs(std::min(64, (pl.m_max * pl.m_max + 255) / 256 + 1), B);
+      sub::split_planes_kernel<<<gs, 256, 0, s>>>(ctx->d_plan, ctx->G, ctx->Ghi, ctx->Glo, ctx->ld);
+      LAUNCH_CHECK(ctx);
+    }
     prof_mark(ctx, ST_GRAM, 1, s);
     prof_mark(ctx, ST_EIG, 0, s);
-    int init_blocks = (pl.p_max * (pl.m_max + 3) + 255) / 256;
-    dim3 gi(init_blocks > 64 ? 64 : init_blocks, B);
-    eig_init_kernel<<<gi, 256, 0, s>>>(ctx->d_plan, ctx->U0);
+    sub::basis_init_kernel<<<gb, 256, 0, s>>>(ctx->d_plan, ctx->Yp[0][0], ctx->Yp[0][1], ctx->Yp[1][0],
+                                              ctx->Yp[1][1], ctx->ld);
     LAUNCH_CHECK(ctx);
-    size_t chol_smem = ((size_t)pl.p_max * pl.p_max + 2 * pl.p_max) * sizeof(double);
-    size_t jac_smem = (size_t)2 * pl.p_max * (pl.p_max + 1) * sizeof(float) +
-                      (size_t)4 * ((pl.p_max + 1) / 2 + 1) * sizeof(float);
-    for (int it = 0; it < cfg.eig_iters; ++it) {
-      // U1 = U0 G ; orthonormalise rows of U1 into U0
-      if ((st = launch_table<float, float, float, float, false>(ctx, T_MULG_01, 0, s))) return st;
-      if ((st = launch_table<float, float, double, double, false>(ctx, T_GRAM_U1, 0, s))) return st;
-      chol_inv_kernel<<<B, 1024, chol_smem, s>>>(ctx->d_plan, ctx->B64, ctx->Linv);
+    size_t tri_smem = ((size_t)pl.p_max * (pl.p_max + 1) / 2 + 2 * pl.p_max) * sizeof(double);
+    size_t ritz_smem = tri_smem + ((size_t)pl.p_max * (pl.p_max | 1) + pl.p_max) * sizeof(float);
+    int grid = std::min(pl.n_ptiles, ctx->num_sms);
+    for (int pass = 0; pass <= cfg.eig_iters; ++pass) {
+      sub::PowerParams pp{};
+      pp.plan = ctx->d_plan; pp.batch = B; pp.n_items = pl.n_ptiles;
+      pp.identity = pass == 0; pp.last = pass == cfg.eig_iters;
+      pp.lbuf = ctx->Lbuf;
+      int in = pass & 1, out = in ^ 1;
+      pp.y_hi = ctx->Yp[out][0]; pp.y_lo = ctx->Yp[out][1]; pp.ld = ctx->ld;
+      pp.yf = ctx->Yf; pp.partial = ctx->partial; pp.status = ctx->status;
+      sub::power_tc_kernel<<<grid, 192, sub::kPowSmem, s>>>(ctx->map_gh, ctx->map_gl, ctx->map_y[in][0],
+                                                            ctx->map_y[in][1], pp);
       LAUNCH_CHECK(ctx);
-      if ((st = launch_table<float, float, float, float, true>(ctx, T_APPLY_10, 0, s))) return st;
+      if (pass < cfg.eig_iters) {
+        chol_kernel<<<B, 512, tri_smem, s>>>(ctx->d_plan, ctx->partial, ctx->Lbuf);
+        LAUNCH_CHECK(ctx);
+      }
     }
-    // second Cholesky-QR pass for an orthonormal basis: U1 = orth(U0)
-    if ((st = launch_table<float, float, double, double, false>(ctx, T_GRAM_U0, 0, s))) return st;
-    chol_inv_kernel<<<B, 1024, chol_smem, s>>>(ctx->d_plan, ctx->B64, ctx->Linv);
+    ritz_kernel<<<B, 1024, ritz_smem, s>>>(ctx->d_plan, ctx->partial, ctx->Ut, ctx->theta, 30, ctx->status);
     LAUNCH_CHECK(ctx);
-    if ((st = launch_table<float, float, float, float, true>(ctx, T_APPLY_01, 0, s))) return st;
-    // Rayleigh-Ritz: U0 = U1 G, S = U0 U1^T, eig(S), Ritz vectors U0 = Wr U1
-    if ((st = launch_table<float, float, float, float, false>(ctx, T_MULG_10, 0, s))) return st;
-    if ((st = launch_table<float, float, float, float, false>(ctx, T_RR, 0, s))) return st;
-    jacobi_kernel<<<B, 1024, jac_smem, s>>>(ctx->d_plan, ctx->S32, ctx->Wr, ctx->theta, 30, ctx->status);
-    LAUNCH_CHECK(ctx);
-    if ((st = launch_table<float, float, float, float, true>(ctx, T_RITZ, 0, s))) return st;
   }
-  dim3 ge((pl.m_max + 255) / 256, B);
-  energy_kernel<<<ge, 256, 0, s>>>(ctx->d_plan, ctx->U0, ctx->theta, energy);
+  dim3 ge((pl.m_max + 63) / 64, B);
+  size_t en_smem = (size_t)pl.p_max * pl.r_max * sizeof(float);
+  energy_kernel<<<ge, 256, en_smem, s>>>(ctx->d_plan, ctx->Yf, ctx->Ut, energy);
   LAUNCH_CHECK(ctx);
   if (pl.n_stage2 > 0) prof_mark(ctx, ST_EIG, 1, s);
   prof_mark(ctx, ST_FINAL, 0, s);
@@ -623,12 +628,15 @@ int covspec_prune_init(const covspec_config* cfg, covspec_ctx** out) {
   rows = rows < 256 ? 256 : rows / 64 * 64;
   if (rows > c.max_total_vis) rows = round_up(c.max_total_vis, 64);
   ctx->kp_rows = c.n_heads > 0 ? rows : 0;
+  bool f32 = c.dtype == COVSPEC_F32;
   long long ldm_max = round_up(c.max_presel_per_req, 4);
-  ctx->g_cap = (c.max_total_presel + 4ll * c.max_batch) * ldm_max;
-  ctx->u_cap = (long long)kPMax * (c.max_total_presel + 4ll * c.max_batch);
+  ctx->g_cap = f32 ? (c.max_total_presel + 4ll * c.max_batch) * ldm_max : 0;
+  ctx->ld = (int)round_up(c.max_presel_per_req, 64);
+  ctx->cap_rows = c.max_total_presel;
+  ctx->cap_ptiles = c.max_total_presel / sub::kTile + c.max_batch;
 
   long long off = 0;
-  auto carve = [&](long long bytes) { long long o = off; off += round_up(bytes, 256); return o; };
+  auto carve = [&](long long bytes) { long long o = off; off += round_up(bytes, 1024); return o; };
   long long o_status = carve(256);
   long long o_plan = carve(sizeof(ReqPlan) * c.max_batch);
   long long o_tab = carve(sizeof(GemmProb) * (long long)T_COUNT * c.max_batch);
@@ -639,10 +647,15 @@ int covspec_prune_init(const covspec_config* cfg, covspec_ctx** out) {
   long long o_presel = carve(4ll * c.max_total_presel), o_energy = carve(4ll * c.max_total_presel);
   long long o_zg = carve((long long)ctx->esize * c.max_total_presel * c.d);
   long long o_g = carve(4ll * ctx->g_cap);
-  long long o_u0 = carve(4ll * ctx->u_cap), o_u1 = carve(4ll * ctx->u_cap);
-  long long small = (long long)c.max_batch * kPMax * kPMax;
-  long long o_b64 = carve(8ll * small), o_linv = carve(4ll * small), o_s32 = carve(4ll * small);
-  long long o_wr = carve(4ll * small), o_theta = carve(4ll * c.max_batch * kPMax);
+  long long plane = 2ll * ctx->cap_rows * ctx->ld;
+  long long o_gh = carve(plane), o_gl = carve(plane);
+  long long yplane = 2ll * c.max_batch * kPMax * ctx->ld;
+  long long o_y[2][2];
+  for (int i = 0; i < 2; ++i) for (int j = 0; j < 2; ++j) o_y[i][j] = carve(yplane);
+  long long o_yf = carve(4ll * ctx->cap_rows * kPMax);
+  long long o_part = carve(8ll * ctx->cap_ptiles * sub::kTriMax);
+  long long o_lbuf = carve(4ll * c.max_batch * sub::kLbufStride);
+  long long o_ut = carve(4ll * c.max_batch * kPMax * kPMax), o_theta = carve(4ll * c.max_batch * kPMax);
   ctx->ws_bytes = off;
   cudaError_t e = cudaMalloc(&ctx->ws, (size_t)off);
   if (e != cudaSuccess) {
@@ -663,12 +676,14 @@ int covspec_prune_init(const covspec_config* cfg, covspec_ctx** out) {
   ctx->energy = reinterpret_cast<float*>(w + o_energy);
   ctx->Zg = w + o_zg;
   ctx->G = reinterpret_cast<float*>(w + o_g);
-  ctx->U0 = reinterpret_cast<float*>(w + o_u0);
-  ctx->U1 = reinterpret_cast<float*>(w + o_u1);
-  ctx->B64 = reinterpret_cast<double*>(w + o_b64);
-  ctx->Linv = reinterpret_cast<float*>(w + o_linv);
-  ctx->S32 = reinterpret_cast<float*>(w + o_s32);
-  ctx->Wr = reinterpret_cast<float*>(w + o_wr);
+  ctx->Ghi = reinterpret_cast<__nv_bfloat16*>(w + o_gh);
+  ctx->Glo = reinterpret_cast<__nv_bfloat16*>(w + o_gl);
+  for (int i = 0; i < 2; ++i)
+    for (int j = 0; j < 2; ++j) ctx->Yp[i][j] = reinterpret_cast<__nv_bfloat16*>(w + o_y[i][j]);
+  ctx->Yf = reinterpret_cast<float*>(w + o_yf);
+  ctx->partial = reinterpret_cast<double*>(w + o_part);
+  ctx->Lbuf = reinterpret_cast<float*>(w + o_lbuf);
+  ctx->Ut = reinterpret_cast<float*>(w + o_ut);
   ctx->theta = reinterpret_cast<float*>(w + o_theta);
   ctx->stage_bytes = round_up(sizeof(ReqPlan) * c.max_batch, 256) +
                      sizeof(GemmProb) * (long long)T_COUNT * c.max_batch;
@@ -676,21 +691,43 @@ int covspec_prune_init(const covspec_config* cfg, covspec_ctx** out) {
             cudaMallocHost(&ctx->h_stage, (size_t)ctx->stage_bytes) == cudaSuccess &&
             cudaEventCreateWithFlags(&ctx->stage_free, cudaEventDisableTiming) == cudaSuccess;
   // the small dense kernels need more than the default 48 KB of dynamic shared memory
-  ok = ok && cudaFuncSetAttribute(chol_inv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                  (int)(((size_t)kPMax * kPMax + 2 * kPMax) * sizeof(double))) == cudaSuccess;
-  ok = ok && cudaFuncSetAttribute(jacobi_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                  (int)((size_t)2 * kPMax * (kPMax + 1) * 4 + 4 * (kPMax / 2 + 2) * 4)) == cudaSuccess;
+  const int tri_bytes = (int)(((size_t)kPMax * (kPMax + 1) / 2 + 2 * kPMax) * sizeof(double));
+  ok = ok && cudaFuncSetAttribute(chol_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, tri_bytes) == cudaSuccess;
+  ok = ok && cudaFuncSetAttribute(ritz_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                  tri_bytes + (int)(((size_t)kPMax * (kPMax | 1) + kPMax) * sizeof(float))) == cudaSuccess;
+  ok = ok && cudaFuncSetAttribute(energy_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                  (int)((size_t)kPMax * kPMax * sizeof(float))) == cudaSuccess;
   int dev = 0, cc_major = 0;
   ok = ok && cudaGetDevice(&dev) == cudaSuccess &&
        cudaDeviceGetAttribute(&ctx->num_sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess &&
        cudaDeviceGetAttribute(&cc_major, cudaDevAttrComputeCapabilityMajor, dev) == cudaSuccess;
-  if (ok && cc_major == 10 && encode_tiled_fn() != nullptr) {
+  if (ok && (cc_major != 10 || encode_tiled_fn() == nullptr)) {
+    g_cuda_error = "the library needs a compute capability 10.x device and cuTensorMapEncodeTiled";
+    covspec_prune_destroy(ctx);
+    return COVSPEC_ERR_UNSUPPORTED;
+  }
+  if (ok) {
     ctx->tc_ready =
         cudaFuncSetAttribute(tc::relevance_tc_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              tc::kSmemBytes) == cudaSuccess &&
         cudaFuncSetAttribute(tc::relevance_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             tc::kSmemBytes) == cudaSuccess;
+                             tc::kSmemBytes) == cudaSuccess &&
+        cudaFuncSetAttribute(sub::gram_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             sub::kGramSmem) == cudaSuccess &&
+        cudaFuncSetAttribute(sub::power_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             sub::kPowSmem) == cudaSuccess;
     ok = ctx->tc_ready;
+  }
+  if (ok) {
+    // tensor maps over the workspace arrays of the subspace iteration (fixed for the context)
+    int st = COVSPEC_OK;
+    if (!f32) st = make_map_bf16(&ctx->map_zg, ctx->Zg, c.max_total_presel, c.d, sub::kTile);
+    if (!st) st = make_map_bf16(&ctx->map_gh, ctx->Ghi, ctx->cap_rows, ctx->ld, sub::kTile);
+    if (!st) st = make_map_bf16(&ctx->map_gl, ctx->Glo, ctx->cap_rows, ctx->ld, sub::kTile);
+    for (int i = 0; i < 2 && !st; ++i)
+      for (int j = 0; j < 2 && !st; ++j)
+        st = make_map_bf16(&ctx->map_y[i][j], ctx->Yp[i][j], (long long)c.max_batch * kPMax, ctx->ld, kPMax);
+    if (st) { covspec_prune_destroy(ctx); return st; }
   }
   if (!ok) {
     g_cuda_error = std::string("context set-up: ") + cudaGetErrorString(cudaGetLastError());

@@ -1,0 +1,523 @@
+// Tensor-core kernels of the low-rank redundancy step (Eq. 13-15): the Gram matrix of the stacked
+// preselected tokens and the block power step of the subspace iteration that reaches its top-r
+// eigenspace.
+//
+// G = Z_M^T Z_M (Eq. 13-14; its eigenpairs are sigma_k^2 and the right singular vectors of Z_M) is
+// produced by tcgen05.mma kind::f16 from the gathered bf16 rows, accumulated in float32 in TMEM and
+// stored as two bf16 planes G = G_hi + G_lo (16 mantissa bits), which is the operand format of the
+// power step.  One power step computes, per 128-row tile of one request,
+//     T      = G[tile, :] * Y                    3 MMAs per k-step: hi*hi + lo*hi + hi*lo
+//     Y_next = T * L^-T                          forward substitution per row, L = chol(Y^T Y)
+//     B_tile = Y_next[tile]^T Y_next[tile]       float64 partial Gram of the new block
+// so that orthonormalising the previous block (Y L^-T) never needs its own pass over memory: the
+// triangular factor is applied to the product instead (G (Y L^-T) = (G Y) L^-T).
+//
+// Layouts.  All requests share 2-D arrays so that one tensor map serves the whole batch:
+//   G planes   [sum M_b (+pad), ld]  row presel_off(b) + i, column j          (ld = max M rounded to 64)
+//   Y planes   [batch * 160, ld]     row b*160 + basis vector, column = token position (K-major B operand)
+//   Yf         [sum M_b, 160]        float32 copy of the last block, one token per row
+//   partial    [tiles, 12880]        packed lower triangles (a*(a+1)/2 + b) in float64
+// Columns of G and Y between M_b and the next multiple of 64 are kept finite / zero respectively so
+// that whole 64-wide k-chunks can be multiplied.
+#pragma once
+#include "tc_common.cuh"
+
+namespace covspec {
+namespace sub {
+
+using namespace tc;
+
+constexpr int kTile = 128;                 // rows per tile (UMMA M); Gram column tile (UMMA N)
+constexpr int kBK = 64;                    // bf16 elements per k-chunk (one 128-byte swizzle row)
+constexpr int kTriMax = kPMax * (kPMax + 1) / 2;          // 12880 packed lower-triangle entries
+// Triangular factor as the power step reads it: row i holds L[j][i] for j = (i & ~3) .. P-1 so that
+// 8-column blocks are two aligned float4 loads.  Largest size (P = 160) and the per-request stride
+// (factor followed by the reciprocal diagonal).
+constexpr int kLtFloats = kPMax * kPMax - 8 * (kPMax / 4) * (kPMax / 4 - 1);   // 13120
+constexpr int kLbufStride = kLtFloats + kPMax;                                  // 13280
+
+__host__ __device__ __forceinline__ int tri_index(int a, int b) { return a * (a + 1) / 2 + b; }
+// Offset of row i of the padded upper-triangular layout for width P (a multiple of 4).
+__host__ __device__ __forceinline__ int lt_row_offset(int i, int P) {
+  int a = i >> 2, b = i & 3;
+  return i * P - 8 * a * (a - 1) - 4 * a * b;
+}
+
+__device__ __forceinline__ void split_bf16(float v, __nv_bfloat16& hi, __nv_bfloat16& lo) {
+  hi = __float2bfloat16_rn(v);
+  lo = __float2bfloat16_rn(v - __bfloat162float(hi));
+}
+
+// Row / column tile of the t-th lower-triangle tile (row-major over (ti, tj <= ti)).
+__device__ __forceinline__ void tri_decode(int t, int& ti, int& tj) {
+  ti = (int)((sqrtf(8.f * (float)t + 1.f) - 1.f) * 0.5f);
+  while ((ti + 1) * (ti + 2) / 2 <= t) ++ti;
+  while (ti * (ti + 1) / 2 > t) --ti;
+  tj = t - ti * (ti + 1) / 2;
+}
+
+// ================================================================================================
+// Gram kernel
+// ================================================================================================
+constexpr int kGramStages = 6;
+constexpr int kGramStageBytes = 2 * kTile * kBK * 2;     // A and B tile, 16 KB each
+constexpr int kGramSmem = kGramStages * kGramStageBytes + 1024 + 1024;
+constexpr int kGramTmemCols = 256;                        // two 128-column accumulators
+
+struct GramParams {
+  const ReqPlan* plan;
+  int batch;
+  int n_items;          // lower-triangle tiles over all stage-2 requests
+  int k_chunks;         // ceil(d / 64)
+  __nv_bfloat16* g_hi;
+  __nv_bfloat16* g_lo;
+  int ld;
+  int* status;
+};
+
+__global__ void __launch_bounds__(192, 1)
+gram_tc_kernel(const __grid_constant__ CUtensorMap map_z,   // gathered rows [sum M_b, d] bf16
+               const GramParams prm) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kGramStages * kGramStageBytes);
+  uint64_t* full = bars;                       // [kGramStages]
+  uint64_t* empty = bars + kGramStages;        // [kGramStages]
+  uint64_t* acc_full = bars + 2 * kGramStages; // [2]
+  uint64_t* acc_empty = acc_full + 2;          // [2]
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_full + 4);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kGramStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+    for (int i = 0; i < 2; ++i) { mbar_init(&acc_full[i], 1); mbar_init(&acc_empty[i], 128); }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 5) tmem_alloc(tmem_slot, kGramTmemCols);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  auto decode = [&](int item, ReqPlan& rp, int& ti, int& tj) {
+    int b = find_request(item, prm.batch, [&](int q) { return prm.plan[q].gram_tile_off; });
+    rp = prm.plan[b];
+    tri_decode(item - rp.gram_tile_off, ti, tj);
+  };
+
+  if (warp == 4) {
+    if (lane == 0) {
+      uint32_t it = 0;
+      bool ok = true;
+      for (int item = blockIdx.x; item < prm.n_items && ok; item += gridDim.x) {
+        ReqPlan rp; int ti, tj;
+        decode(item, rp, ti, tj);
+        for (int kc = 0; kc < prm.k_chunks; ++kc, ++it) {
+          int s = it % kGramStages;
+          if (!(ok = mbar_wait(&empty[s], ((it / kGramStages) & 1u) ^ 1u, abort_flag))) break;
+          mbar_expect_tx(&full[s], kGramStageBytes);
+          uint32_t dst = smem_u32(smem + s * kGramStageBytes);
+          tma_load_2d(dst, &map_z, kc * kBK, rp.presel_off + ti * kTile, &full[s]);
+          tma_load_2d(dst + kGramStageBytes / 2, &map_z, kc * kBK, rp.presel_off + tj * kTile, &full[s]);
+        }
+      }
+    }
+    __syncwarp();
+  } else if (warp == 5) {
+    if (lane == 0) {
+      const uint32_t idesc = umma_idesc(kTile, kTile);
+      uint32_t it = 0, n = 0;
+      bool ok = true;
+      for (int item = blockIdx.x; item < prm.n_items && ok; item += gridDim.x, ++n) {
+        int buf = n & 1;
+        if (!(ok = mbar_wait(&acc_empty[buf], ((n >> 1) & 1u) ^ 1u, abort_flag))) break;
+        tc_fence_after();
+        for (int kc = 0; kc < prm.k_chunks; ++kc, ++it) {
+          int s = it % kGramStages;
+          if (!(ok = mbar_wait(&full[s], (it / kGramStages) & 1u, abort_flag))) break;
+          tc_fence_after();
+          uint32_t a_addr = smem_u32(smem + s * kGramStageBytes);
+          uint64_t adesc = umma_desc(a_addr), bdesc = umma_desc(a_addr + kGramStageBytes / 2);
+#pragma unroll
+          for (int k = 0; k < kBK / 16; ++k)
+            umma_bf16(tmem_base + buf * kTile, adesc + 2 * k, bdesc + 2 * k, idesc, (kc | k) != 0);
+          umma_commit(&empty[s]);
+        }
+        if (!ok) break;
+        umma_commit(&acc_full[buf]);
+      }
+    }
+    __syncwarp();
+  } else {
+    const int r = warp * 32 + lane;
+    const uint32_t t_lane = tmem_base + ((uint32_t)(warp * 32) << 16);
+    uint32_t n = 0;
+    bool ok = true;
+    for (int item = blockIdx.x; item < prm.n_items && ok; item += gridDim.x, ++n) {
+      ReqPlan rp; int ti, tj;
+      decode(item, rp, ti, tj);
+      int buf = n & 1;
+      if (!(ok = mbar_wait(&acc_full[buf], (n >> 1) & 1u, abort_flag))) break;
+      tc_fence_after();
+      const int row = ti * kTile + r;                 // row of G inside the request
+      const bool row_ok = row < rp.m;
+      const size_t ld = (size_t)prm.ld;
+#pragma unroll 1
+      for (int c4 = 0; c4 < 4; ++c4) {
+        float v[32];
+        tmem_ld32(t_lane + buf * kTile + c4 * 32, v);
+        const int col0 = tj * kTile + c4 * 32;
+        // entries outside the request's M x M block are stored as zeros: the power step multiplies
+        // whole 64-wide k-chunks and must not meet stale non-finite values in the padding
+#pragma unroll
+        for (int e = 0; e < 32; ++e)
+          if (col0 + e >= rp.m || !row_ok) v[e] = 0.f;
+        uint32_t ph[16], pl[16];
+#pragma unroll
+        for (int e = 0; e < 16; ++e) {
+          __nv_bfloat162 hi = __floats2bfloat162_rn(v[2 * e], v[2 * e + 1]);
+          ph[e] = *reinterpret_cast<uint32_t*>(&hi);
+          pl[e] = pack_bf16(v[2 * e] - __low2float(hi), v[2 * e + 1] - __high2float(hi));
+        }
+        if (row_ok && col0 < prm.ld) {
+          size_t o = ((size_t)rp.presel_off + row) * ld + col0;
+          uint4* dh = reinterpret_cast<uint4*>(prm.g_hi + o);
+          uint4* dl = reinterpret_cast<uint4*>(prm.g_lo + o);
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            dh[q] = make_uint4(ph[4 * q], ph[4 * q + 1], ph[4 * q + 2], ph[4 * q + 3]);
+            dl[q] = make_uint4(pl[4 * q], pl[4 * q + 1], pl[4 * q + 2], pl[4 * q + 3]);
+          }
+        }
+        if (ti != tj && row < prm.ld) {
+          // mirrored tile: G[col, row] = G[row, col]; consecutive threads write consecutive columns
+          unsigned short* mh = reinterpret_cast<unsigned short*>(prm.g_hi);
+          unsigned short* ml = reinterpret_cast<unsigned short*>(prm.g_lo);
+#pragma unroll
+          for (int e = 0; e < 32; ++e) {
+            int mrow = col0 + e;
+            if (mrow < rp.m) {
+              size_t o = ((size_t)rp.presel_off + mrow) * ld + row;
+              uint32_t wh = ph[e >> 1], wl = pl[e >> 1];
+              mh[o] = (unsigned short)((e & 1) ? (wh >> 16) : (wh & 0xffffu));
+              ml[o] = (unsigned short)((e & 1) ? (wl >> 16) : (wl & 0xffffu));
+            }
+          }
+        }
+      }
+      tc_fence_before();
+      mbar_arrive(&acc_empty[buf]);
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 5) tmem_dealloc(tmem_base, kGramTmemCols);
+  if (threadIdx.x == 0 && *abort_flag) atomicOr(prm.status, kStatusTimeout);
+}
+
+// Splits a float32 Gram matrix (CUDA-core path, float32 inputs) into the two bf16 planes.
+__global__ void __launch_bounds__(256)
+split_planes_kernel(const ReqPlan* __restrict__ plan, const float* __restrict__ G,
+                    __nv_bfloat16* __restrict__ g_hi, __nv_bfloat16* __restrict__ g_lo, int ld) {
+  ReqPlan rp = plan[blockIdx.y];
+  if (!rp.stage2) return;
+  int cols = (rp.m + 63) & ~63;
+  int total = rp.m * cols;
+  for (int e = blockIdx.x * blockDim.x + threadIdx.x; e < total; e += gridDim.x * blockDim.x) {
+    int i = e / cols, j = e % cols;
+    float v = j < rp.m ? G[rp.g_off + (size_t)i * rp.ldm + j] : 0.f;
+    __nv_bfloat16 hi, lo;
+    split_bf16(v, hi, lo);
+    size_t o = ((size_t)rp.presel_off + i) * ld + j;
+    g_hi[o] = hi; g_lo[o] = lo;
+  }
+}
+
+// Start block of the subspace iteration: entries uniform in [-1, 1) from a counter hash of
+// (request, basis vector, position); zero in the padding columns and in the unused basis rows
+// p .. round_up(p, 16) - 1 of both plane buffers (the MMA reads them, nothing else writes them).
+__global__ void __launch_bounds__(256)
+basis_init_kernel(const ReqPlan* __restrict__ plan, __nv_bfloat16* __restrict__ y_hi,
+                  __nv_bfloat16* __restrict__ y_lo, __nv_bfloat16* __restrict__ y2_hi,
+                  __nv_bfloat16* __restrict__ y2_lo, int ld) {
+  ReqPlan rp = plan[blockIdx.y];
+  if (!rp.stage2) return;
+  int cols = (rp.m + 63) & ~63;
+  int rows = (rp.p + 15) & ~15;
+  int total = rows * cols;
+  for (int e = blockIdx.x * blockDim.x + threadIdx.x; e < total; e += gridDim.x * blockDim.x) {
+    int j = e / cols, i = e % cols;
+    float v = 0.f;
+    if (j < rp.p && i < rp.m) {
+      unsigned h = (unsigned)(j * rp.m + i) * 0x9E3779B1u ^ ((unsigned)blockIdx.y + 1u) * 0x85EBCA77u;
+      h ^= h >> 16; h *= 0x7FEB352Du; h ^= h >> 15; h *= 0x846CA68Bu; h ^= h >> 16;
+      v = (float)(h >> 8) * (2.0f / 16777216.0f) - 1.0f;
+    }
+    __nv_bfloat16 hi, lo;
+    split_bf16(v, hi, lo);
+    size_t o = ((size_t)blockIdx.y * kPMax + j) * ld + i;
+    y_hi[o] = hi; y_lo[o] = lo;
+    if (j >= rp.p) { y2_hi[o] = hi; y2_lo[o] = lo; }
+  }
+}
+
+// ================================================================================================
+// Power step
+// ================================================================================================
+constexpr int kPowStages = 2;
+constexpr int kPowBytesA = kTile * kBK * 2;              // one plane of the G tile, 16 KB
+constexpr int kPowBytesB = kPMax * kBK * 2;              // one plane of the Y tile, 20 KB
+constexpr int kPowStageBytes = 2 * kPowBytesA + 2 * kPowBytesB;   // 72 KB
+constexpr int kXsLd = kTile + 1;                         // row stride of the staged block (floats)
+constexpr int kPowSmem = kPowStages * kPowStageBytes + kLbufStride * 4 + 1024 + 1024;
+constexpr int kPowTmemCols = 256;
+static_assert(kPMax * kXsLd * 4 <= kPowStages * kPowStageBytes, "staged block must fit in the ring");
+
+struct PowerParams {
+  const ReqPlan* plan;
+  int batch;
+  int n_items;              // 128-row tiles over all stage-2 requests
+  int identity;             // first step: no triangular factor yet
+  int last;                 // last step: also write the float32 block
+  const float* lbuf;        // [batch][kLbufStride] triangular factor + reciprocal diagonal
+  __nv_bfloat16* y_hi;      // output planes
+  __nv_bfloat16* y_lo;
+  int ld;
+  float* yf;                // [sum M_b, kPMax] (last step)
+  double* partial;          // [tiles][kTriMax]
+  int* status;
+};
+
+__global__ void __launch_bounds__(192, 1)
+power_tc_kernel(const __grid_constant__ CUtensorMap map_gh, const __grid_constant__ CUtensorMap map_gl,
+                const __grid_constant__ CUtensorMap map_yh, const __grid_constant__ CUtensorMap map_yl,
+                const PowerParams prm) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  float* xs = reinterpret_cast<float*>(smem);                       // aliases the ring after the MMAs
+  float* lt = reinterpret_cast<float*>(smem + kPowStages * kPowStageBytes);
+  float* dinv = lt + kLtFloats;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(lt + kLbufStride);
+  uint64_t* full = bars;                 // [2]
+  uint64_t* empty = bars + 2;            // [2]
+  uint64_t* acc_full = bars + 4;
+  uint64_t* acc_empty = bars + 5;
+  uint64_t* epi_done = bars + 6;         // the staged block no longer occupies the ring
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 8);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kPowStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+    mbar_init(acc_full, 1);
+    mbar_init(acc_empty, 128);
+    mbar_init(epi_done, 128);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 5) tmem_alloc(tmem_slot, kPowTmemCols);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  auto decode = [&](int item, int& b, ReqPlan& rp, int& tile) {
+    b = find_request(item, prm.batch, [&](int q) { return prm.plan[q].ptile_off; });
+    rp = prm.plan[b];
+    tile = item - rp.ptile_off;
+  };
+
+  if (warp == 4) {
+    if (lane == 0) {
+      uint32_t it = 0, n = 0;
+      bool ok = true;
+      for (int item = blockIdx.x; item < prm.n_items && ok; item += gridDim.x, ++n) {
+        int b, tile; ReqPlan rp;
+        decode(item, b, rp, tile);
+        // the previous item's staged block lives in the ring until its epilogue is done
+        if (n > 0 && !(ok = mbar_wait(epi_done, (n - 1) & 1u, abort_flag))) break;
+        int k_chunks = (rp.m + kBK - 1) / kBK;
+        for (int kc = 0; kc < k_chunks; ++kc, ++it) {
+          int s = it % kPowStages;
+          if (!(ok = mbar_wait(&empty[s], ((it / kPowStages) & 1u) ^ 1u, abort_flag))) break;
+          mbar_expect_tx(&full[s], kPowStageBytes);
+          uint32_t dst = smem_u32(smem + s * kPowStageBytes);
+          int grow = rp.presel_off + tile * kTile;
+          tma_load_2d(dst, &map_gh, kc * kBK, grow, &full[s]);
+          tma_load_2d(dst + kPowBytesA, &map_gl, kc * kBK, grow, &full[s]);
+          tma_load_2d(dst + 2 * kPowBytesA, &map_yh, kc * kBK, b * kPMax, &full[s]);
+          tma_load_2d(dst + 2 * kPowBytesA + kPowBytesB, &map_yl, kc * kBK, b * kPMax, &full[s]);
+        }
+      }
+    }
+    __syncwarp();
+  } else if (warp == 5) {
+    if (lane == 0) {
+      uint32_t it = 0, n = 0;
+      bool ok = true;
+      for (int item = blockIdx.x; item < prm.n_items && ok; item += gridDim.x, ++n) {
+        int b, tile; ReqPlan rp;
+        decode(item, b, rp, tile);
+        const uint32_t idesc = umma_idesc(kTile, (rp.p + 15) & ~15);
+        if (!(ok = mbar_wait(acc_empty, (n & 1u) ^ 1u, abort_flag))) break;
+        tc_fence_after();
+        int k_chunks = (rp.m + kBK - 1) / kBK;
+        for (int kc = 0; kc < k_chunks; ++kc, ++it) {
+          int s = it % kPowStages;
+          if (!(ok = mbar_wait(&full[s], (it / kPowStages) & 1u, abort_flag))) break;
+          tc_fence_after();
+          uint32_t base = smem_u32(smem + s * kPowStageBytes);
+          // T += G_hi Y_hi + G_lo Y_hi + G_hi Y_lo
+#pragma unroll
+          for (int term = 0; term < 3; ++term) {
+            uint64_t adesc = umma_desc(base + (term == 1 ? kPowBytesA : 0));
+            uint64_t bdesc = umma_desc(base + 2 * kPowBytesA + (term == 2 ? kPowBytesB : 0));
+#pragma unroll
+            for (int k = 0; k < kBK / 16; ++k)
+              umma_bf16(tmem_base, adesc + 2 * k, bdesc + 2 * k, idesc, (kc | term | k) != 0);
+          }
+          umma_commit(&empty[s]);
+        }
+        if (!ok) break;
+        umma_commit(acc_full);
+      }
+    }
+    __syncwarp();
+  } else {
+    const int r = warp * 32 + lane;
+    const uint32_t t_lane = tmem_base + ((uint32_t)(warp * 32) << 16);
+    uint32_t n = 0;
+    int cached_b = -1;
+    bool ok = true;
+    for (int item = blockIdx.x; item < prm.n_items && ok; item += gridDim.x, ++n) {
+      int b, tile; ReqPlan rp;
+      decode(item, b, rp, tile);
+      const int p = rp.p, P = (p + 7) & ~7;
+      if (!prm.identity && b != cached_b) {
+        named_barrier(1, 128);                     // nobody still reads the previous factor
+        const float4* src = reinterpret_cast<const float4*>(prm.lbuf + (size_t)b * kLbufStride);
+        float4* dst = reinterpret_cast<float4*>(lt);
+        int n4 = (lt_row_offset(P, P) + 3) / 4;    // floats used by the P-wide layout
+        for (int e = r; e < n4; e += 128) dst[e] = src[e];
+        const float* dsrc = prm.lbuf + (size_t)b * kLbufStride + kLtFloats;
+        for (int e = r; e < P; e += 128) dinv[e] = dsrc[e];
+        named_barrier(1, 128);
+        cached_b = b;
+      }
+      if (!(ok = mbar_wait(acc_full, n & 1u, abort_flag))) break;
+      tc_fence_after();
+      const int row = tile * kTile + r;
+      const bool row_ok = row < rp.m;
+      // ---- Y_next row = T row * L^-T by blocked forward substitution; staged as xs[c][r] ----
+#pragma unroll 1
+      for (int cb = 0; cb * 32 < P; ++cb) {
+        float v[32];
+        tmem_ld32(t_lane + cb * 32, v);
+#pragma unroll
+        for (int sb = 0; sb < 4; ++sb) {
+          const int jb = cb * 32 + sb * 8;
+          if (jb < P) {
+            float acc[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) acc[e] = v[sb * 8 + e];
+            if (!prm.identity) {
+              int off = jb;                         // lt_row_offset(i, P) + jb - 4 * (i >> 2), i = 0
+#pragma unroll 2
+              for (int i = 0; i < jb; ++i) {
+                float xi = xs[i * kXsLd + r];
+                float4 l0 = *reinterpret_cast<const float4*>(lt + off);
+                float4 l1 = *reinterpret_cast<const float4*>(lt + off + 4);
+                acc[0] -= xi * l0.x; acc[1] -= xi * l0.y; acc[2] -= xi * l0.z; acc[3] -= xi * l0.w;
+                acc[4] -= xi * l1.x; acc[5] -= xi * l1.y; acc[6] -= xi * l1.z; acc[7] -= xi * l1.w;
+                off += P - 4 * (i >> 2) - (((i & 3) == 3) ? 4 : 0);
+              }
+              // triangular solve inside the 8-column block (rows jb .. jb+7 of the layout)
+              const float* lrow = lt + lt_row_offset(jb, P);          // row jb starts at column jb
+#pragma unroll
+              for (int jj = 0; jj < 8; ++jj) {
+                float x = acc[jj] * dinv[jb + jj];
+                acc[jj] = x;
+                // row jb+jj holds columns from jb + (jj & ~3)
+                const float* lr = lt + lt_row_offset(jb + jj, P) - (jj & ~3);
+#pragma unroll
+                for (int j2 = jj + 1; j2 < 8; ++j2) acc[j2] -= x * lr[j2];
+              }
+              (void)lrow;
+            }
+#pragma unroll
+            for (int e = 0; e < 8; ++e) xs[(jb + e) * kXsLd + r] = row_ok ? acc[e] : 0.f;
+          }
+        }
+      }
+      tc_fence_before();
+      mbar_arrive(acc_empty);
+      named_barrier(1, 128);                       // the staged block is complete
+      // ---- bf16 planes of the new block (K-major operand of the next step) ----
+      const int cols = (rp.m + kBK - 1) / kBK * kBK;
+      if (row < cols) {
+        size_t o = ((size_t)b * kPMax) * prm.ld + row;
+        for (int c = 0; c < p; ++c) {
+          __nv_bfloat16 hi, lo;
+          split_bf16(xs[c * kXsLd + r], hi, lo);
+          prm.y_hi[o + (size_t)c * prm.ld] = hi;
+          prm.y_lo[o + (size_t)c * prm.ld] = lo;
+        }
+      }
+      if (prm.last) {
+        // float32 block, one token per row: thread e of the tile walks (row, column) pairs so that
+        // consecutive threads write consecutive columns
+        int nrows = min(kTile, rp.m - tile * kTile);
+        for (int e = r; e < nrows * p; e += 128) {
+          int rr = e / p, c = e % p;
+          prm.yf[((size_t)rp.presel_off + tile * kTile + rr) * kPMax + c] = xs[c * kXsLd + rr];
+        }
+      }
+      // ---- float64 partial Gram of the tile: B[a][b] = sum_r x[a][r] x[b][r], b <= a ----
+      {
+        int nrows = min(kTile, rp.m - tile * kTile);
+        int nb = (p + 3) >> 2, nblk = nb * (nb + 1) / 2;
+        double* out = prm.partial + (size_t)item * kTriMax;
+        for (int blk = r; blk < nblk; blk += 128) {
+          int ba, bb;
+          tri_decode(blk, ba, bb);
+          double acc[4][4];
+#pragma unroll
+          for (int i = 0; i < 4; ++i)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) acc[i][j] = 0.0;
+          const float* xa = xs + (4 * ba) * kXsLd;
+          const float* xb = xs + (4 * bb) * kXsLd;
+          for (int rr = 0; rr < nrows; ++rr) {
+            double a[4], c[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) { a[i] = (double)xa[i * kXsLd + rr]; c[i] = (double)xb[i * kXsLd + rr]; }
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+              for (int j = 0; j < 4; ++j) acc[i][j] += a[i] * c[j];
+          }
+#pragma unroll
+          for (int i = 0; i < 4; ++i)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              int ia = 4 * ba + i, ib = 4 * bb + j;
+              if (ia < p && ib <= ia) out[tri_index(ia, ib)] = acc[i][j];
+            }
+        }
+      }
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      mbar_arrive(epi_done);
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 5) tmem_dealloc(tmem_base, kPowTmemCols);
+  if (threadIdx.x == 0 && *abort_flag) atomicOr(prm.status, kStatusTimeout);
+}
+
+}  // namespace sub
+}  // namespace covspec
