@@ -24,7 +24,7 @@ struct ReqPlan {
   int tile_off;            // first 128-token tile of the request in the tensor-core relevance kernel
   int gram_tile_off;       // first lower-triangle 128 x 128 tile of the request's Gram matrix
   int ptile_off;           // first 128-row tile of the request's subspace-iteration block
-  int pad_;
+  int win;                 // basis vectors in the Rayleigh-Ritz window next to the cut at r
   long long g_off;         // float offset of the request's float32 Gram matrix (float32 inputs only)
 };
 

@@ -57,7 +57,7 @@ struct Plan {
   std::vector<int> keep_offsets, presel_offsets;
   int n_stage2 = 0;
   int tiles[T_COUNT] = {0};
-  int t_max = 0, p_max = 0, m_max = 0, r_max = 0;
+  int t_max = 0, p_max = 0, m_max = 0, win_max = 0, nbot_max = 0;
   int n_tiles = 0;                            // 128-token tiles over all requests
   int n_gram_tiles = 0, n_ptiles = 0;         // lower-triangle Gram tiles / 128-row block tiles (stage 2)
   long long total_vis = 0, total_txt = 0, total_keep = 0, total_presel = 0;
@@ -90,9 +90,9 @@ struct covspec_ctx {
   long long cap_rows = 0, cap_ptiles = 0;
   __nv_bfloat16 *Ghi = nullptr, *Glo = nullptr;
   __nv_bfloat16* Yp[2][2] = {{nullptr, nullptr}, {nullptr, nullptr}};   // [buffer][hi / lo]
-  float* Yf = nullptr;
+  float* Yf[2] = {nullptr, nullptr};     // float32 blocks before / after the last power step
   double* partial = nullptr;
-  float *Lbuf = nullptr, *Ut = nullptr, *theta = nullptr;
+  float *Lbuf = nullptr, *Ub = nullptr;
   CUtensorMap map_zg, map_gh, map_gl, map_y[2][2];
   // pinned staging for the plan upload
   char* h_stage = nullptr;
@@ -186,7 +186,7 @@ int get_plan(covspec_ctx* ctx, const covspec_problem* p, cudaStream_t stream) {
   pl.presel_offsets.assign(B + 1, 0);
   pl.n_stage2 = 0; pl.t_max = 0; pl.p_max = 0; pl.m_max = 0; pl.n_tiles = 0;
   pl.n_gram_tiles = 0; pl.n_ptiles = 0;
-  pl.r_max = 0;
+  pl.win_max = 0; pl.nbot_max = 0;
   long long g_off = 0;
   int n_max = 0;
   bool f32 = cfg.dtype == COVSPEC_F32;
@@ -212,7 +212,10 @@ int get_plan(covspec_ctx* ctx, const covspec_problem* p, cudaStream_t stream) {
       pl.n_gram_tiles += nt * (nt + 1) / 2;
       pl.n_ptiles += nt;
       if (f32) g_off += (long long)r.m * r.ldm;
-      if (r.r > pl.r_max) pl.r_max = r.r;
+      r.win = r.p - r.r + std::min(32, r.r);
+      if (r.win > r.p) r.win = r.p;
+      pl.win_max = std::max(pl.win_max, r.win);
+      pl.nbot_max = std::max(pl.nbot_max, r.p - r.r);
     }
     r.keep_off = pl.keep_offsets[b]; r.presel_off = pl.presel_offsets[b];
     pl.keep_offsets[b + 1] = r.keep_off + r.b_vis;
@@ -503,31 +506,34 @@ int select_impl(covspec_ctx* ctx, const covspec_problem* p, const float* s_fused
     sub::basis_init_kernel<<<gb, 256, 0, s>>>(ctx->d_plan, ctx->Yp[0][0], ctx->Yp[0][1], ctx->Yp[1][0],
                                               ctx->Yp[1][1], ctx->ld);
     LAUNCH_CHECK(ctx);
-    size_t tri_smem = ((size_t)pl.p_max * (pl.p_max + 1) / 2 + 2 * pl.p_max) * sizeof(double);
-    size_t ritz_smem = tri_smem + ((size_t)pl.p_max * (pl.p_max | 1) + pl.p_max) * sizeof(float);
     int grid = std::min(pl.n_ptiles, ctx->num_sms);
     for (int pass = 0; pass <= cfg.eig_iters; ++pass) {
       sub::PowerParams pp{};
       pp.plan = ctx->d_plan; pp.batch = B; pp.n_items = pl.n_ptiles;
-      pp.identity = pass == 0; pp.last = pass == cfg.eig_iters;
+      pp.identity = pass == 0;
       pp.lbuf = ctx->Lbuf;
       int in = pass & 1, out = in ^ 1;
       pp.y_hi = ctx->Yp[out][0]; pp.y_lo = ctx->Yp[out][1]; pp.ld = ctx->ld;
-      pp.yf = ctx->Yf; pp.partial = ctx->partial; pp.status = ctx->status;
-      sub::power_tc_kernel<<<grid, 192, sub::kPowSmem, s>>>(ctx->map_gh, ctx->map_gl, ctx->map_y[in][0],
-                                                            ctx->map_y[in][1], pp);
+      // the two last blocks are also kept in float32 for the energy kernel
+      pp.yf = pass == cfg.eig_iters ? ctx->Yf[1] : pass == cfg.eig_iters - 1 ? ctx->Yf[0] : nullptr;
+      pp.partial = ctx->partial; pp.status = ctx->status;
+      sub::power_tc_kernel<<<grid, sub::kPowThreads, sub::kPowSmem, s>>>(
+          ctx->map_gh, ctx->map_gl, ctx->map_y[in][0], ctx->map_y[in][1], pp);
       LAUNCH_CHECK(ctx);
       if (pass < cfg.eig_iters) {
-        chol_kernel<<<B, 512, tri_smem, s>>>(ctx->d_plan, ctx->partial, ctx->Lbuf);
+        chol_kernel<<<B, 512, cholesky_smem_bytes(pl.p_max), s>>>(ctx->d_plan, ctx->partial, ctx->Lbuf);
         LAUNCH_CHECK(ctx);
       }
     }
-    ritz_kernel<<<B, 1024, ritz_smem, s>>>(ctx->d_plan, ctx->partial, ctx->Ut, ctx->theta, 30, ctx->status);
+    size_t ritz_smem = (((size_t)pl.win_max * (pl.win_max | 1) + pl.win_max + 1) & ~(size_t)1) * sizeof(float) +
+                       cholesky_smem_bytes(pl.win_max);
+    ritz_kernel<<<B, 512, ritz_smem, s>>>(ctx->d_plan, ctx->partial, ctx->Ub, 30, ctx->status);
     LAUNCH_CHECK(ctx);
   }
-  dim3 ge((pl.m_max + 63) / 64, B);
-  size_t en_smem = (size_t)pl.p_max * pl.r_max * sizeof(float);
-  energy_kernel<<<ge, 256, en_smem, s>>>(ctx->d_plan, ctx->Yf, ctx->Ut, energy);
+  dim3 ge((pl.m_max + sub::kTile - 1) / sub::kTile, B);
+  int p8 = (pl.p_max + 7) & ~7;
+  size_t en_smem = ((size_t)sub::kLbufStride + (size_t)p8 * sub::kXsLd + (size_t)pl.win_max * pl.nbot_max) * sizeof(float);
+  energy_kernel<<<ge, 256, en_smem, s>>>(ctx->d_plan, ctx->Yf[0], ctx->Yf[1], ctx->Lbuf, ctx->Ub, p8, energy);
   LAUNCH_CHECK(ctx);
   if (pl.n_stage2 > 0) prof_mark(ctx, ST_EIG, 1, s);
   prof_mark(ctx, ST_FINAL, 0, s);
@@ -579,7 +585,7 @@ void covspec_default_config(covspec_config* c) {
   c->presel_factor = 2.0f;
   c->rank_frac = 0.5f;
   c->rank_cap = 128;
-  c->eig_iters = 6;
+  c->eig_iters = 5;
   c->eig_oversample = 32;
   c->relevance_path = 0;
 }
@@ -652,10 +658,10 @@ int covspec_prune_init(const covspec_config* cfg, covspec_ctx** out) {
   long long yplane = 2ll * c.max_batch * kPMax * ctx->ld;
   long long o_y[2][2];
   for (int i = 0; i < 2; ++i) for (int j = 0; j < 2; ++j) o_y[i][j] = carve(yplane);
-  long long o_yf = carve(4ll * ctx->cap_rows * kPMax);
+  long long o_yf0 = carve(4ll * ctx->cap_rows * kPMax), o_yf1 = carve(4ll * ctx->cap_rows * kPMax);
   long long o_part = carve(8ll * ctx->cap_ptiles * sub::kTriMax);
   long long o_lbuf = carve(4ll * c.max_batch * sub::kLbufStride);
-  long long o_ut = carve(4ll * c.max_batch * kPMax * kPMax), o_theta = carve(4ll * c.max_batch * kPMax);
+  long long o_ub = carve(4ll * c.max_batch * kPMax * kPMax);
   ctx->ws_bytes = off;
   cudaError_t e = cudaMalloc(&ctx->ws, (size_t)off);
   if (e != cudaSuccess) {
@@ -680,23 +686,24 @@ int covspec_prune_init(const covspec_config* cfg, covspec_ctx** out) {
   ctx->Glo = reinterpret_cast<__nv_bfloat16*>(w + o_gl);
   for (int i = 0; i < 2; ++i)
     for (int j = 0; j < 2; ++j) ctx->Yp[i][j] = reinterpret_cast<__nv_bfloat16*>(w + o_y[i][j]);
-  ctx->Yf = reinterpret_cast<float*>(w + o_yf);
+  ctx->Yf[0] = reinterpret_cast<float*>(w + o_yf0);
+  ctx->Yf[1] = reinterpret_cast<float*>(w + o_yf1);
   ctx->partial = reinterpret_cast<double*>(w + o_part);
   ctx->Lbuf = reinterpret_cast<float*>(w + o_lbuf);
-  ctx->Ut = reinterpret_cast<float*>(w + o_ut);
-  ctx->theta = reinterpret_cast<float*>(w + o_theta);
+  ctx->Ub = reinterpret_cast<float*>(w + o_ub);
   ctx->stage_bytes = round_up(sizeof(ReqPlan) * c.max_batch, 256) +
                      sizeof(GemmProb) * (long long)T_COUNT * c.max_batch;
   bool ok = cudaMemset(ctx->status, 0, 256) == cudaSuccess &&
             cudaMallocHost(&ctx->h_stage, (size_t)ctx->stage_bytes) == cudaSuccess &&
             cudaEventCreateWithFlags(&ctx->stage_free, cudaEventDisableTiming) == cudaSuccess;
   // the small dense kernels need more than the default 48 KB of dynamic shared memory
-  const int tri_bytes = (int)(((size_t)kPMax * (kPMax + 1) / 2 + 2 * kPMax) * sizeof(double));
-  ok = ok && cudaFuncSetAttribute(chol_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, tri_bytes) == cudaSuccess;
+  ok = ok && cudaFuncSetAttribute(chol_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                  (int)cholesky_smem_bytes(kPMax)) == cudaSuccess;
   ok = ok && cudaFuncSetAttribute(ritz_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                  tri_bytes + (int)(((size_t)kPMax * (kPMax | 1) + kPMax) * sizeof(float))) == cudaSuccess;
+                                  (int)(((size_t)kPMax * (kPMax | 1) + kPMax + 2) * sizeof(float) +
+                                        cholesky_smem_bytes(kPMax))) == cudaSuccess;
   ok = ok && cudaFuncSetAttribute(energy_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                  (int)((size_t)kPMax * kPMax * sizeof(float))) == cudaSuccess;
+                                  220 * 1024) == cudaSuccess;
   int dev = 0, cc_major = 0;
   ok = ok && cudaGetDevice(&dev) == cudaSuccess &&
        cudaDeviceGetAttribute(&ctx->num_sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess &&

@@ -6,12 +6,19 @@
 // vectors (power_tc_kernel).  Every step leaves the float64 Gram matrix B = Y^T Y of the new block
 // as per-tile partial sums; this file holds
 //   chol_kernel    B = L L^T (float64, one block per request), stored in the layout the next power
-//                  step reads, so that Y L^-T is an orthonormal basis;
-//   ritz_kernel    after the last step: the singular value decomposition of L by one-sided Jacobi
-//                  rotations, L W = U diag(s).  With Y = G Q (Q the previous orthonormal basis),
-//                  B = Q G^2 Q^T, so U holds the Ritz vectors of G^2 in the basis Q, s_k ~ lambda_k,
-//                  and Y u_k / s_k is the Ritz vector after one more power step;
-//   energy_kernel  c_i = sum_{k<r} (Y[i,:] a_k)^2 / s_k^3 with a_k = s_k u_k the rotated columns.
+//                  step reads, so that Q = Y L^-T is an orthonormal basis.
+//   ritz_kernel    after the last step Y' = G Q^T: Rayleigh-Ritz for G^2 on the span of the last
+//                  `win` basis vectors, whose Ritz matrix is the trailing win x win block of
+//                  B' = Y'^T Y' = Q G^2 Q^T.  Its Cholesky factor is diagonalised by one-sided Jacobi
+//                  rotations; the eigenvectors u_k of the p - r smallest Ritz values are kept.
+//   energy_kernel  for an orthonormal basis of a G-invariant subspace, sum_k lambda_k V_ik^2 =
+//                  sum_j Y'_ij Q_ij; the energy in the top-r subspace is that total over all p basis
+//                  vectors minus the part of the p - r smallest Ritz pairs,
+//                  c_i = sum_j Y'_ij Q_ij - sum_k (Y'_i,win u_k)(Q_i,win u_k).
+// Only the Ritz pairs next to the cut at r have to be resolved individually: basis vectors more
+// than 32 places above the cut are separated from the discarded ones by the same eigenvalue ratios
+// that drive the subspace iteration itself, so the window has p - r + min(32, r) vectors (all p when
+// the problem is small).
 #pragma once
 #include "subspace_tc.cuh"
 
@@ -20,110 +27,169 @@ namespace covspec {
 using sub::kLbufStride;
 using sub::kLtFloats;
 using sub::kTriMax;
+using sub::kXsLd;
 using sub::lt_row_offset;
 using sub::tri_index;
 
-// Sums the per-tile partial Gram matrices of a request in tile order (deterministic) into the
-// packed lower triangle A, then factors it in place: on return A[tri(i,k)] (i > k) holds the
-// unscaled column entries and piv[k] the (clamped) pivots of the square-root-free elimination, so
-// that L[i][k] = A[tri(i,k)] / sqrt(piv[k]) and L[k][k] = sqrt(piv[k]).  A pivot that falls below
-// 1e-12 of its original diagonal entry (a numerically dependent direction) is clamped there; the
-// next multiplication by G restores the direction.  One __syncthreads per column.
-__device__ __forceinline__ void gram_cholesky(const ReqPlan& rp, const double* __restrict__ partial,
-                                              double* A, double* piv, double* d0) {
-  const int p = rp.p, tri = p * (p + 1) / 2, tid = threadIdx.x, nt = blockDim.x;
-  const int lane = tid & 31, w = tid >> 5, nw = nt >> 5;
-  const int ntile = (rp.m + sub::kTile - 1) / sub::kTile;
-  for (int e = tid; e < tri; e += nt) {
-    double s = 0.0;
-    for (int t = 0; t < ntile; ++t) s += partial[(size_t)(rp.ptile_off + t) * kTriMax + e];
-    A[e] = s;
+// 1 / sqrt(x) in float64: float32 estimate (~22 bits) refined by two Newton steps written as short
+// dependency chains (the factorisation's critical path runs through this once per column); the
+// library routine outside the float32 range.
+__device__ __forceinline__ double rsqrt_f64(double x) {
+  if (!(x > 1e-37 && x < 1e37)) return 1.0 / sqrt(x);
+  double y = (double)rsqrtf((float)x);
+  double hx = 0.5 * x;
+  double e = fma(-hx * y, y, 0.5);        // (1 - x y^2) / 2
+  y = fma(y, e, y);
+  e = fma(-hx * y, y, 0.5);
+  y = fma(y, e, y);
+  return y;
+}
+
+// Blocked right-looking Cholesky factorisation of an n x n float64 matrix kept in shared memory as
+// 8 x 8 tiles of its lower triangle (tile (I, J <= I) at T + tri_index(I, J) * 64, row-major).
+// Per 8-column panel: the diagonal tile is factored by one warp, the tiles below it are solved one
+// row per thread, and the trailing tiles take their rank-8 update on the FP64 tensor cores
+// (two m8n8k4 instructions per tile).  Three __syncthreads per panel.
+// A pivot below 1e-12 of its original diagonal entry (a numerically dependent direction) is
+// clamped there; the next multiplication by G restores the direction.
+//   load(i, j)         value of entry (i, j), i >= j
+//   store(i, j, v, rd) receives L[i][j] and 1 / L[j][j]
+//   T: 64 * nb (nb + 1) / 2 doubles, nb = ceil(n / 8);  aux: 2 * 8 * nb doubles
+template <typename Load, typename Store>
+__device__ __forceinline__ void cholesky_blocked(int n, double* T, double* aux, Load load, Store store) {
+  const int tid = threadIdx.x, nt = blockDim.x, lane = tid & 31, warp = tid >> 5, nw = nt >> 5;
+  const int nb = (n + 7) >> 3, ntile = nb * (nb + 1) / 2;
+  double* d0 = aux;                 // original diagonal
+  double* rd = aux + 8 * nb;        // 1 / L[j][j]
+  for (int e = tid; e < ntile * 64; e += nt) {
+    int I, J;
+    sub::tri_decode(e >> 6, I, J);
+    int i = 8 * I + ((e >> 3) & 7), j = 8 * J + (e & 7);
+    double v;
+    if (i < n && j < n) v = j <= i ? load(i, j) : load(j, i);
+    else v = i == j ? 1.0 : 0.0;
+    T[e] = v;
+    if (i == j) d0[i] = v;
   }
   __syncthreads();
-  for (int i = tid; i < p; i += nt) d0[i] = A[tri_index(i, i)];
-  __syncthreads();
-  for (int k = 0; k < p; ++k) {
-    double pv = A[tri_index(k, k)], floor_ = 1e-12 * d0[k];
-    if (!(pv > floor_)) pv = floor_ > 0.0 ? floor_ : 1.0;
-    if (tid == 0) piv[k] = pv;
-    double inv = 1.0 / pv;
-    for (int i = k + 1 + w; i < p; i += nw) {
-      double lik = A[tri_index(i, k)] * inv;
-      double* row = A + tri_index(i, 0);
-      for (int j = k + 1 + lane; j <= i; j += 32) row[j] -= lik * A[tri_index(j, k)];
+  for (int J = 0; J < nb; ++J) {
+    double* D = T + tri_index(J, J) * 64;
+    if (warp == 0) {
+      // lanes 0..27 own the strictly-lower pairs (l, m < l) of the trailing updates
+      int l = 1, m = 0;
+      { int q = lane; while (q >= l) { q -= l; ++l; } m = q; }   // pair index -> (l, m), l in 1..7
+      for (int c = 0; c < 8; ++c) {
+        double piv = D[c * 8 + c], floor_ = 1e-12 * d0[8 * J + c];
+        if (!(piv > floor_)) piv = floor_ > 0.0 ? floor_ : 1.0;
+        double rs = rsqrt_f64(piv);
+        __syncwarp();
+        if (lane == 0) { D[c * 8 + c] = piv * rs; rd[8 * J + c] = rs; }
+        if (lane > c && lane < 8) D[lane * 8 + c] *= rs;
+        __syncwarp();
+        // D[l][m] -= L[l][c] L[m][c] for c < m <= l, including the diagonal (lanes 28..31 + spare)
+        if (lane < 28 && m > c) D[l * 8 + m] -= D[l * 8 + c] * D[m * 8 + c];
+        if (lane >= 24 && lane - 24 > c) { int dgl = lane - 24; D[dgl * 8 + dgl] -= D[dgl * 8 + c] * D[dgl * 8 + c]; }
+        __syncwarp();
+      }
+    }
+    __syncthreads();
+    // tiles below the diagonal tile: row i of tile (I, J) <- row * L_JJ^-T
+    for (int i = 8 * (J + 1) + tid; i < 8 * nb; i += nt) {
+      double* row = T + tri_index(i >> 3, J) * 64 + (i & 7) * 8;
+      double x[8];
+#pragma unroll
+      for (int c = 0; c < 8; ++c) x[c] = row[c];
+#pragma unroll
+      for (int c = 0; c < 8; ++c) {
+        double v = x[c];
+#pragma unroll
+        for (int k = 0; k < c; ++k) v -= x[k] * D[c * 8 + k];
+        x[c] = v * rd[8 * J + c];
+      }
+#pragma unroll
+      for (int c = 0; c < 8; ++c) row[c] = x[c];
+    }
+    __syncthreads();
+    // trailing tiles (I, K), J < K <= I: C -= X_I X_K^T
+    const int mrem = nb - J - 1, ntr = mrem * (mrem + 1) / 2;
+    const int fr = lane >> 2, fk = lane & 3;
+    for (int q = warp; q < ntr; q += nw) {
+      int ii, kk;
+      sub::tri_decode(q, ii, kk);
+      const double* XI = T + tri_index(J + 1 + ii, J) * 64 + fr * 8 + fk;
+      const double* XK = T + tri_index(J + 1 + kk, J) * 64 + fr * 8 + fk;
+      double* C = T + tri_index(J + 1 + ii, J + 1 + kk) * 64 + fr * 8 + 2 * fk;
+      double c0 = C[0], c1 = C[1];
+      sub::dmma_8x8x4(c0, c1, -XI[0], XK[0]);
+      sub::dmma_8x8x4(c0, c1, -XI[4], XK[4]);
+      C[0] = c0; C[1] = c1;
     }
     __syncthreads();
   }
+  for (int e = tid; e < ntile * 64; e += nt) {
+    int I, J;
+    sub::tri_decode(e >> 6, I, J);
+    int i = 8 * I + ((e >> 3) & 7), j = 8 * J + (e & 7);
+    if (i < n && j <= i) store(i, j, T[e], rd[j]);
+  }
 }
 
-// Dynamic shared memory: (p(p+1)/2 + 2p) doubles.
+// Sum of the per-tile partial Gram matrices of a request, in tile order (deterministic).
+__device__ __forceinline__ double gram_entry(const ReqPlan& rp, const double* __restrict__ partial,
+                                             int i, int j) {
+  const int ntile = (rp.m + sub::kTile - 1) / sub::kTile;
+  const double* src = partial + (size_t)rp.ptile_off * kTriMax + tri_index(i, j);
+  double s = 0.0;
+  for (int t = 0; t < ntile; ++t) s += src[(size_t)t * kTriMax];
+  return s;
+}
+
+// Bytes of shared memory cholesky_blocked needs for an n x n matrix.
+__host__ __device__ inline size_t cholesky_smem_bytes(int n) {
+  int nb = (n + 7) / 8;
+  return ((size_t)nb * (nb + 1) / 2 * 64 + 16 * nb) * sizeof(double);
+}
+
+// One block of 512 threads per request.  Dynamic shared memory: cholesky_smem_bytes(p_max).
 __global__ void __launch_bounds__(512)
 chol_kernel(const ReqPlan* __restrict__ plan, const double* __restrict__ partial,
             float* __restrict__ lbuf) {
   extern __shared__ double sm_d[];
   ReqPlan rp = plan[blockIdx.x];
   if (!rp.stage2) return;
-  const int p = rp.p, P = (p + 7) & ~7, tri = p * (p + 1) / 2;
-  double* A = sm_d;
-  double* piv = A + tri;
-  double* d0 = piv + p;
-  gram_cholesky(rp, partial, A, piv, d0);
-  // rsqrt of the pivots once
-  for (int k = threadIdx.x; k < p; k += blockDim.x) d0[k] = 1.0 / sqrt(piv[k]);
-  __syncthreads();
+  const int p = rp.p, P = (p + 7) & ~7, nb = (p + 7) >> 3;
   float* out = lbuf + (size_t)blockIdx.x * kLbufStride;
-  // row i of the layout holds L[j][i] for j = (i & ~3) .. P-1; identity beyond p
-  const int total = lt_row_offset(P, P);
+  // identity padding of the layout rows / columns p .. P-1 and the entries left of the diagonal
   for (int i = threadIdx.x >> 5; i < P; i += blockDim.x >> 5) {
     int j0 = i & ~3;
     float* row = out + lt_row_offset(i, P) - j0;
-    for (int j = j0 + (threadIdx.x & 31); j < P; j += 32) {
-      float v = 0.f;
-      if (i < p && j < p) {
-        if (j == i) v = (float)sqrt(piv[i]);
-        else if (j > i) v = (float)(A[tri_index(j, i)] * d0[i]);
-      } else if (i == j) {
-        v = 1.f;
-      }
-      row[j] = v;
-    }
+    for (int j = j0 + (threadIdx.x & 31); j < P; j += 32)
+      if (j < i || i >= p || j >= p) row[j] = (i == j) ? 1.f : 0.f;
   }
-  (void)total;
-  for (int j = threadIdx.x; j < P; j += blockDim.x)
-    out[kLtFloats + j] = j < p ? (float)d0[j] : 1.f;
+  for (int j = p + threadIdx.x; j < P; j += blockDim.x) out[kLtFloats + j] = 1.f;
+  auto load = [&](int i, int j) { return gram_entry(rp, partial, i, j); };
+  // row j of the layout holds L[i][j] for i >= (j & ~3)
+  auto store = [&](int i, int j, double v, double rdj) {
+    out[lt_row_offset(j, P) + i - (j & ~3)] = (float)v;
+    if (i == j) out[kLtFloats + j] = (float)rdj;
+  };
+  cholesky_blocked(p, sm_d, sm_d + (size_t)nb * (nb + 1) / 2 * 64, load, store);
 }
 
-// Dynamic shared memory: (p(p+1)/2 + 2p) doubles + p * ldc floats, ldc = p | 1.
-__global__ void __launch_bounds__(1024)
-ritz_kernel(const ReqPlan* __restrict__ plan, const double* __restrict__ partial,
-            float* __restrict__ ut, float* __restrict__ theta, int max_sweeps, int* status) {
-  extern __shared__ double sm_d[];
-  __shared__ float s_max;
-  ReqPlan rp = plan[blockIdx.x];
-  if (!rp.stage2) return;
-  const int p = rp.p, tri = p * (p + 1) / 2, tid = threadIdx.x, nt = blockDim.x;
-  double* A = sm_d;
-  double* piv = A + tri;
-  double* d0 = piv + p;
-  const int ldc = p | 1;
-  float* C = reinterpret_cast<float*>(d0 + p);          // columns of L: C[c * ldc + row]
-  float* sig = C + (size_t)p * ldc;                     // [p] column norms at the end
-  gram_cholesky(rp, partial, A, piv, d0);
-  for (int k = tid; k < p; k += nt) d0[k] = 1.0 / sqrt(piv[k]);
-  __syncthreads();
-  for (int e = tid; e < p * p; e += nt) {
-    int c = e / p, row = e % p;
-    float v = 0.f;
-    if (row == c) v = (float)sqrt(piv[c]);
-    else if (row > c) v = (float)(A[tri_index(row, c)] * d0[c]);
-    C[c * ldc + row] = v;
-  }
-  __syncthreads();
-  // One-sided Jacobi: rotate column pairs until all columns are mutually orthogonal.  Round-robin
-  // ordering, p/2 disjoint pairs per round, one 16-lane group per pair.
-  const int np = (p + 1) & ~1, half = np >> 1;
+// One-sided Jacobi on the w columns C[c * ldc + row] (w <= 16 * ROWS): rotate column pairs until
+// they are mutually orthogonal.  Round-robin ordering, w/2 disjoint pairs per round, one 16-lane
+// group per pair, the two columns held in registers between the inner products and the rotation.
+// A pair is left alone when its inner product g is negligible against the two norms
+// (g^2 <= 1e-12 |a|^2 |b|^2) or so small that the energies move by less than ~2e-5 of the
+// problem's scale s1 (g^2 <= (2e-5 s1)^2 min(|a|^2, |b|^2)).  Returns false when max_sweeps sweeps
+// did not reach a sweep without rotations.
+template <int ROWS>
+__device__ __forceinline__ bool jacobi_sweeps(float* C, int ldc, int w, float s1, int max_sweeps) {
+  const int tid = threadIdx.x, nt = blockDim.x;
+  const int np = (w + 1) & ~1, half = np >> 1;
   const int g = tid >> 4, gl = tid & 15, ng = nt >> 4;
-  bool converged = p < 2;
+  const float abs2 = (2e-5f * s1) * (2e-5f * s1);
+  bool converged = w < 2;
   for (int sweep = 0; sweep < max_sweeps && !converged; ++sweep) {
     int rotated = 0;
     for (int round = 0; round < np - 1; ++round) {
@@ -132,33 +198,45 @@ ritz_kernel(const ReqPlan* __restrict__ plan, const double* __restrict__ partial
         int a = 0, b = 0;
         bool active = i < half;
         if (active) {
-          a = i == 0 ? round : (round + i) % (np - 1);
-          b = i == 0 ? np - 1 : (round - i + np - 1) % (np - 1);
+          a = round + i; if (a >= np - 1) a -= np - 1;
+          b = round - i; if (b < 0) b += np - 1;
+          if (i == 0) { a = round; b = np - 1; }
           if (a > b) { int t = a; a = b; b = t; }
-          active = b < p;
+          active = b < w;
         }
         float* ca = C + a * ldc;
         float* cb = C + b * ldc;
+        float xa[ROWS], xb[ROWS];
         float al = 0.f, be = 0.f, ga = 0.f;
-        if (active)
-          for (int row = gl; row < p; row += 16) {
-            float x = ca[row], y = cb[row];
-            al += x * x; be += y * y; ga += x * y;
-          }
+#pragma unroll
+        for (int q = 0; q < ROWS; ++q) {
+          int row = gl + 16 * q;
+          bool in = active && row < w;
+          xa[q] = in ? ca[row] : 0.f;
+          xb[q] = in ? cb[row] : 0.f;
+          al += xa[q] * xa[q]; be += xb[q] * xb[q]; ga += xa[q] * xb[q];
+        }
 #pragma unroll
         for (int o = 8; o > 0; o >>= 1) {
           al += __shfl_xor_sync(0xffffffffu, al, o);
           be += __shfl_xor_sync(0xffffffffu, be, o);
           ga += __shfl_xor_sync(0xffffffffu, ga, o);
         }
-        if (active && fabsf(ga) > 1e-6f * sqrtf(al * be) && fabsf(ga) > 1e-36f) {
-          float zeta = (be - al) / (2.f * ga);
-          float t = (zeta >= 0.f ? 1.f : -1.f) / (fabsf(zeta) + sqrtf(zeta * zeta + 1.f));
-          float c = rsqrtf(t * t + 1.f), s = t * c;
-          for (int row = gl; row < p; row += 16) {
-            float x = ca[row], y = cb[row];
-            ca[row] = c * x - s * y;
-            cb[row] = s * x + c * y;
+        float g2 = ga * ga;
+        float thr2 = fmaxf(1e-12f * al * be, abs2 * fminf(al, be));
+        if (active && g2 > thr2 && g2 > 1e-37f) {
+          // tan of the rotation angle: t = sign(d g) 2|g| / (|d| + sqrt(d^2 + 4 g^2)), d = |b|^2 - |a|^2
+          float d = be - al;
+          float t = __fdividef(2.f * ga, fabsf(d) + __fsqrt_rn(d * d + 4.f * g2));
+          if (d < 0.f) t = -t;
+          float c = rsqrtf(t * t + 1.f), sn = t * c;
+#pragma unroll
+          for (int q = 0; q < ROWS; ++q) {
+            int row = gl + 16 * q;
+            if (row < w) {
+              ca[row] = c * xa[q] - sn * xb[q];
+              cb[row] = sn * xa[q] + c * xb[q];
+            }
           }
           rotated = 1;
         }
@@ -167,85 +245,147 @@ ritz_kernel(const ReqPlan* __restrict__ plan, const double* __restrict__ partial
     }
     converged = __syncthreads_or(rotated) == 0;
   }
+  return converged;
+}
+
+// Rayleigh-Ritz on the trailing window (see the file comment).  One block of 512 threads per
+// request.  Output ub[j * nbot + k]: component j (window coordinates) of the unit eigenvector of
+// the k-th smallest Ritz value, k < nbot = p - r.
+// Dynamic shared memory: round_up(win * (win | 1) + win, 2) floats, then cholesky_smem_bytes(win).
+__global__ void __launch_bounds__(512)
+ritz_kernel(const ReqPlan* __restrict__ plan, const double* __restrict__ partial,
+            float* __restrict__ ub, int max_sweeps, int* status) {
+  extern __shared__ float sm_f[];
+  __shared__ float s_scale;
+  ReqPlan rp = plan[blockIdx.x];
+  if (!rp.stage2) return;
+  const int p = rp.p, w = rp.win, w0 = p - w, nbot = p - rp.r;
+  const int tid = threadIdx.x, nt = blockDim.x;
+  const int ldc = w | 1;
+  float* C = sm_f;                                  // columns of the factor: C[c * ldc + row]
+  float* sig = C + (size_t)w * ldc;                 // [w] column norms at the end
+  for (int e = tid; e < w * ldc; e += nt) C[e] = 0.f;
+  if (tid == 0) s_scale = 0.f;
+  __syncthreads();
+  // scale of the whole problem: sqrt of the largest diagonal entry of B' (~ the largest Ritz value)
+  {
+    float m = 0.f;
+    for (int i = tid; i < p; i += nt) m = fmaxf(m, (float)gram_entry(rp, partial, i, i));
+    m = warp_max(m);
+    if ((tid & 31) == 0 && m > 0.f) atomicMax(reinterpret_cast<int*>(&s_scale), __float_as_int(m));
+  }
+  auto load = [&](int i, int j) { return gram_entry(rp, partial, w0 + i, w0 + j); };
+  auto store = [&](int i, int j, double v, double) { C[j * ldc + i] = (float)v; };
+  {
+    const int nbw = (w + 7) >> 3;
+    double* Tw = reinterpret_cast<double*>(sm_f + (((size_t)w * ldc + w + 1) & ~(size_t)1));   // 8-byte aligned
+    cholesky_blocked(w, Tw, Tw + (size_t)nbw * (nbw + 1) / 2 * 64, load, store);
+  }
+  __syncthreads();
+  const float s1 = sqrtf(s_scale);
+  bool converged;
+  if (w <= 64) converged = jacobi_sweeps<4>(C, ldc, w, s1, max_sweeps);
+  else if (w <= 128) converged = jacobi_sweeps<8>(C, ldc, w, s1, max_sweeps);
+  else converged = jacobi_sweeps<(kPMax + 15) / 16>(C, ldc, w, s1, max_sweeps);
   if (!converged && tid == 0) atomicOr(status, kStatusNoConverge);
   // singular values = column norms
-  for (int k = tid >> 5; k < p; k += nt >> 5) {
+  for (int k = tid >> 5; k < w; k += nt >> 5) {
     float s = 0.f;
-    for (int row = tid & 31; row < p; row += 32) { float x = C[k * ldc + row]; s += x * x; }
+    for (int row = tid & 31; row < w; row += 32) { float x = C[k * ldc + row]; s += x * x; }
     s = warp_sum(s);
     if ((tid & 31) == 0) sig[k] = sqrtf(s);
   }
-  if (tid == 0) s_max = 0.f;
   __syncthreads();
-  if (tid < 32) {
-    float m = 0.f;
-    for (int k = tid; k < p; k += 32) m = fmaxf(m, sig[k]);
-    m = warp_max(m);
-    if (tid == 0) s_max = m;
-  }
-  __syncthreads();
-  // rank the columns by singular value (descending, ties by index); the r largest, scaled by
-  // s^-3/2, become the rows-by-rank matrix the energy kernel multiplies with: ut[j * r + rank]
-  float* out_u = ut + (size_t)blockIdx.x * kPMax * kPMax;
-  float* out_t = theta + (size_t)blockIdx.x * kPMax;
-  const int r = rp.r;
-  for (int k = tid >> 5; k < p; k += nt >> 5) {
+  // rank the columns by singular value (ascending, ties by larger index first so that the order is
+  // the reverse of the descending one); the nbot smallest become unit vectors ub[j * nbot + rank]
+  float* out_u = ub + (size_t)blockIdx.x * kPMax * kPMax;
+  for (int k = tid >> 5; k < w; k += nt >> 5) {
     float sk = sig[k];
     int rank = 0;
-    for (int q = tid & 31; q < p; q += 32) {
+    for (int q = tid & 31; q < w; q += 32) {
       float sq = sig[q];
-      rank += (sq > sk) || (sq == sk && q < k);
+      rank += (sq < sk) || (sq == sk && q > k);
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) rank += __shfl_xor_sync(0xffffffffu, rank, o);
-    if (rank < r) {
-      float scale = sk > 1e-6f * s_max ? 1.f / (sk * sqrtf(sk)) : 0.f;
-      for (int j = tid & 31; j < p; j += 32) out_u[j * r + rank] = C[k * ldc + j] * scale;
-      if ((tid & 31) == 0) out_t[rank] = sk;
+    if (rank < nbot) {
+      float scale = sk > 0.f ? 1.f / sk : 0.f;
+      for (int j = tid & 31; j < w; j += 32) out_u[j * nbot + rank] = C[k * ldc + j] * scale;
     }
   }
 }
 
-// Eq. 15 for the preselected tokens of every request: c_i = sum_{k<r} (sum_j Yf[i][j] ut[j][k])^2.
-// Requests without stage 2 get zeros.  grid = (ceil(max M / 64), batch), 256 threads: one warp per
-// token row, lanes over k.  Dynamic shared memory: p_max * r_max floats.
+// Eq. 15 for the preselected tokens (see the file comment).  grid = (ceil(max M / 128), batch),
+// 256 threads.  yq / yn: float32 blocks before and after the last power step, [sum M_b, kPMax].
+// Requests without stage 2 get zeros.
+// Dynamic shared memory: kLbufStride floats + p_max * kXsLd floats + win_max * nbot_max floats.
 __global__ void __launch_bounds__(256)
-energy_kernel(const ReqPlan* __restrict__ plan, const float* __restrict__ yf,
-              const float* __restrict__ ut, float* __restrict__ energy) {
-  extern __shared__ float sm_u[];
+energy_kernel(const ReqPlan* __restrict__ plan, const float* __restrict__ yq,
+              const float* __restrict__ yn, const float* __restrict__ lbuf,
+              const float* __restrict__ ub, int p_max, float* __restrict__ energy) {
+  extern __shared__ float sm_f[];
   ReqPlan rp = plan[blockIdx.y];
-  const int row0 = blockIdx.x * 64;
+  const int row0 = blockIdx.x * sub::kTile;
   if (row0 >= rp.m) return;
-  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int nrows = min(sub::kTile, rp.m - row0);
   if (!rp.stage2) {
-    for (int i = row0 + threadIdx.x; i < min(rp.m, row0 + 64); i += blockDim.x) energy[rp.presel_off + i] = 0.f;
+    for (int i = tid; i < nrows; i += blockDim.x) energy[rp.presel_off + row0 + i] = 0.f;
     return;
   }
-  const int p = rp.p, r = rp.r;
-  const float* u = ut + (size_t)blockIdx.y * kPMax * kPMax;
-  for (int e = threadIdx.x; e < p * r; e += blockDim.x) sm_u[e] = u[e];
-  __syncthreads();
-  for (int i = row0 + w; i < min(rp.m, row0 + 64); i += 8) {
-    const float* y = yf + ((size_t)rp.presel_off + i) * kPMax;
-    float acc[5] = {0.f, 0.f, 0.f, 0.f, 0.f};
-    for (int jc = 0; jc < p; jc += 32) {
-      float yv = jc + lane < p ? y[jc + lane] : 0.f;
-      int jn = min(32, p - jc);
-      for (int jj = 0; jj < jn; ++jj) {
-        float yj = __shfl_sync(0xffffffffu, yv, jj);
-        const float* ur = sm_u + (jc + jj) * r;
-#pragma unroll
-        for (int kk = 0; kk < 5; ++kk) {
-          int k = lane + 32 * kk;
-          if (k < r) acc[kk] += yj * ur[k];
-        }
-      }
+  const int p = rp.p, P = (p + 7) & ~7, w = rp.win, w0 = p - w, nbot = p - rp.r;
+  float* lt = sm_f;
+  float* dinv = lt + kLtFloats;
+  float* xs = lt + kLbufStride;                         // [P][kXsLd]: Y rows, then Q rows in place
+  float* us = xs + (size_t)p_max * kXsLd;               // [w][nbot]
+  {
+    const float4* src = reinterpret_cast<const float4*>(lbuf + (size_t)blockIdx.y * kLbufStride);
+    float4* dst = reinterpret_cast<float4*>(lt);
+    int n4 = (lt_row_offset(P, P) + 3) / 4;
+    for (int e = tid; e < n4; e += blockDim.x) dst[e] = src[e];
+    const float* dsrc = lbuf + (size_t)blockIdx.y * kLbufStride + kLtFloats;
+    for (int e = tid; e < P; e += blockDim.x) dinv[e] = dsrc[e];
+    const float* usrc = ub + (size_t)blockIdx.y * kPMax * kPMax;
+    for (int e = tid; e < w * nbot; e += blockDim.x) us[e] = usrc[e];
+    // previous block, transposed into xs[c][row]; rows beyond the tile and columns beyond p are 0
+    for (int e = tid; e < sub::kTile * P; e += blockDim.x) {
+      int rr = e / P, c = e - rr * P;
+      xs[c * kXsLd + rr] = (rr < nrows && c < p) ? yq[((size_t)rp.presel_off + row0 + rr) * kPMax + c] : 0.f;
     }
-    float c = 0.f;
+  }
+  __syncthreads();
+  // Q row = Y row * L^-T, one thread per row, in place
+  if (tid < sub::kTile) {
+    for (int jb = 0; jb < P; jb += 8) {
+      float acc[8];
 #pragma unroll
-    for (int kk = 0; kk < 5; ++kk) c += acc[kk] * acc[kk];
-    c = warp_sum(c);
-    if (lane == 0) energy[rp.presel_off + i] = c;
+      for (int e = 0; e < 8; ++e) acc[e] = xs[(jb + e) * kXsLd + tid];
+      sub::solve_block8(acc, jb, sub::smem_u32(lt), sub::smem_u32(dinv), sub::smem_u32(xs), tid, P);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) xs[(jb + e) * kXsLd + tid] = acc[e];
+    }
+  }
+  __syncthreads();
+  // one warp per row: total = sum_j Y'_ij Q_ij, minus the discarded Ritz pairs of the window
+  for (int rr = warp; rr < nrows; rr += 8) {
+    const float* yrow = yn + ((size_t)rp.presel_off + row0 + rr) * kPMax;
+    float total = 0.f;
+    for (int c = lane; c < p; c += 32) total += yrow[c] * xs[c * kXsLd + rr];
+    total = warp_sum(total);
+    float sub_ = 0.f;
+    for (int k0 = 0; k0 < nbot; k0 += 32) {
+      int k = k0 + lane;
+      float ya = 0.f, qa = 0.f;
+      if (k < nbot)
+        for (int j = 0; j < w; ++j) {
+          float u = us[j * nbot + k];
+          ya += yrow[w0 + j] * u;
+          qa += xs[(w0 + j) * kXsLd + rr] * u;
+        }
+      sub_ += ya * qa;
+    }
+    sub_ = warp_sum(sub_);
+    if (lane == 0) energy[rp.presel_off + row0 + rr] = fmaxf(total - sub_, 0.f);
   }
 }
 

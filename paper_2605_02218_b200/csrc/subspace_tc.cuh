@@ -271,9 +271,10 @@ constexpr int kPowStages = 2;
 constexpr int kPowBytesA = kTile * kBK * 2;              // one plane of the G tile, 16 KB
 constexpr int kPowBytesB = kPMax * kBK * 2;              // one plane of the Y tile, 20 KB
 constexpr int kPowStageBytes = 2 * kPowBytesA + 2 * kPowBytesB;   // 72 KB
-constexpr int kXsLd = kTile + 1;                         // row stride of the staged block (floats)
+constexpr int kXsLd = kTile + 4;                         // row stride of the staged block (floats)
 constexpr int kPowSmem = kPowStages * kPowStageBytes + kLbufStride * 4 + 1024 + 1024;
 constexpr int kPowTmemCols = 256;
+constexpr int kPowThreads = 320;                         // 8 epilogue warps, TMA producer, MMA issuer
 static_assert(kPMax * kXsLd * 4 <= kPowStages * kPowStageBytes, "staged block must fit in the ring");
 
 struct PowerParams {
@@ -281,17 +282,161 @@ struct PowerParams {
   int batch;
   int n_items;              // 128-row tiles over all stage-2 requests
   int identity;             // first step: no triangular factor yet
-  int last;                 // last step: also write the float32 block
   const float* lbuf;        // [batch][kLbufStride] triangular factor + reciprocal diagonal
   __nv_bfloat16* y_hi;      // output planes
   __nv_bfloat16* y_lo;
   int ld;
-  float* yf;                // [sum M_b, kPMax] (last step)
+  float* yf;                // [sum M_b, kPMax] float32 copy of the new block, or nullptr
   double* partial;          // [tiles][kTriMax]
   int* status;
 };
 
-__global__ void __launch_bounds__(192, 1)
+__device__ __forceinline__ float lds_f32(uint32_t addr) {
+  float v;
+  asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(addr));
+  return v;
+}
+__device__ __forceinline__ float4 lds_v4(uint32_t addr) {
+  float4 v;
+  asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
+  return v;
+}
+
+// Four rows i .. i+3 of the triangular layout (two float4 each) and the matching four x_i.
+struct SolveGroup {
+  float x[4];
+  float4 l[4][2];
+};
+__device__ __forceinline__ void solve_group_load(SolveGroup& g, uint32_t xs_row, uint32_t lt_at, int stride) {
+#pragma unroll
+  for (int q = 0; q < 4; ++q) g.x[q] = lds_f32(xs_row + q * kXsLd * 4);
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    g.l[q][0] = lds_v4(lt_at + q * stride * 4);
+    g.l[q][1] = lds_v4(lt_at + q * stride * 4 + 16);
+  }
+}
+__device__ __forceinline__ void solve_group_apply(const SolveGroup& g, float (&acc)[8]) {
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    acc[0] -= g.x[q] * g.l[q][0].x; acc[1] -= g.x[q] * g.l[q][0].y;
+    acc[2] -= g.x[q] * g.l[q][0].z; acc[3] -= g.x[q] * g.l[q][0].w;
+    acc[4] -= g.x[q] * g.l[q][1].x; acc[5] -= g.x[q] * g.l[q][1].y;
+    acc[6] -= g.x[q] * g.l[q][1].z; acc[7] -= g.x[q] * g.l[q][1].w;
+  }
+}
+
+// Columns jb .. jb+7 of one row of X = T L^-T (blocked forward substitution).  acc holds
+// t[jb..jb+7] on entry and x[jb..jb+7] on return; the x_i already solved are read from the staged
+// block xs[i * kXsLd + r].  lt / dinv: the factor in the layout of lt_row_offset for width P and
+// its reciprocal diagonal.  All three are shared-memory addresses (32-bit window offsets); the
+// loads of one group of four rows are in flight while the previous group is applied.
+__device__ __forceinline__ void solve_block8(float (&acc)[8], int jb, uint32_t lt, uint32_t dinv,
+                                             uint32_t xs, int r, int P) {
+  const int groups = jb >> 2;                      // even: jb is a multiple of 8
+  if (groups > 0) {
+    uint32_t xr = xs + r * 4;
+    uint32_t at = lt + jb * 4;                     // lt_row_offset(i, P) + jb - 4 * (i >> 2) at i = 0
+    int stride = P;                                // rows 4a .. 4a+3 have P - 4a entries
+    SolveGroup ga, gb;
+    solve_group_load(ga, xr, at, stride);
+    for (int g = 0; g < groups; g += 2) {
+      xr += 4 * kXsLd * 4; at += (4 * stride - 4) * 4; stride -= 4;
+      solve_group_load(gb, xr, at, stride);
+      solve_group_apply(ga, acc);
+      xr += 4 * kXsLd * 4; at += (4 * stride - 4) * 4; stride -= 4;
+      if (g + 2 < groups) solve_group_load(ga, xr, at, stride);
+      solve_group_apply(gb, acc);
+    }
+  }
+  // triangular solve inside the block: row jb+jj of the layout starts at column jb + (jj & ~3)
+#pragma unroll
+  for (int jj = 0; jj < 8; ++jj) {
+    float x = acc[jj] * lds_f32(dinv + (jb + jj) * 4);
+    acc[jj] = x;
+    uint32_t lr = lt + (lt_row_offset(jb + jj, P) - (jj & ~3)) * 4;
+#pragma unroll
+    for (int j2 = jj + 1; j2 < 8; ++j2) acc[j2] -= x * lds_f32(lr + j2 * 4);
+  }
+}
+
+// C (8x8 float64, two entries per thread) += A (8x4) * B (4x8): one tensor-core instruction.
+__device__ __forceinline__ void dmma_8x8x4(double& c0, double& c1, double a, double b) {
+  asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};"
+               : "+d"(c0), "+d"(c1)
+               : "d"(a), "d"(b));
+}
+
+// The float64 Gram of the staged block is accumulated from 16-row slabs converted to float64 in
+// shared memory (slab[c * kSlabLd + row]); a warp owns two strips of 8x8 tiles, (ta, tb <= ta) and
+// (tz = nb8-1-ta, tb <= tz), so that every warp carries nb8 + 1 tiles.
+constexpr int kSlabRows = 16;
+constexpr int kSlabLd = 20;                      // doubles; conflict-free fragment loads
+constexpr int kMaxTiles8 = kPMax / 8;            // 20
+constexpr int kXsBytes = (kPMax * kXsLd * 4 + 1023) / 1024 * 1024;
+static_assert(kXsBytes + 2 * kPMax * kSlabLd * 8 <= kPowStages * kPowStageBytes, "slabs must fit in the ring");
+
+// Accumulator slots of one warp: strip ta (the shorter one) uses slots 0 .. ta for tb = slot,
+// strip tz uses slots kMaxTiles8 - tb for tb = 0 .. tz; ta + tz = nb8 - 1 <= 19, so they never meet.
+struct GramAcc {
+  double a[kMaxTiles8 + 1][2];
+};
+
+// The tensor-core instructions sit behind warp-uniform jump tables (switch fall-through), not
+// predicates: a predicated-off mma still occupies the FP64 pipe.
+#define COVSPEC_GRAM_A(u) case u: dmma_8x8x4(acc.a[u][0], acc.a[u][1], xa, b[u]);
+#define COVSPEC_GRAM_Z(t) case t: dmma_8x8x4(acc.a[kMaxTiles8 - t][0], acc.a[kMaxTiles8 - t][1], xz, b[t]);
+__device__ __forceinline__ void gram_unit_accumulate(GramAcc& acc, const double* slab, int ta, int tz,
+                                                     int lane) {
+  const int fr = lane >> 2, fk = lane & 3;
+  const double* base = slab + fr * kSlabLd + fk;
+#pragma unroll 1
+  for (int ks = 0; ks < kSlabRows / 4; ++ks) {
+    double b[kMaxTiles8];
+#pragma unroll
+    for (int t = 0; t < kMaxTiles8; ++t)
+      if (t <= tz) b[t] = base[t * 8 * kSlabLd + 4 * ks];
+    const double xa = base[ta * 8 * kSlabLd + 4 * ks], xz = base[tz * 8 * kSlabLd + 4 * ks];
+    switch (ta) {
+      COVSPEC_GRAM_A(19) COVSPEC_GRAM_A(18) COVSPEC_GRAM_A(17) COVSPEC_GRAM_A(16) COVSPEC_GRAM_A(15)
+      COVSPEC_GRAM_A(14) COVSPEC_GRAM_A(13) COVSPEC_GRAM_A(12) COVSPEC_GRAM_A(11) COVSPEC_GRAM_A(10)
+      COVSPEC_GRAM_A(9) COVSPEC_GRAM_A(8) COVSPEC_GRAM_A(7) COVSPEC_GRAM_A(6) COVSPEC_GRAM_A(5)
+      COVSPEC_GRAM_A(4) COVSPEC_GRAM_A(3) COVSPEC_GRAM_A(2) COVSPEC_GRAM_A(1) COVSPEC_GRAM_A(0)
+      default: break;
+    }
+    if (tz != ta) {
+      switch (tz) {
+        COVSPEC_GRAM_Z(19) COVSPEC_GRAM_Z(18) COVSPEC_GRAM_Z(17) COVSPEC_GRAM_Z(16) COVSPEC_GRAM_Z(15)
+        COVSPEC_GRAM_Z(14) COVSPEC_GRAM_Z(13) COVSPEC_GRAM_Z(12) COVSPEC_GRAM_Z(11) COVSPEC_GRAM_Z(10)
+        COVSPEC_GRAM_Z(9) COVSPEC_GRAM_Z(8) COVSPEC_GRAM_Z(7) COVSPEC_GRAM_Z(6) COVSPEC_GRAM_Z(5)
+        COVSPEC_GRAM_Z(4) COVSPEC_GRAM_Z(3) COVSPEC_GRAM_Z(2) COVSPEC_GRAM_Z(1) COVSPEC_GRAM_Z(0)
+        default: break;
+      }
+    }
+  }
+}
+#undef COVSPEC_GRAM_A
+#undef COVSPEC_GRAM_Z
+
+// Writes the accumulated tiles of one warp to the packed lower triangle.
+__device__ __forceinline__ void gram_unit_store(const GramAcc& acc, int ta, int tz, int p, int lane,
+                                                double* __restrict__ out) {
+  const int fr = lane >> 2, fk = lane & 3;
+#pragma unroll
+  for (int u = 0; u <= kMaxTiles8; ++u) {
+    int strip = -1, tb = 0;
+    if (u < kMaxTiles8 && u <= ta) { strip = ta; tb = u; }
+    else if (u >= 1 && kMaxTiles8 - u <= tz && tz != ta) { strip = tz; tb = kMaxTiles8 - u; }
+    if (strip < 0) continue;
+    int row = 8 * strip + fr, col = 8 * tb + 2 * fk;
+    if (row < p) {
+      if (col <= row) out[tri_index(row, col)] = acc.a[u][0];
+      if (col + 1 <= row) out[tri_index(row, col + 1)] = acc.a[u][1];
+    }
+  }
+}
+
+__global__ void __launch_bounds__(kPowThreads, 1)
 power_tc_kernel(const __grid_constant__ CUtensorMap map_gh, const __grid_constant__ CUtensorMap map_gl,
                 const __grid_constant__ CUtensorMap map_yh, const __grid_constant__ CUtensorMap map_yl,
                 const PowerParams prm) {
@@ -314,11 +459,11 @@ power_tc_kernel(const __grid_constant__ CUtensorMap map_gh, const __grid_constan
     for (int s = 0; s < kPowStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
     mbar_init(acc_full, 1);
     mbar_init(acc_empty, 128);
-    mbar_init(epi_done, 128);
+    mbar_init(epi_done, 256);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (warp == 5) tmem_alloc(tmem_slot, kPowTmemCols);
+  if (warp == 9) tmem_alloc(tmem_slot, kPowTmemCols);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -330,7 +475,7 @@ power_tc_kernel(const __grid_constant__ CUtensorMap map_gh, const __grid_constan
     tile = item - rp.ptile_off;
   };
 
-  if (warp == 4) {
+  if (warp == 8) {
     if (lane == 0) {
       uint32_t it = 0, n = 0;
       bool ok = true;
@@ -354,7 +499,7 @@ power_tc_kernel(const __grid_constant__ CUtensorMap map_gh, const __grid_constan
       }
     }
     __syncwarp();
-  } else if (warp == 5) {
+  } else if (warp == 9) {
     if (lane == 0) {
       uint32_t it = 0, n = 0;
       bool ok = true;
@@ -387,125 +532,110 @@ power_tc_kernel(const __grid_constant__ CUtensorMap map_gh, const __grid_constan
     }
     __syncwarp();
   } else {
-    const int r = warp * 32 + lane;
-    const uint32_t t_lane = tmem_base + ((uint32_t)(warp * 32) << 16);
+    // ------------------------------------------------------------ epilogue, warps 0-7
+    const int et = threadIdx.x;                    // 0 .. 255
+    const int r = (warp & 3) * 32 + lane;          // TMEM lane = row of the tile (warps 0-3 solve)
+    const uint32_t t_lane = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
     uint32_t n = 0;
     int cached_b = -1;
     bool ok = true;
-    for (int item = blockIdx.x; item < prm.n_items && ok; item += gridDim.x, ++n) {
+    for (int item = blockIdx.x; item < prm.n_items; item += gridDim.x, ++n) {
       int b, tile; ReqPlan rp;
       decode(item, b, rp, tile);
       const int p = rp.p, P = (p + 7) & ~7;
       if (!prm.identity && b != cached_b) {
-        named_barrier(1, 128);                     // nobody still reads the previous factor
+        named_barrier(1, 256);                     // nobody still reads the previous factor
         const float4* src = reinterpret_cast<const float4*>(prm.lbuf + (size_t)b * kLbufStride);
         float4* dst = reinterpret_cast<float4*>(lt);
         int n4 = (lt_row_offset(P, P) + 3) / 4;    // floats used by the P-wide layout
-        for (int e = r; e < n4; e += 128) dst[e] = src[e];
+        for (int e = et; e < n4; e += 256) dst[e] = src[e];
         const float* dsrc = prm.lbuf + (size_t)b * kLbufStride + kLtFloats;
-        for (int e = r; e < P; e += 128) dinv[e] = dsrc[e];
-        named_barrier(1, 128);
+        for (int e = et; e < P; e += 256) dinv[e] = dsrc[e];
+        named_barrier(1, 256);
         cached_b = b;
       }
-      if (!(ok = mbar_wait(acc_full, n & 1u, abort_flag))) break;
-      tc_fence_after();
-      const int row = tile * kTile + r;
-      const bool row_ok = row < rp.m;
-      // ---- Y_next row = T row * L^-T by blocked forward substitution; staged as xs[c][r] ----
+      const int nrows = min(kTile, rp.m - tile * kTile);
+      if (warp < 4) {
+        ok = ok && mbar_wait(acc_full, n & 1u, abort_flag);
+        tc_fence_after();
+        const bool row_ok = r < nrows;
+        // ---- Y_next row = T row * L^-T; staged as xs[c][r] ----
 #pragma unroll 1
-      for (int cb = 0; cb * 32 < P; ++cb) {
-        float v[32];
-        tmem_ld32(t_lane + cb * 32, v);
+        for (int cb = 0; cb * 32 < P; ++cb) {
+          float v[32];
+          tmem_ld32(t_lane + cb * 32, v);
 #pragma unroll
-        for (int sb = 0; sb < 4; ++sb) {
-          const int jb = cb * 32 + sb * 8;
-          if (jb < P) {
-            float acc[8];
+          for (int sb = 0; sb < 4; ++sb) {
+            const int jb = cb * 32 + sb * 8;
+            if (jb < P) {
+              float acc[8];
 #pragma unroll
-            for (int e = 0; e < 8; ++e) acc[e] = v[sb * 8 + e];
-            if (!prm.identity) {
-              int off = jb;                         // lt_row_offset(i, P) + jb - 4 * (i >> 2), i = 0
-#pragma unroll 2
-              for (int i = 0; i < jb; ++i) {
-                float xi = xs[i * kXsLd + r];
-                float4 l0 = *reinterpret_cast<const float4*>(lt + off);
-                float4 l1 = *reinterpret_cast<const float4*>(lt + off + 4);
-                acc[0] -= xi * l0.x; acc[1] -= xi * l0.y; acc[2] -= xi * l0.z; acc[3] -= xi * l0.w;
-                acc[4] -= xi * l1.x; acc[5] -= xi * l1.y; acc[6] -= xi * l1.z; acc[7] -= xi * l1.w;
-                off += P - 4 * (i >> 2) - (((i & 3) == 3) ? 4 : 0);
-              }
-              // triangular solve inside the 8-column block (rows jb .. jb+7 of the layout)
-              const float* lrow = lt + lt_row_offset(jb, P);          // row jb starts at column jb
+              for (int e = 0; e < 8; ++e) acc[e] = v[sb * 8 + e];
+              if (!prm.identity) solve_block8(acc, jb, smem_u32(lt), smem_u32(dinv), smem_u32(xs), r, P);
 #pragma unroll
-              for (int jj = 0; jj < 8; ++jj) {
-                float x = acc[jj] * dinv[jb + jj];
-                acc[jj] = x;
-                // row jb+jj holds columns from jb + (jj & ~3)
-                const float* lr = lt + lt_row_offset(jb + jj, P) - (jj & ~3);
-#pragma unroll
-                for (int j2 = jj + 1; j2 < 8; ++j2) acc[j2] -= x * lr[j2];
-              }
-              (void)lrow;
+              for (int e = 0; e < 8; ++e) xs[(jb + e) * kXsLd + r] = (row_ok && ok) ? acc[e] : 0.f;
             }
-#pragma unroll
-            for (int e = 0; e < 8; ++e) xs[(jb + e) * kXsLd + r] = row_ok ? acc[e] : 0.f;
           }
         }
+        tc_fence_before();
+        mbar_arrive(acc_empty);
       }
-      tc_fence_before();
-      mbar_arrive(acc_empty);
-      named_barrier(1, 128);                       // the staged block is complete
-      // ---- bf16 planes of the new block (K-major operand of the next step) ----
-      const int cols = (rp.m + kBK - 1) / kBK * kBK;
-      if (row < cols) {
-        size_t o = ((size_t)b * kPMax) * prm.ld + row;
-        for (int c = 0; c < p; ++c) {
-          __nv_bfloat16 hi, lo;
-          split_bf16(xs[c * kXsLd + r], hi, lo);
-          prm.y_hi[o + (size_t)c * prm.ld] = hi;
-          prm.y_lo[o + (size_t)c * prm.ld] = lo;
+      named_barrier(1, 256);                       // the staged block is complete
+      // ---- bf16 planes of the new block (K-major operand of the next step): 8 positions per thread
+      {
+        const int cols = (rp.m + kBK - 1) / kBK * kBK;
+        for (int wi = et; wi < p * 16; wi += 256) {
+          int c = wi >> 4, ch = wi & 15;
+          int pos = tile * kTile + ch * 8;
+          if (pos >= cols) continue;
+          const float4* xp = reinterpret_cast<const float4*>(xs + c * kXsLd + ch * 8);
+          float4 a = xp[0], d = xp[1];
+          float f[8] = {a.x, a.y, a.z, a.w, d.x, d.y, d.z, d.w};
+          uint32_t ph[4], pl[4];
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            __nv_bfloat162 hi = __floats2bfloat162_rn(f[2 * e], f[2 * e + 1]);
+            ph[e] = *reinterpret_cast<uint32_t*>(&hi);
+            pl[e] = pack_bf16(f[2 * e] - __low2float(hi), f[2 * e + 1] - __high2float(hi));
+          }
+          size_t o = ((size_t)b * kPMax + c) * prm.ld + pos;
+          *reinterpret_cast<uint4*>(prm.y_hi + o) = make_uint4(ph[0], ph[1], ph[2], ph[3]);
+          *reinterpret_cast<uint4*>(prm.y_lo + o) = make_uint4(pl[0], pl[1], pl[2], pl[3]);
         }
       }
-      if (prm.last) {
-        // float32 block, one token per row: thread e of the tile walks (row, column) pairs so that
-        // consecutive threads write consecutive columns
-        int nrows = min(kTile, rp.m - tile * kTile);
-        for (int e = r; e < nrows * p; e += 128) {
-          int rr = e / p, c = e % p;
+      if (prm.yf != nullptr) {
+        // float32 block, one token per row; consecutive threads write consecutive columns
+        for (int e = et; e < nrows * p; e += 256) {
+          int rr = e / p, c = e - rr * p;
           prm.yf[((size_t)rp.presel_off + tile * kTile + rr) * kPMax + c] = xs[c * kXsLd + rr];
         }
       }
-      // ---- float64 partial Gram of the tile: B[a][b] = sum_r x[a][r] x[b][r], b <= a ----
+      // ---- float64 partial Gram of the tile on the FP64 tensor cores ----
       {
-        int nrows = min(kTile, rp.m - tile * kTile);
-        int nb = (p + 3) >> 2, nblk = nb * (nb + 1) / 2;
+        const int nb8 = (p + 7) >> 3, units = (nb8 + 1) / 2, nslab = (nrows + kSlabRows - 1) / kSlabRows;
+        double* slabs = reinterpret_cast<double*>(smem + kXsBytes);
         double* out = prm.partial + (size_t)item * kTriMax;
-        for (int blk = r; blk < nblk; blk += 128) {
-          int ba, bb;
-          tri_decode(blk, ba, bb);
-          double acc[4][4];
+        for (int u0 = 0; u0 < units; u0 += 8) {
+          const int unit = u0 + warp;
+          const bool have = unit < units;
+          const int ta = have ? unit : 0, tz = have ? nb8 - 1 - unit : 0;
+          GramAcc acc;
 #pragma unroll
-          for (int i = 0; i < 4; ++i)
-#pragma unroll
-            for (int j = 0; j < 4; ++j) acc[i][j] = 0.0;
-          const float* xa = xs + (4 * ba) * kXsLd;
-          const float* xb = xs + (4 * bb) * kXsLd;
-          for (int rr = 0; rr < nrows; ++rr) {
-            double a[4], c[4];
-#pragma unroll
-            for (int i = 0; i < 4; ++i) { a[i] = (double)xa[i * kXsLd + rr]; c[i] = (double)xb[i * kXsLd + rr]; }
-#pragma unroll
-            for (int i = 0; i < 4; ++i)
-#pragma unroll
-              for (int j = 0; j < 4; ++j) acc[i][j] += a[i] * c[j];
-          }
-#pragma unroll
-          for (int i = 0; i < 4; ++i)
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-              int ia = 4 * ba + i, ib = 4 * bb + j;
-              if (ia < p && ib <= ia) out[tri_index(ia, ib)] = acc[i][j];
+          for (int u = 0; u <= kMaxTiles8; ++u) { acc.a[u][0] = 0.0; acc.a[u][1] = 0.0; }
+          for (int sl = 0; sl < nslab; ++sl) {
+            double* slab = slabs + (sl & 1) * (kPMax * kSlabLd);
+            // float32 -> float64, rows 16 sl .. 16 sl + 15 of every column (zero beyond the tile)
+            for (int e = et; e < P * kSlabRows; e += 256) {
+              int c = e >> 4, rr = e & 15;
+              slab[c * kSlabLd + rr] = (double)xs[c * kXsLd + sl * kSlabRows + rr];
             }
+            named_barrier(1, 256);
+            if (have) gram_unit_accumulate(acc, slab, ta, tz, lane);
+            // the other buffer is refilled next; this one is reused two slabs later, after the
+            // barrier of the next slab
+          }
+          if (have) gram_unit_store(acc, ta, tz, p, lane, out);
+          named_barrier(1, 256);
         }
       }
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -515,7 +645,7 @@ power_tc_kernel(const __grid_constant__ CUtensorMap map_gh, const __grid_constan
 
   tc_fence_before();
   __syncthreads();
-  if (warp == 5) tmem_dealloc(tmem_base, kPowTmemCols);
+  if (warp == 9) tmem_dealloc(tmem_base, kPowTmemCols);
   if (threadIdx.x == 0 && *abort_flag) atomicOr(prm.status, kStatusTimeout);
 }
 
