@@ -96,6 +96,47 @@ def test_config_c2():
     _report("c2", parity.run_gpu(wl))
 
 
+def _full_size(name, requests):
+    """Full-size configuration generated on the device (the launch configuration bench.py times);
+    the oracle checks a sample of whole requests, every output of those requests element by element."""
+    wl = workloads.make_config(name, device="cuda:0")
+    if requests is None:                  # ragged batch: the smallest, the largest and one more
+        n = np.diff(wl.vis_offsets)
+        requests = sorted({int(np.argmin(n)), int(np.argmax(n)), 7})
+    stats = parity.run_gpu(wl, requests=requests)
+    _report(name, stats)
+    assert stats["requests"] == len(requests)
+    del wl
+    torch.cuda.empty_cache()
+
+
+def test_config_c3_sampled():
+    _full_size("c3", [0, 31])
+
+
+def test_config_c4_sampled():
+    _full_size("c4", None)
+
+
+def test_config_c5_sampled():
+    _full_size("c5", [3])
+
+
+def test_slowly_decaying_spectrum():
+    # No gap anywhere: singular values k^-0.7.  The subspace iteration converges slowest here; the
+    # default number of steps must still leave the energies inside the tolerance.
+    wl = workloads.make_workload("decay", seed=5, dtype=torch.bfloat16, batch=2, n_vis=1200, n_txt=16,
+                                 d=768, n_heads=0, rank=16, keep_ratio=0.2)
+    g = torch.Generator().manual_seed(9)
+    n, d = wl.X.shape
+    U = torch.linalg.qr(torch.randn(n, d, generator=g))[0]
+    V = torch.linalg.qr(torch.randn(d, d, generator=g))[0]
+    sv = torch.arange(1, d + 1, dtype=torch.float32) ** -0.7
+    wl.X = ((U * sv) @ V.T * 30).to(torch.bfloat16)
+    wl.Hs = [wl.X.clone()] + wl.Hs[1:]
+    _report(wl.name, parity.run_gpu(wl))
+
+
 def test_determinism_and_plan_cache():
     from paper_2605_02218_b200 import api
     wl = workloads.make_workload("det", seed=31, dtype=torch.bfloat16, batch=3, n_vis=(100, 400),
