@@ -206,8 +206,9 @@ def main():
     work = algorithmic_work(wl0)
     copies = args.copies or max(2, int(np.ceil(2 * 126e6 * 2 / work["input_bytes"])))
     copies = min(copies, 8)
-    sets = [wl0] + [workloads.make_config(args.config, device=dev, seed=base_seed + 1000 * rank + 17 * (i + 1))
-                    for i in range(copies - 1)]
+    sizes = (np.diff(wl0.vis_offsets).tolist(), np.diff(wl0.txt_offsets).tolist())
+    sets = [wl0] + [workloads.make_config(args.config, device=dev, seed=base_seed + 1000 * rank + 17 * (i + 1),
+                                          sizes=sizes) for i in range(copies - 1)]
     pr = api.Pruner.for_workload(wl0)
     ms = [pr.marshal(w) for w in sets]
     ko, _ = pr.plan_sizes(ms[0])

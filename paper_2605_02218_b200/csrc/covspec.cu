@@ -516,6 +516,7 @@ int select_impl(covspec_ctx* ctx, const covspec_problem* p, const float* s_fused
       pp.y_hi = ctx->Yp[out][0]; pp.y_lo = ctx->Yp[out][1]; pp.ld = ctx->ld;
       // the two last blocks are also kept in float32 for the energy kernel
       pp.yf = pass == cfg.eig_iters ? ctx->Yf[1] : pass == cfg.eig_iters - 1 ? ctx->Yf[0] : nullptr;
+      pp.qprev = pass == cfg.eig_iters ? ctx->Yf[0] : nullptr;
       pp.partial = ctx->partial; pp.status = ctx->status;
       sub::power_tc_kernel<<<grid, sub::kPowThreads, sub::kPowSmem, s>>>(
           ctx->map_gh, ctx->map_gl, ctx->map_y[in][0], ctx->map_y[in][1], pp);
@@ -527,13 +528,12 @@ int select_impl(covspec_ctx* ctx, const covspec_problem* p, const float* s_fused
     }
     size_t ritz_smem = (((size_t)pl.win_max * (pl.win_max | 1) + pl.win_max + 1) & ~(size_t)1) * sizeof(float) +
                        cholesky_smem_bytes(pl.win_max);
-    ritz_kernel<<<B, 512, ritz_smem, s>>>(ctx->d_plan, ctx->partial, ctx->Ub, 30, ctx->status);
+    ritz_kernel<<<B, pl.win_max <= 64 ? 256 : 512, ritz_smem, s>>>(ctx->d_plan, ctx->partial, ctx->Ub, 30, ctx->status);
     LAUNCH_CHECK(ctx);
   }
-  dim3 ge((pl.m_max + sub::kTile - 1) / sub::kTile, B);
-  int p8 = (pl.p_max + 7) & ~7;
-  size_t en_smem = ((size_t)sub::kLbufStride + (size_t)p8 * sub::kXsLd + (size_t)pl.win_max * pl.nbot_max) * sizeof(float);
-  energy_kernel<<<ge, 256, en_smem, s>>>(ctx->d_plan, ctx->Yf[0], ctx->Yf[1], ctx->Lbuf, ctx->Ub, p8, energy);
+  dim3 ge((pl.m_max + 63) / 64, B);
+  size_t en_smem = (size_t)pl.win_max * pl.nbot_max * sizeof(float);
+  energy_kernel<<<ge, 256, en_smem, s>>>(ctx->d_plan, ctx->Yf[0], ctx->Yf[1], ctx->Ub, energy);
   LAUNCH_CHECK(ctx);
   if (pl.n_stage2 > 0) prof_mark(ctx, ST_EIG, 1, s);
   prof_mark(ctx, ST_FINAL, 0, s);
@@ -703,7 +703,7 @@ int covspec_prune_init(const covspec_config* cfg, covspec_ctx** out) {
                                   (int)(((size_t)kPMax * (kPMax | 1) + kPMax + 2) * sizeof(float) +
                                         cholesky_smem_bytes(kPMax))) == cudaSuccess;
   ok = ok && cudaFuncSetAttribute(energy_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                  220 * 1024) == cudaSuccess;
+                                  (int)((size_t)kPMax * kPMax * sizeof(float))) == cudaSuccess;
   int dev = 0, cc_major = 0;
   ok = ok && cudaGetDevice(&dev) == cudaSuccess &&
        cudaDeviceGetAttribute(&ctx->num_sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess &&

@@ -47,7 +47,7 @@ __device__ __forceinline__ double rsqrt_f64(double x) {
 
 // Blocked right-looking Cholesky factorisation of an n x n float64 matrix kept in shared memory as
 // 8 x 8 tiles of its lower triangle (tile (I, J <= I) at T + tri_index(I, J) * 64, row-major).
-// Per 8-column panel: the diagonal tile is factored by one warp, the tiles below it are solved one
+// Per 8-column panel: the diagonal tile is factored by one thread in registers, the tiles below it are solved one
 // row per thread, and the trailing tiles take their rank-8 update on the FP64 tensor cores
 // (two m8n8k4 instructions per tile).  Three __syncthreads per panel.
 // A pivot below 1e-12 of its original diagonal entry (a numerically dependent direction) is
@@ -74,23 +74,32 @@ __device__ __forceinline__ void cholesky_blocked(int n, double* T, double* aux, 
   __syncthreads();
   for (int J = 0; J < nb; ++J) {
     double* D = T + tri_index(J, J) * 64;
-    if (warp == 0) {
-      // lanes 0..27 own the strictly-lower pairs (l, m < l) of the trailing updates
-      int l = 1, m = 0;
-      { int q = lane; while (q >= l) { q -= l; ++l; } m = q; }   // pair index -> (l, m), l in 1..7
+    if (tid == 0) {
+      // 8 x 8 diagonal tile: one thread, everything in registers (the chain of eight dependent
+      // reciprocal square roots is the critical path of the whole factorisation)
+      double a[8][8];
+#pragma unroll
+      for (int l = 0; l < 8; ++l)
+#pragma unroll
+        for (int m = 0; m <= l; ++m) a[l][m] = D[l * 8 + m];
+#pragma unroll
       for (int c = 0; c < 8; ++c) {
-        double piv = D[c * 8 + c], floor_ = 1e-12 * d0[8 * J + c];
+        double piv = a[c][c], floor_ = 1e-12 * d0[8 * J + c];
         if (!(piv > floor_)) piv = floor_ > 0.0 ? floor_ : 1.0;
         double rs = rsqrt_f64(piv);
-        __syncwarp();
-        if (lane == 0) { D[c * 8 + c] = piv * rs; rd[8 * J + c] = rs; }
-        if (lane > c && lane < 8) D[lane * 8 + c] *= rs;
-        __syncwarp();
-        // D[l][m] -= L[l][c] L[m][c] for c < m <= l, including the diagonal (lanes 28..31 + spare)
-        if (lane < 28 && m > c) D[l * 8 + m] -= D[l * 8 + c] * D[m * 8 + c];
-        if (lane >= 24 && lane - 24 > c) { int dgl = lane - 24; D[dgl * 8 + dgl] -= D[dgl * 8 + c] * D[dgl * 8 + c]; }
-        __syncwarp();
+        a[c][c] = piv * rs;
+        rd[8 * J + c] = rs;
+#pragma unroll
+        for (int l = c + 1; l < 8; ++l) a[l][c] *= rs;
+#pragma unroll
+        for (int l = c + 1; l < 8; ++l)
+#pragma unroll
+          for (int m = c + 1; m <= l; ++m) a[l][m] -= a[l][c] * a[m][c];
       }
+#pragma unroll
+      for (int l = 0; l < 8; ++l)
+#pragma unroll
+        for (int m = 0; m <= l; ++m) D[l * 8 + m] = a[l][m];
     }
     __syncthreads();
     // tiles below the diagonal tile: row i of tile (I, J) <- row * L_JJ^-T
@@ -139,9 +148,17 @@ __device__ __forceinline__ double gram_entry(const ReqPlan& rp, const double* __
                                              int i, int j) {
   const int ntile = (rp.m + sub::kTile - 1) / sub::kTile;
   const double* src = partial + (size_t)rp.ptile_off * kTriMax + tri_index(i, j);
-  double s = 0.0;
-  for (int t = 0; t < ntile; ++t) s += src[(size_t)t * kTriMax];
-  return s;
+  // four independent loads in flight; the summation order is fixed (tile order within each of the
+  // four interleaved partial sums, then a fixed combination), so the result is deterministic
+  double s0 = 0.0, s1 = 0.0, s2 = 0.0, s3 = 0.0;
+  int t = 0;
+  for (; t + 4 <= ntile; t += 4) {
+    double a = src[(size_t)t * kTriMax], b = src[(size_t)(t + 1) * kTriMax];
+    double c = src[(size_t)(t + 2) * kTriMax], d = src[(size_t)(t + 3) * kTriMax];
+    s0 += a; s1 += b; s2 += c; s3 += d;
+  }
+  for (; t < ntile; ++t) s0 += src[(size_t)t * kTriMax];
+  return (s0 + s1) + (s2 + s3);
 }
 
 // Bytes of shared memory cholesky_blocked needs for an n x n matrix.
@@ -176,8 +193,8 @@ chol_kernel(const ReqPlan* __restrict__ plan, const double* __restrict__ partial
   cholesky_blocked(p, sm_d, sm_d + (size_t)nb * (nb + 1) / 2 * 64, load, store);
 }
 
-// One-sided Jacobi on the w columns C[c * ldc + row] (w <= 16 * ROWS): rotate column pairs until
-// they are mutually orthogonal.  Round-robin ordering, w/2 disjoint pairs per round, one 16-lane
+// One-sided Jacobi on the w columns C[c * ldc + row] (w <= 8 * ROWS): rotate column pairs until
+// they are mutually orthogonal.  Round-robin ordering, w/2 disjoint pairs per round, one 8-lane
 // group per pair, the two columns held in registers between the inner products and the rotation.
 // A pair is left alone when its inner product g is negligible against the two norms
 // (g^2 <= 1e-12 |a|^2 |b|^2) or so small that the energies move by less than ~2e-5 of the
@@ -187,7 +204,7 @@ template <int ROWS>
 __device__ __forceinline__ bool jacobi_sweeps(float* C, int ldc, int w, float s1, int max_sweeps) {
   const int tid = threadIdx.x, nt = blockDim.x;
   const int np = (w + 1) & ~1, half = np >> 1;
-  const int g = tid >> 4, gl = tid & 15, ng = nt >> 4;
+  const int g = tid >> 3, gl = tid & 7, ng = nt >> 3;
   const float abs2 = (2e-5f * s1) * (2e-5f * s1);
   bool converged = w < 2;
   for (int sweep = 0; sweep < max_sweeps && !converged; ++sweep) {
@@ -210,14 +227,14 @@ __device__ __forceinline__ bool jacobi_sweeps(float* C, int ldc, int w, float s1
         float al = 0.f, be = 0.f, ga = 0.f;
 #pragma unroll
         for (int q = 0; q < ROWS; ++q) {
-          int row = gl + 16 * q;
+          int row = gl + 8 * q;
           bool in = active && row < w;
           xa[q] = in ? ca[row] : 0.f;
           xb[q] = in ? cb[row] : 0.f;
           al += xa[q] * xa[q]; be += xb[q] * xb[q]; ga += xa[q] * xb[q];
         }
 #pragma unroll
-        for (int o = 8; o > 0; o >>= 1) {
+        for (int o = 4; o > 0; o >>= 1) {
           al += __shfl_xor_sync(0xffffffffu, al, o);
           be += __shfl_xor_sync(0xffffffffu, be, o);
           ga += __shfl_xor_sync(0xffffffffu, ga, o);
@@ -232,7 +249,7 @@ __device__ __forceinline__ bool jacobi_sweeps(float* C, int ldc, int w, float s1
           float c = rsqrtf(t * t + 1.f), sn = t * c;
 #pragma unroll
           for (int q = 0; q < ROWS; ++q) {
-            int row = gl + 16 * q;
+            int row = gl + 8 * q;
             if (row < w) {
               ca[row] = c * xa[q] - sn * xb[q];
               cb[row] = sn * xa[q] + c * xb[q];
@@ -284,9 +301,9 @@ ritz_kernel(const ReqPlan* __restrict__ plan, const double* __restrict__ partial
   __syncthreads();
   const float s1 = sqrtf(s_scale);
   bool converged;
-  if (w <= 64) converged = jacobi_sweeps<4>(C, ldc, w, s1, max_sweeps);
-  else if (w <= 128) converged = jacobi_sweeps<8>(C, ldc, w, s1, max_sweeps);
-  else converged = jacobi_sweeps<(kPMax + 15) / 16>(C, ldc, w, s1, max_sweeps);
+  if (w <= 64) converged = jacobi_sweeps<8>(C, ldc, w, s1, max_sweeps);
+  else if (w <= 128) converged = jacobi_sweeps<16>(C, ldc, w, s1, max_sweeps);
+  else converged = jacobi_sweeps<(kPMax + 7) / 8>(C, ldc, w, s1, max_sweeps);
   if (!converged && tid == 0) atomicOr(status, kStatusNoConverge);
   // singular values = column norms
   for (int k = tid >> 5; k < w; k += nt >> 5) {
@@ -315,73 +332,60 @@ ritz_kernel(const ReqPlan* __restrict__ plan, const double* __restrict__ partial
   }
 }
 
-// Eq. 15 for the preselected tokens (see the file comment).  grid = (ceil(max M / 128), batch),
-// 256 threads.  yq / yn: float32 blocks before and after the last power step, [sum M_b, kPMax].
-// Requests without stage 2 get zeros.
-// Dynamic shared memory: kLbufStride floats + p_max * kXsLd floats + win_max * nbot_max floats.
+// Eq. 15 for the preselected tokens (see the file comment).  grid = (ceil(max M / 64), batch),
+// 256 threads, one warp per token.  q / yn: the orthonormal basis Q (rows) and the block Y' = G Q^T,
+// float32 [sum M_b, kPMax].  Requests without stage 2 get zeros.
+// Dynamic shared memory: win_max * nbot_max floats.
 __global__ void __launch_bounds__(256)
-energy_kernel(const ReqPlan* __restrict__ plan, const float* __restrict__ yq,
-              const float* __restrict__ yn, const float* __restrict__ lbuf,
-              const float* __restrict__ ub, int p_max, float* __restrict__ energy) {
+energy_kernel(const ReqPlan* __restrict__ plan, const float* __restrict__ q,
+              const float* __restrict__ yn, const float* __restrict__ ub, float* __restrict__ energy) {
   extern __shared__ float sm_f[];
   ReqPlan rp = plan[blockIdx.y];
-  const int row0 = blockIdx.x * sub::kTile;
+  const int row0 = blockIdx.x * 64;
   if (row0 >= rp.m) return;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int nrows = min(sub::kTile, rp.m - row0);
+  const int nrows = min(64, rp.m - row0);
   if (!rp.stage2) {
     for (int i = tid; i < nrows; i += blockDim.x) energy[rp.presel_off + row0 + i] = 0.f;
     return;
   }
-  const int p = rp.p, P = (p + 7) & ~7, w = rp.win, w0 = p - w, nbot = p - rp.r;
-  float* lt = sm_f;
-  float* dinv = lt + kLtFloats;
-  float* xs = lt + kLbufStride;                         // [P][kXsLd]: Y rows, then Q rows in place
-  float* us = xs + (size_t)p_max * kXsLd;               // [w][nbot]
-  {
-    const float4* src = reinterpret_cast<const float4*>(lbuf + (size_t)blockIdx.y * kLbufStride);
-    float4* dst = reinterpret_cast<float4*>(lt);
-    int n4 = (lt_row_offset(P, P) + 3) / 4;
-    for (int e = tid; e < n4; e += blockDim.x) dst[e] = src[e];
-    const float* dsrc = lbuf + (size_t)blockIdx.y * kLbufStride + kLtFloats;
-    for (int e = tid; e < P; e += blockDim.x) dinv[e] = dsrc[e];
-    const float* usrc = ub + (size_t)blockIdx.y * kPMax * kPMax;
-    for (int e = tid; e < w * nbot; e += blockDim.x) us[e] = usrc[e];
-    // previous block, transposed into xs[c][row]; rows beyond the tile and columns beyond p are 0
-    for (int e = tid; e < sub::kTile * P; e += blockDim.x) {
-      int rr = e / P, c = e - rr * P;
-      xs[c * kXsLd + rr] = (rr < nrows && c < p) ? yq[((size_t)rp.presel_off + row0 + rr) * kPMax + c] : 0.f;
-    }
-  }
+  const int p = rp.p, w = rp.win, w0 = p - w, nbot = p - rp.r;
+  float* us = sm_f;                                     // [w][nbot]
+  const float* usrc = ub + (size_t)blockIdx.y * kPMax * kPMax;
+  for (int e = tid; e < w * nbot; e += blockDim.x) us[e] = usrc[e];
   __syncthreads();
-  // Q row = Y row * L^-T, one thread per row, in place
-  if (tid < sub::kTile) {
-    for (int jb = 0; jb < P; jb += 8) {
-      float acc[8];
-#pragma unroll
-      for (int e = 0; e < 8; ++e) acc[e] = xs[(jb + e) * kXsLd + tid];
-      sub::solve_block8(acc, jb, sub::smem_u32(lt), sub::smem_u32(dinv), sub::smem_u32(xs), tid, P);
-#pragma unroll
-      for (int e = 0; e < 8; ++e) xs[(jb + e) * kXsLd + tid] = acc[e];
-    }
-  }
-  __syncthreads();
-  // one warp per row: total = sum_j Y'_ij Q_ij, minus the discarded Ritz pairs of the window
   for (int rr = warp; rr < nrows; rr += 8) {
     const float* yrow = yn + ((size_t)rp.presel_off + row0 + rr) * kPMax;
+    const float* qrow = q + ((size_t)rp.presel_off + row0 + rr) * kPMax;
+    // total over all p basis vectors; the window part of both rows stays in registers
     float total = 0.f;
-    for (int c = lane; c < p; c += 32) total += yrow[c] * xs[c * kXsLd + rr];
+    float yw[(kPMax + 31) / 32], qw[(kPMax + 31) / 32];
+#pragma unroll
+    for (int t = 0; t < (kPMax + 31) / 32; ++t) {
+      int c = lane + 32 * t;
+      float yv = c < p ? yrow[c] : 0.f, qv = c < p ? qrow[c] : 0.f;
+      total += yv * qv;
+      yw[t] = yv; qw[t] = qv;
+    }
     total = warp_sum(total);
+    // discarded Ritz pairs: lanes over k, window components broadcast from the owning lane
     float sub_ = 0.f;
     for (int k0 = 0; k0 < nbot; k0 += 32) {
       int k = k0 + lane;
       float ya = 0.f, qa = 0.f;
-      if (k < nbot)
-        for (int j = 0; j < w; ++j) {
-          float u = us[j * nbot + k];
-          ya += yrow[w0 + j] * u;
-          qa += xs[(w0 + j) * kXsLd + rr] * u;
+#pragma unroll
+      for (int t = 0; t < (kPMax + 31) / 32; ++t) {
+        int cbase = 32 * t;
+        if (cbase + 31 < w0 || cbase >= p) continue;    // chunk entirely outside the window
+        for (int l = 0; l < 32; ++l) {
+          int c = cbase + l;
+          float yv = __shfl_sync(0xffffffffu, yw[t], l), qv = __shfl_sync(0xffffffffu, qw[t], l);
+          if (c >= w0 && c < p && k < nbot) {
+            float u = us[(c - w0) * nbot + k];
+            ya += yv * u; qa += qv * u;
+          }
         }
+      }
       sub_ += ya * qa;
     }
     sub_ = warp_sum(sub_);

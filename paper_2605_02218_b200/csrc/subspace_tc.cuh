@@ -272,7 +272,11 @@ constexpr int kPowBytesA = kTile * kBK * 2;              // one plane of the G t
 constexpr int kPowBytesB = kPMax * kBK * 2;              // one plane of the Y tile, 20 KB
 constexpr int kPowStageBytes = 2 * kPowBytesA + 2 * kPowBytesB;   // 72 KB
 constexpr int kXsLd = kTile + 4;                         // row stride of the staged block (floats)
-constexpr int kPowSmem = kPowStages * kPowStageBytes + kLbufStride * 4 + 1024 + 1024;
+constexpr int kXsBytes = (kPMax * kXsLd * 4 + 1023) / 1024 * 1024;   // one staged block [kPMax][kXsLd] of float32
+// The ring is followed by padding up to two staged blocks: after the MMAs the region holds the new
+// block, and either the previous block (last step) or the float64 slabs of the Gram accumulation.
+constexpr int kPowRegion = 2 * kXsBytes > kPowStages * kPowStageBytes ? 2 * kXsBytes : kPowStages * kPowStageBytes;
+constexpr int kPowSmem = kPowRegion + kLbufStride * 4 + 1024 + 1024;
 constexpr int kPowTmemCols = 256;
 constexpr int kPowThreads = 320;                         // 8 epilogue warps, TMA producer, MMA issuer
 static_assert(kPMax * kXsLd * 4 <= kPowStages * kPowStageBytes, "staged block must fit in the ring");
@@ -287,6 +291,8 @@ struct PowerParams {
   __nv_bfloat16* y_lo;
   int ld;
   float* yf;                // [sum M_b, kPMax] float32 copy of the new block, or nullptr
+  float* qprev;             // last step: float32 copy of the previous block Y on entry, overwritten
+                            // with the orthonormal basis Q = Y L^-T it stands for; else nullptr
   double* partial;          // [tiles][kTriMax]
   int* status;
 };
@@ -373,8 +379,7 @@ __device__ __forceinline__ void dmma_8x8x4(double& c0, double& c1, double a, dou
 constexpr int kSlabRows = 16;
 constexpr int kSlabLd = 20;                      // doubles; conflict-free fragment loads
 constexpr int kMaxTiles8 = kPMax / 8;            // 20
-constexpr int kXsBytes = (kPMax * kXsLd * 4 + 1023) / 1024 * 1024;
-static_assert(kXsBytes + 2 * kPMax * kSlabLd * 8 <= kPowStages * kPowStageBytes, "slabs must fit in the ring");
+static_assert(kXsBytes + 2 * kPMax * kSlabLd * 8 <= kPowRegion, "slabs must fit behind the staged block");
 
 // Accumulator slots of one warp: strip ta (the shorter one) uses slots 0 .. ta for tb = slot,
 // strip tz uses slots kMaxTiles8 - tb for tb = 0 .. tz; ta + tz = nb8 - 1 <= 19, so they never meet.
@@ -419,8 +424,8 @@ __device__ __forceinline__ void gram_unit_accumulate(GramAcc& acc, const double*
 #undef COVSPEC_GRAM_Z
 
 // Writes the accumulated tiles of one warp to the packed lower triangle.
-__device__ __forceinline__ void gram_unit_store(const GramAcc& acc, int ta, int tz, int p, int lane,
-                                                double* __restrict__ out) {
+__device__ __forceinline__ void gram_unit_store(const GramAcc& acc, int ta, int tz, int p, int coff,
+                                                int lane, double* __restrict__ out) {
   const int fr = lane >> 2, fk = lane & 3;
 #pragma unroll
   for (int u = 0; u <= kMaxTiles8; ++u) {
@@ -430,8 +435,8 @@ __device__ __forceinline__ void gram_unit_store(const GramAcc& acc, int ta, int 
     if (strip < 0) continue;
     int row = 8 * strip + fr, col = 8 * tb + 2 * fk;
     if (row < p) {
-      if (col <= row) out[tri_index(row, col)] = acc.a[u][0];
-      if (col + 1 <= row) out[tri_index(row, col + 1)] = acc.a[u][1];
+      if (col <= row) out[tri_index(coff + row, coff + col)] = acc.a[u][0];
+      if (col + 1 <= row) out[tri_index(coff + row, coff + col + 1)] = acc.a[u][1];
     }
   }
 }
@@ -443,7 +448,8 @@ power_tc_kernel(const __grid_constant__ CUtensorMap map_gh, const __grid_constan
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   float* xs = reinterpret_cast<float*>(smem);                       // aliases the ring after the MMAs
-  float* lt = reinterpret_cast<float*>(smem + kPowStages * kPowStageBytes);
+  float* xq = reinterpret_cast<float*>(smem + kXsBytes);            // previous block (last step)
+  float* lt = reinterpret_cast<float*>(smem + kPowRegion);
   float* dinv = lt + kLtFloats;
   uint64_t* bars = reinterpret_cast<uint64_t*>(lt + kLbufStride);
   uint64_t* full = bars;                 // [2]
@@ -579,10 +585,33 @@ power_tc_kernel(const __grid_constant__ CUtensorMap map_gh, const __grid_constan
         }
         tc_fence_before();
         mbar_arrive(acc_empty);
+      } else if (prm.qprev != nullptr) {
+        // ---- last step, warps 4-7: rows of Q = Y L^-T for the previous block Y, in place ----
+        ok = ok && mbar_wait(acc_full, n & 1u, abort_flag);      // the ring is no longer read
+        const int t4 = et - 128;
+        float* qrows = prm.qprev + ((size_t)rp.presel_off + tile * kTile) * kPMax;
+        for (int e = t4; e < kTile * P; e += 128) {
+          int rr = e / P, c = e - rr * P;
+          xq[c * kXsLd + rr] = (rr < nrows && c < p) ? qrows[(size_t)rr * kPMax + c] : 0.f;
+        }
+        named_barrier(2, 128);
+        for (int jb = 0; jb < P; jb += 8) {
+          float acc[8];
+#pragma unroll
+          for (int e = 0; e < 8; ++e) acc[e] = xq[(jb + e) * kXsLd + t4];
+          solve_block8(acc, jb, smem_u32(lt), smem_u32(dinv), smem_u32(xq), t4, P);
+#pragma unroll
+          for (int e = 0; e < 8; ++e) xq[(jb + e) * kXsLd + t4] = acc[e];
+        }
+        named_barrier(2, 128);
+        for (int e = t4; e < nrows * p; e += 128) {
+          int rr = e / p, c = e - rr * p;
+          qrows[(size_t)rr * kPMax + c] = xq[c * kXsLd + rr];
+        }
       }
       named_barrier(1, 256);                       // the staged block is complete
       // ---- bf16 planes of the new block (K-major operand of the next step): 8 positions per thread
-      {
+      if (prm.qprev == nullptr) {
         const int cols = (rp.m + kBK - 1) / kBK * kBK;
         for (int wi = et; wi < p * 16; wi += 256) {
           int c = wi >> 4, ch = wi & 15;
@@ -612,9 +641,18 @@ power_tc_kernel(const __grid_constant__ CUtensorMap map_gh, const __grid_constan
       }
       // ---- float64 partial Gram of the tile on the FP64 tensor cores ----
       {
-        const int nb8 = (p + 7) >> 3, units = (nb8 + 1) / 2, nslab = (nrows + kSlabRows - 1) / kSlabRows;
+        // The last step only feeds the Rayleigh-Ritz window: the trailing block of columns from
+        // coff on, plus the diagonal of the leading columns (the scale of the problem).
+        const int coff = prm.qprev != nullptr ? ((p - rp.win) & ~7) : 0;
+        const int pw = p - coff;
+        const int nb8 = (pw + 7) >> 3, units = (nb8 + 1) / 2, nslab = (nrows + kSlabRows - 1) / kSlabRows;
         double* slabs = reinterpret_cast<double*>(smem + kXsBytes);
         double* out = prm.partial + (size_t)item * kTriMax;
+        for (int c = et; c < coff; c += 256) {
+          double sq = 0.0;
+          for (int rr = 0; rr < nrows; ++rr) { double x = (double)xs[c * kXsLd + rr]; sq += x * x; }
+          out[tri_index(c, c)] = sq;
+        }
         for (int u0 = 0; u0 < units; u0 += 8) {
           const int unit = u0 + warp;
           const bool have = unit < units;
@@ -625,16 +663,16 @@ power_tc_kernel(const __grid_constant__ CUtensorMap map_gh, const __grid_constan
           for (int sl = 0; sl < nslab; ++sl) {
             double* slab = slabs + (sl & 1) * (kPMax * kSlabLd);
             // float32 -> float64, rows 16 sl .. 16 sl + 15 of every column (zero beyond the tile)
-            for (int e = et; e < P * kSlabRows; e += 256) {
+            for (int e = et; e < nb8 * 8 * kSlabRows; e += 256) {
               int c = e >> 4, rr = e & 15;
-              slab[c * kSlabLd + rr] = (double)xs[c * kXsLd + sl * kSlabRows + rr];
+              slab[c * kSlabLd + rr] = (double)xs[(coff + c) * kXsLd + sl * kSlabRows + rr];
             }
             named_barrier(1, 256);
             if (have) gram_unit_accumulate(acc, slab, ta, tz, lane);
             // the other buffer is refilled next; this one is reused two slabs later, after the
             // barrier of the next slab
           }
-          if (have) gram_unit_store(acc, ta, tz, p, lane, out);
+          if (have) gram_unit_store(acc, ta, tz, pw, coff, lane, out);
           named_barrier(1, 256);
         }
       }

@@ -151,9 +151,12 @@ def _xavier_heads(gen, n_heads, head_dim, d, device):
 def make_workload(name="custom", *, seed=0, dtype=torch.bfloat16, batch=1, n_vis=576,
                   n_txt=32, d=1024, n_heads=1, head_dim=128, rank=32, n_clusters=8,
                   kind="mixture", keep=None, keep_ratio=None, act_layers=4, lam=0.5,
-                  device="cpu") -> Workload:
+                  device="cpu", sizes=None) -> Workload:
     """Build one batch.  `n_vis` / `n_txt` are an int (uniform) or an inclusive (lo, hi) range
-    drawn per request.  `n_heads=0` gives the identity embedding (Wq = Wk = None)."""
+    drawn per request.  `n_heads=0` gives the identity embedding (Wq = Wk = None).  `sizes`
+    = (list of N_b, list of T_b) fixes the request sizes instead (another batch of the same shape
+    with different contents); the size draws are still consumed so that the rest of the stream
+    does not depend on it."""
     gen = torch.Generator(device=device)
     gen.manual_seed(seed)
 
@@ -165,6 +168,9 @@ def make_workload(name="custom", *, seed=0, dtype=torch.bfloat16, batch=1, n_vis
         return [int(spec)] * batch
 
     ns, ts = draw(n_vis), draw(n_txt)
+    if sizes is not None:
+        ns, ts = [int(v) for v in sizes[0]], [int(v) for v in sizes[1]]
+        assert len(ns) == batch and len(ts) == batch
     xs, qs = [], []
     hs = [[] for _ in range(act_layers + 1)] if act_layers > 0 else []
     for b in range(batch):
