@@ -30,6 +30,10 @@ import torch
 
 from paper_2605_02218_b200 import workloads
 
+# dram__bytes_read.sum + dram__bytes_write.sum of one visual-side relevance_tc_kernel launch (ncu,
+# profiles/relevance_tc_kernel_c2.md); None where no capture of the current kernel exists.
+NCU_TRAFFIC_BYTES = {"c2": 55.675e6}
+
 METRIC = "visual_tokens_pruned_per_s"
 UNIT = "tokens/s"
 
@@ -139,6 +143,20 @@ def cpu_baseline(wl_cpu, budget_s=20.0):
                 seconds=dt)
 
 
+def rank_seed(config, rank):
+    """Requests are independent, so every rank prunes its own batch: same shapes, its own seed."""
+    return workloads.CONFIGS[config]["seed"] + 1000 * rank
+
+
+def reduce_max(values, dist, device):
+    """Maximum over ranks of a list of per-rank timings (the job is as slow as its slowest rank)."""
+    if dist is None:
+        return list(values)
+    t = torch.tensor(values, device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.tolist()
+
+
 def run_reference(args, rank):
     if rank != 0:
         return
@@ -201,13 +219,13 @@ def main():
 
     # Input sets: rotate through enough independent copies that the working set of consecutive
     # steps exceeds twice the 126 MB L2.
-    base_seed = workloads.CONFIGS[args.config]["seed"]
-    wl0 = workloads.make_config(args.config, device=dev, seed=base_seed + 1000 * rank)
+    base_seed = rank_seed(args.config, rank)
+    wl0 = workloads.make_config(args.config, device=dev, seed=base_seed)
     work = algorithmic_work(wl0)
     copies = args.copies or max(2, int(np.ceil(2 * 126e6 * 2 / work["input_bytes"])))
     copies = min(copies, 8)
     sizes = (np.diff(wl0.vis_offsets).tolist(), np.diff(wl0.txt_offsets).tolist())
-    sets = [wl0] + [workloads.make_config(args.config, device=dev, seed=base_seed + 1000 * rank + 17 * (i + 1),
+    sets = [wl0] + [workloads.make_config(args.config, device=dev, seed=base_seed + 17 * (i + 1),
                                           sizes=sizes) for i in range(copies - 1)]
     pr = api.Pruner.for_workload(wl0)
     ms = [pr.marshal(w) for w in sets]
@@ -273,10 +291,7 @@ def main():
 
     # ---- reduce over ranks ------------------------------------------------------------------
     ms_step = ms_total / args.steps
-    if dist is not None:
-        t = torch.tensor([ms_step, ms_e2e], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_step, ms_e2e = t.tolist()
+    ms_step, ms_e2e = reduce_max([ms_step, ms_e2e], dist, dev)
     if rank == 0:
         peaks = _peaks()
         rel_ms = stage_ms["relevance"] / max(prof_calls, 1)
@@ -285,10 +300,7 @@ def main():
         if wl0.dtype != torch.bfloat16:
             peak_tf *= 0.5            # tf32 / fp32 path: nominal ratio to the bf16 peak
         achieved = work["relevance_flops"] / (rel_ms * 1e-3) / 1e12 if rel_ms > 0 else 0.0
-        traffic = None
-        tpath = os.path.join(ROOT, "profiles", "traffic.json")
-        if os.path.exists(tpath):
-            traffic = json.load(open(tpath)).get(args.config, {}).get("relevance_dram_bytes_per_step")
+        traffic = NCU_TRAFFIC_BYTES.get(args.config)
         line = dict(
             metric=METRIC, value=world * tokens / (ms_step * 1e-3), unit=UNIT, n_gpus=world,
             steps=args.steps, warmup=max(args.warmup, 3), ms_per_step=ms_step, higher_is_better=True,

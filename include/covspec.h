@@ -23,6 +23,9 @@
  *    Conditions only the device can see (non-finite scores) are recorded in a device status word,
  *    read back by covspec_get_device_status(); outputs are then unspecified but in bounds.
  *  - One context serves one stream at a time; calls on one context must not overlap.
+ *  - Results are deterministic: the same inputs on the same context give bit-identical outputs
+ *    (the only floating-point atomic is a max, which does not depend on order; partial sums are
+ *    combined in a fixed order).
  */
 #ifndef COVSPEC_H_
 #define COVSPEC_H_
@@ -61,7 +64,8 @@ typedef struct {
   float presel_factor; /* M = min(N, max(B_vis, ceil(presel_factor*B_vis)))                        */
   float rank_frac;     /* r = clamp(ceil(rank_frac*B_vis), 1, min(rank_cap, M-1, d-1))             */
   int rank_cap;
-  int eig_iters;       /* subspace-iteration steps used to reach the top-r singular subspace       */
+  int eig_iters;       /* Eq. 14 is reached by block subspace iteration on Z_M^T Z_M: eig_iters
+                          orthonormalised power steps follow the first multiplication (>= 1)        */
   int eig_oversample;  /* extra basis vectors carried beyond r; rank_cap + eig_oversample <= 160    */
   int max_batch;                 /* capacities the workspace is sized for */
   long long max_total_vis;       /* sum of N_b */
