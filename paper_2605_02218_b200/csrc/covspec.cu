@@ -526,9 +526,8 @@ int select_impl(covspec_ctx* ctx, const covspec_problem* p, const float* s_fused
         LAUNCH_CHECK(ctx);
       }
     }
-    size_t ritz_smem = (((size_t)pl.win_max * (pl.win_max | 1) + pl.win_max + 1) & ~(size_t)1) * sizeof(float) +
-                       cholesky_smem_bytes(pl.win_max);
-    ritz_kernel<<<B, pl.win_max <= 64 ? 256 : 512, ritz_smem, s>>>(ctx->d_plan, ctx->partial, ctx->Ub, 30, ctx->status);
+    size_t ritz_smem = ritz_smem_bytes(pl.win_max);
+    ritz_kernel<<<B, 512, ritz_smem, s>>>(ctx->d_plan, ctx->partial, ctx->Ub, 30, ctx->status);
     LAUNCH_CHECK(ctx);
   }
   dim3 ge((pl.m_max + 63) / 64, B);
@@ -700,8 +699,7 @@ int covspec_prune_init(const covspec_config* cfg, covspec_ctx** out) {
   ok = ok && cudaFuncSetAttribute(chol_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                   (int)cholesky_smem_bytes(kPMax)) == cudaSuccess;
   ok = ok && cudaFuncSetAttribute(ritz_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                  (int)(((size_t)kPMax * (kPMax | 1) + kPMax + 2) * sizeof(float) +
-                                        cholesky_smem_bytes(kPMax))) == cudaSuccess;
+                                  (int)ritz_smem_bytes(kPMax)) == cudaSuccess;
   ok = ok && cudaFuncSetAttribute(energy_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                   (int)((size_t)kPMax * kPMax * sizeof(float))) == cudaSuccess;
   int dev = 0, cc_major = 0;

@@ -193,92 +193,106 @@ chol_kernel(const ReqPlan* __restrict__ plan, const double* __restrict__ partial
   cholesky_blocked(p, sm_d, sm_d + (size_t)nb * (nb + 1) / 2 * 64, load, store);
 }
 
-// One-sided Jacobi on the w columns C[c * ldc + row] (w <= 8 * ROWS): rotate column pairs until
-// they are mutually orthogonal.  Round-robin ordering, w/2 disjoint pairs per round, one 8-lane
-// group per pair, the two columns held in registers between the inner products and the rotation.
-// A pair is left alone when its inner product g is negligible against the two norms
-// (g^2 <= 1e-12 |a|^2 |b|^2) or so small that the energies move by less than ~2e-5 of the
-// problem's scale s1 (g^2 <= (2e-5 s1)^2 min(|a|^2, |b|^2)).  Returns false when max_sweeps sweeps
-// did not reach a sweep without rotations.
+// One-sided Jacobi on the w columns C[c * ldc + row] (w <= 4 * ROWS): rotate column pairs until
+// they are mutually orthogonal.  Round-robin ordering, w/2 disjoint pairs per round, one 4-lane
+// group per pair with the two columns held in registers between the inner products and the
+// rotation, so that a round is a short instruction stream on few warps and the barrier between
+// rounds spans only those warps (named barrier 1 over `nact` threads; the caller guarantees that
+// exactly the threads tid < nact enter).  A pair is left alone when its inner product g is
+// negligible against the two norms (g^2 <= 1e-12 |a|^2 |b|^2) or so small that the energies move by
+// less than ~2e-5 of the problem's scale s1 (g^2 <= (2e-5 s1)^2 min(|a|^2, |b|^2)).  Returns false
+// when max_sweeps sweeps did not reach a sweep without rotations.
 template <int ROWS>
-__device__ __forceinline__ bool jacobi_sweeps(float* C, int ldc, int w, float s1, int max_sweeps) {
-  const int tid = threadIdx.x, nt = blockDim.x;
+__device__ __forceinline__ bool jacobi_sweeps(float* C, int ldc, int w, float s1, int max_sweeps,
+                                              int nact, volatile int* flag) {
+  const int tid = threadIdx.x;
   const int np = (w + 1) & ~1, half = np >> 1;
-  const int g = tid >> 3, gl = tid & 7, ng = nt >> 3;
+  const int g = tid >> 2, gl = tid & 3;
   const float abs2 = (2e-5f * s1) * (2e-5f * s1);
   bool converged = w < 2;
   for (int sweep = 0; sweep < max_sweeps && !converged; ++sweep) {
     int rotated = 0;
     for (int round = 0; round < np - 1; ++round) {
-      for (int base = 0; base < half; base += ng) {
-        int i = base + g;
-        int a = 0, b = 0;
-        bool active = i < half;
-        if (active) {
-          a = round + i; if (a >= np - 1) a -= np - 1;
-          b = round - i; if (b < 0) b += np - 1;
-          if (i == 0) { a = round; b = np - 1; }
-          if (a > b) { int t = a; a = b; b = t; }
-          active = b < w;
-        }
-        float* ca = C + a * ldc;
-        float* cb = C + b * ldc;
-        float xa[ROWS], xb[ROWS];
-        float al = 0.f, be = 0.f, ga = 0.f;
+      int a = 0, b = 0;
+      bool active = g < half;
+      if (active) {
+        a = round + g; if (a >= np - 1) a -= np - 1;
+        b = round - g; if (b < 0) b += np - 1;
+        if (g == 0) { a = round; b = np - 1; }
+        if (a > b) { int t = a; a = b; b = t; }
+        active = b < w;
+      }
+      float* ca = C + a * ldc;
+      float* cb = C + b * ldc;
+      float xa[ROWS], xb[ROWS];
+      float al = 0.f, be = 0.f, ga = 0.f;
+#pragma unroll
+      for (int q = 0; q < ROWS; ++q) {
+        int row = gl + 4 * q;
+        bool in = active && row < w;
+        xa[q] = in ? ca[row] : 0.f;
+        xb[q] = in ? cb[row] : 0.f;
+        al += xa[q] * xa[q]; be += xb[q] * xb[q]; ga += xa[q] * xb[q];
+      }
+#pragma unroll
+      for (int o = 2; o > 0; o >>= 1) {
+        al += __shfl_xor_sync(0xffffffffu, al, o);
+        be += __shfl_xor_sync(0xffffffffu, be, o);
+        ga += __shfl_xor_sync(0xffffffffu, ga, o);
+      }
+      float g2 = ga * ga;
+      float thr2 = fmaxf(1e-12f * al * be, abs2 * fminf(al, be));
+      if (active && g2 > thr2 && g2 > 1e-37f) {
+        // tan of the rotation angle: t = sign(d g) 2|g| / (|d| + sqrt(d^2 + 4 g^2)), d = |b|^2 - |a|^2
+        float d = be - al;
+        float t = __fdividef(2.f * ga, fabsf(d) + __fsqrt_rn(d * d + 4.f * g2));
+        if (d < 0.f) t = -t;
+        float c = rsqrtf(t * t + 1.f), sn = t * c;
 #pragma unroll
         for (int q = 0; q < ROWS; ++q) {
-          int row = gl + 8 * q;
-          bool in = active && row < w;
-          xa[q] = in ? ca[row] : 0.f;
-          xb[q] = in ? cb[row] : 0.f;
-          al += xa[q] * xa[q]; be += xb[q] * xb[q]; ga += xa[q] * xb[q];
-        }
-#pragma unroll
-        for (int o = 4; o > 0; o >>= 1) {
-          al += __shfl_xor_sync(0xffffffffu, al, o);
-          be += __shfl_xor_sync(0xffffffffu, be, o);
-          ga += __shfl_xor_sync(0xffffffffu, ga, o);
-        }
-        float g2 = ga * ga;
-        float thr2 = fmaxf(1e-12f * al * be, abs2 * fminf(al, be));
-        if (active && g2 > thr2 && g2 > 1e-37f) {
-          // tan of the rotation angle: t = sign(d g) 2|g| / (|d| + sqrt(d^2 + 4 g^2)), d = |b|^2 - |a|^2
-          float d = be - al;
-          float t = __fdividef(2.f * ga, fabsf(d) + __fsqrt_rn(d * d + 4.f * g2));
-          if (d < 0.f) t = -t;
-          float c = rsqrtf(t * t + 1.f), sn = t * c;
-#pragma unroll
-          for (int q = 0; q < ROWS; ++q) {
-            int row = gl + 8 * q;
-            if (row < w) {
-              ca[row] = c * xa[q] - sn * xb[q];
-              cb[row] = sn * xa[q] + c * xb[q];
-            }
+          int row = gl + 4 * q;
+          if (row < w) {
+            ca[row] = c * xa[q] - sn * xb[q];
+            cb[row] = sn * xa[q] + c * xb[q];
           }
-          rotated = 1;
         }
+        rotated = 1;
       }
-      __syncthreads();
+      sub::named_barrier(1, nact);
     }
-    converged = __syncthreads_or(rotated) == 0;
+    if (rotated) *flag = 1;
+    sub::named_barrier(1, nact);
+    converged = *flag == 0;
+    sub::named_barrier(1, nact);
+    if (tid == 0) *flag = 0;
+    sub::named_barrier(1, nact);
   }
   return converged;
+}
+
+// Column stride of the window factor in shared memory: >= w and congruent to 4 modulo 32, so that
+// the eight 4-lane groups of a warp, which hold consecutive columns, hit distinct banks.
+__host__ __device__ inline int ritz_ldc(int w) { return (w + 27) / 32 * 32 + 4; }
+// Bytes of dynamic shared memory of ritz_kernel for a window of w vectors.
+__host__ __device__ inline size_t ritz_smem_bytes(int w) {
+  return ((((size_t)w * ritz_ldc(w) + w + 1) & ~(size_t)1)) * sizeof(float) + cholesky_smem_bytes(w);
 }
 
 // Rayleigh-Ritz on the trailing window (see the file comment).  One block of 512 threads per
 // request.  Output ub[j * nbot + k]: component j (window coordinates) of the unit eigenvector of
 // the k-th smallest Ritz value, k < nbot = p - r.
-// Dynamic shared memory: round_up(win * (win | 1) + win, 2) floats, then cholesky_smem_bytes(win).
+// Dynamic shared memory: ritz_smem_bytes(win_max).
 __global__ void __launch_bounds__(512)
 ritz_kernel(const ReqPlan* __restrict__ plan, const double* __restrict__ partial,
             float* __restrict__ ub, int max_sweeps, int* status) {
   extern __shared__ float sm_f[];
   __shared__ float s_scale;
+  __shared__ int s_flag;
   ReqPlan rp = plan[blockIdx.x];
   if (!rp.stage2) return;
   const int p = rp.p, w = rp.win, w0 = p - w, nbot = p - rp.r;
   const int tid = threadIdx.x, nt = blockDim.x;
-  const int ldc = w | 1;
+  const int ldc = ritz_ldc(w);
   float* C = sm_f;                                  // columns of the factor: C[c * ldc + row]
   float* sig = C + (size_t)w * ldc;                 // [w] column norms at the end
   for (int e = tid; e < w * ldc; e += nt) C[e] = 0.f;
@@ -300,11 +314,18 @@ ritz_kernel(const ReqPlan* __restrict__ plan, const double* __restrict__ partial
   }
   __syncthreads();
   const float s1 = sqrtf(s_scale);
-  bool converged;
-  if (w <= 64) converged = jacobi_sweeps<8>(C, ldc, w, s1, max_sweeps);
-  else if (w <= 128) converged = jacobi_sweeps<16>(C, ldc, w, s1, max_sweeps);
-  else converged = jacobi_sweeps<(kPMax + 7) / 8>(C, ldc, w, s1, max_sweeps);
-  if (!converged && tid == 0) atomicOr(status, kStatusNoConverge);
+  // the rotations run on the first 4 * (pairs per round) threads (whole warps); the rest wait
+  const int nact = min(nt, ((((w + 1) >> 1) * 4) + 31) & ~31);
+  if (tid == 0) s_flag = 0;
+  __syncthreads();
+  if (tid < nact) {
+    bool converged;
+    if (w <= 64) converged = jacobi_sweeps<16>(C, ldc, w, s1, max_sweeps, nact, &s_flag);
+    else if (w <= 96) converged = jacobi_sweeps<24>(C, ldc, w, s1, max_sweeps, nact, &s_flag);
+    else converged = jacobi_sweeps<(kPMax + 3) / 4>(C, ldc, w, s1, max_sweeps, nact, &s_flag);
+    if (!converged && tid == 0) atomicOr(status, kStatusNoConverge);
+  }
+  __syncthreads();
   // singular values = column norms
   for (int k = tid >> 5; k < w; k += nt >> 5) {
     float s = 0.f;
