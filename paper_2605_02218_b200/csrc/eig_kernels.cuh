@@ -49,7 +49,8 @@ __device__ __forceinline__ double rsqrt_f64(double x) {
 // 8 x 8 tiles of its lower triangle (tile (I, J <= I) at T + tri_index(I, J) * 64, row-major).
 // Per 8-column panel: the diagonal tile is factored by one thread in registers, the tiles below it are solved one
 // row per thread, and the trailing tiles take their rank-8 update on the FP64 tensor cores
-// (two m8n8k4 instructions per tile).  Three __syncthreads per panel.
+// (two m8n8k4 instructions per tile); the next panel's diagonal tile is factored while the rest of
+// the trailing matrix is still being updated.  Three __syncthreads per panel.
 // A pivot below 1e-12 of its original diagonal entry (a numerically dependent direction) is
 // clamped there; the next multiplication by G restores the direction.
 //   load(i, j)         value of entry (i, j), i >= j
@@ -61,47 +62,72 @@ __device__ __forceinline__ void cholesky_blocked(int n, double* T, double* aux, 
   const int nb = (n + 7) >> 3, ntile = nb * (nb + 1) / 2;
   double* d0 = aux;                 // original diagonal
   double* rd = aux + 8 * nb;        // 1 / L[j][j]
-  for (int e = tid; e < ntile * 64; e += nt) {
-    int I, J;
-    sub::tri_decode(e >> 6, I, J);
-    int i = 8 * I + ((e >> 3) & 7), j = 8 * J + (e & 7);
-    double v;
-    if (i < n && j < n) v = j <= i ? load(i, j) : load(j, i);
-    else v = i == j ? 1.0 : 0.0;
-    T[e] = v;
-    if (i == j) d0[i] = v;
+  // four entries per thread and trip, so that their global loads overlap
+  for (int e0 = tid; e0 < ntile * 64; e0 += 4 * nt) {
+    double v[4];
+    int ii[4], jj[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      int e = e0 + u * nt, I = 0, J = 0;
+      if (e < ntile * 64) sub::tri_decode(e >> 6, I, J);
+      ii[u] = 8 * I + ((e >> 3) & 7); jj[u] = 8 * J + (e & 7);
+      if (e >= ntile * 64) v[u] = 0.0;
+      else if (ii[u] < n && jj[u] < n) v[u] = jj[u] <= ii[u] ? load(ii[u], jj[u]) : load(jj[u], ii[u]);
+      else v[u] = ii[u] == jj[u] ? 1.0 : 0.0;
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      int e = e0 + u * nt;
+      if (e < ntile * 64) {
+        T[e] = v[u];
+        if (ii[u] == jj[u]) d0[ii[u]] = v[u];
+      }
+    }
   }
   __syncthreads();
-  for (int J = 0; J < nb; ++J) {
+  // factor the diagonal tile (J, J) in registers: one thread; the chain of eight dependent
+  // reciprocal square roots is the critical path of the whole factorisation
+  auto factor_diag = [&](int J) {
     double* D = T + tri_index(J, J) * 64;
-    if (tid == 0) {
-      // 8 x 8 diagonal tile: one thread, everything in registers (the chain of eight dependent
-      // reciprocal square roots is the critical path of the whole factorisation)
-      double a[8][8];
+    double a[8][8];
 #pragma unroll
-      for (int l = 0; l < 8; ++l)
+    for (int l = 0; l < 8; ++l)
 #pragma unroll
-        for (int m = 0; m <= l; ++m) a[l][m] = D[l * 8 + m];
+      for (int m = 0; m <= l; ++m) a[l][m] = D[l * 8 + m];
 #pragma unroll
-      for (int c = 0; c < 8; ++c) {
-        double piv = a[c][c], floor_ = 1e-12 * d0[8 * J + c];
-        if (!(piv > floor_)) piv = floor_ > 0.0 ? floor_ : 1.0;
-        double rs = rsqrt_f64(piv);
-        a[c][c] = piv * rs;
-        rd[8 * J + c] = rs;
+    for (int c = 0; c < 8; ++c) {
+      double piv = a[c][c], floor_ = 1e-12 * d0[8 * J + c];
+      if (!(piv > floor_)) piv = floor_ > 0.0 ? floor_ : 1.0;
+      double rs = rsqrt_f64(piv);
+      a[c][c] = piv * rs;
+      rd[8 * J + c] = rs;
 #pragma unroll
-        for (int l = c + 1; l < 8; ++l) a[l][c] *= rs;
+      for (int l = c + 1; l < 8; ++l) a[l][c] *= rs;
 #pragma unroll
-        for (int l = c + 1; l < 8; ++l)
+      for (int l = c + 1; l < 8; ++l)
 #pragma unroll
-          for (int m = c + 1; m <= l; ++m) a[l][m] -= a[l][c] * a[m][c];
-      }
-#pragma unroll
-      for (int l = 0; l < 8; ++l)
-#pragma unroll
-        for (int m = 0; m <= l; ++m) D[l * 8 + m] = a[l][m];
+        for (int m = c + 1; m <= l; ++m) a[l][m] -= a[l][c] * a[m][c];
     }
-    __syncthreads();
+#pragma unroll
+    for (int l = 0; l < 8; ++l)
+#pragma unroll
+      for (int m = 0; m <= l; ++m) D[l * 8 + m] = a[l][m];
+  };
+  // C(I, K) -= X_I X_K^T for one trailing tile of panel J (rank-8 update, two tensor-core instructions)
+  const int fr = lane >> 2, fk = lane & 3;
+  auto update_tile = [&](int J, int I, int K) {
+    const double* XI = T + tri_index(I, J) * 64 + fr * 8 + fk;
+    const double* XK = T + tri_index(K, J) * 64 + fr * 8 + fk;
+    double* C = T + tri_index(I, K) * 64 + fr * 8 + 2 * fk;
+    double c0 = C[0], c1 = C[1];
+    sub::dmma_8x8x4(c0, c1, -XI[0], XK[0]);
+    sub::dmma_8x8x4(c0, c1, -XI[4], XK[4]);
+    C[0] = c0; C[1] = c1;
+  };
+  if (tid == 0) factor_diag(0);
+  __syncthreads();
+  for (int J = 0; J < nb; ++J) {
+    const double* D = T + tri_index(J, J) * 64;
     // tiles below the diagonal tile: row i of tile (I, J) <- row * L_JJ^-T
     for (int i = 8 * (J + 1) + tid; i < 8 * nb; i += nt) {
       double* row = T + tri_index(i >> 3, J) * 64 + (i & 7) * 8;
@@ -119,19 +145,22 @@ __device__ __forceinline__ void cholesky_blocked(int n, double* T, double* aux, 
       for (int c = 0; c < 8; ++c) row[c] = x[c];
     }
     __syncthreads();
-    // trailing tiles (I, K), J < K <= I: C -= X_I X_K^T
-    const int mrem = nb - J - 1, ntr = mrem * (mrem + 1) / 2;
-    const int fr = lane >> 2, fk = lane & 3;
-    for (int q = warp; q < ntr; q += nw) {
-      int ii, kk;
-      sub::tri_decode(q, ii, kk);
-      const double* XI = T + tri_index(J + 1 + ii, J) * 64 + fr * 8 + fk;
-      const double* XK = T + tri_index(J + 1 + kk, J) * 64 + fr * 8 + fk;
-      double* C = T + tri_index(J + 1 + ii, J + 1 + kk) * 64 + fr * 8 + 2 * fk;
-      double c0 = C[0], c1 = C[1];
-      sub::dmma_8x8x4(c0, c1, -XI[0], XK[0]);
-      sub::dmma_8x8x4(c0, c1, -XI[4], XK[4]);
-      C[0] = c0; C[1] = c1;
+    if (J + 1 == nb) break;
+    // look-ahead: the tiles of column J+1 take their update first ...
+    for (int I = J + 1 + warp; I < nb; I += nw) update_tile(J, I, J + 1);
+    __syncthreads();
+    // ... so that its diagonal tile is factored (warp 0, one thread) while the other warps update
+    // the rest of the trailing matrix, tiles (I, K) with J+1 < K <= I
+    if (warp == 0) {
+      if (lane == 0) factor_diag(J + 1);
+      __syncwarp();
+    } else {
+      const int mrem = nb - J - 2, ntr = mrem * (mrem + 1) / 2;
+      for (int q = warp - 1; q < ntr; q += nw - 1) {
+        int ii, kk;
+        sub::tri_decode(q, ii, kk);
+        update_tile(J, J + 2 + ii, J + 2 + kk);
+      }
     }
     __syncthreads();
   }

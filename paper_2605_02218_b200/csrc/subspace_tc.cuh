@@ -590,9 +590,17 @@ power_tc_kernel(const __grid_constant__ CUtensorMap map_gh, const __grid_constan
         ok = ok && mbar_wait(acc_full, n & 1u, abort_flag);      // the ring is no longer read
         const int t4 = et - 128;
         float* qrows = prm.qprev + ((size_t)rp.presel_off + tile * kTile) * kPMax;
-        for (int e = t4; e < kTile * P; e += 128) {
-          int rr = e / P, c = e - rr * P;
-          xq[c * kXsLd + rr] = (rr < nrows && c < p) ? qrows[(size_t)rr * kPMax + c] : 0.f;
+        // thread = column (two columns when P > 128), eight rows per trip so that the loads overlap
+        for (int c = t4; c < P; c += 128) {
+#pragma unroll 1
+          for (int r0 = 0; r0 < kTile; r0 += 8) {
+            float v[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u)
+              v[u] = (r0 + u < nrows && c < p) ? qrows[(size_t)(r0 + u) * kPMax + c] : 0.f;
+#pragma unroll
+            for (int u = 0; u < 8; ++u) xq[c * kXsLd + r0 + u] = v[u];
+          }
         }
         named_barrier(2, 128);
         for (int jb = 0; jb < P; jb += 8) {
@@ -604,10 +612,8 @@ power_tc_kernel(const __grid_constant__ CUtensorMap map_gh, const __grid_constan
           for (int e = 0; e < 8; ++e) xq[(jb + e) * kXsLd + t4] = acc[e];
         }
         named_barrier(2, 128);
-        for (int e = t4; e < nrows * p; e += 128) {
-          int rr = e / p, c = e - rr * p;
-          qrows[(size_t)rr * kPMax + c] = xq[c * kXsLd + rr];
-        }
+        for (int c = t4; c < p; c += 128)
+          for (int rr = 0; rr < nrows; ++rr) qrows[(size_t)rr * kPMax + c] = xq[c * kXsLd + rr];
       }
       named_barrier(1, 256);                       // the staged block is complete
       // ---- bf16 planes of the new block (K-major operand of the next step): 8 positions per thread
@@ -634,10 +640,9 @@ power_tc_kernel(const __grid_constant__ CUtensorMap map_gh, const __grid_constan
       }
       if (prm.yf != nullptr) {
         // float32 block, one token per row; consecutive threads write consecutive columns
-        for (int e = et; e < nrows * p; e += 256) {
-          int rr = e / p, c = e - rr * p;
-          prm.yf[((size_t)rp.presel_off + tile * kTile + rr) * kPMax + c] = xs[c * kXsLd + rr];
-        }
+        float* yrows = prm.yf + ((size_t)rp.presel_off + tile * kTile) * kPMax;
+        for (int c = et & 127; c < p; c += 128)
+          for (int rr = et >> 7; rr < nrows; rr += 2) yrows[(size_t)rr * kPMax + c] = xs[c * kXsLd + rr];
       }
       // ---- float64 partial Gram of the tile on the FP64 tensor cores ----
       {
