@@ -60,6 +60,8 @@ struct Plan {
   int t_max = 0, p_max = 0, m_max = 0, win_max = 0, nbot_max = 0;
   int n_tiles = 0;                            // 128-token tiles over all requests
   int n_gram_tiles = 0, n_ptiles = 0;         // lower-triangle Gram tiles / 128-row block tiles (stage 2)
+  int pow_grid = 0;                           // CTAs of the power step
+  std::vector<int> sched;                     // [pow_grid + 1] offsets + item lists (longest first)
   long long total_vis = 0, total_txt = 0, total_keep = 0, total_presel = 0;
   bool valid = false;
 };
@@ -75,6 +77,7 @@ struct covspec_ctx {
   // carved regions
   int* status = nullptr;
   ReqPlan* d_plan = nullptr;
+  int* d_sched = nullptr;                // power-step schedule: [grid + 1] offsets + item lists
   GemmProb* d_tables = nullptr;          // [T_COUNT][max_batch]
   float* Qn = nullptr;
   float* Kp = nullptr;
@@ -96,7 +99,7 @@ struct covspec_ctx {
   CUtensorMap map_zg, map_gh, map_gl, map_y[2][2];
   // pinned staging for the plan upload
   char* h_stage = nullptr;
-  long long stage_bytes = 0;
+  long long stage_bytes = 0, stage_sched_off = 0;
   cudaEvent_t stage_free = nullptr;      // the previous upload has been consumed
   Plan plan;
   int num_sms = 148;
@@ -232,6 +235,40 @@ int get_plan(covspec_ctx* ctx, const covspec_problem* p, cudaStream_t stream) {
       pl.total_presel > ctx->cfg.max_total_presel || pl.n_ptiles > ctx->cap_ptiles)
     return COVSPEC_ERR_WORKSPACE;
 
+  // Schedule of the power step: its items differ in cost (basis size p, rows in the tile), so they
+  // are handed to the CTAs longest first, each to the least loaded CTA.
+  pl.pow_grid = std::min(pl.n_ptiles, ctx->num_sms);
+  pl.sched.assign((size_t)pl.pow_grid + 1 + pl.n_ptiles, 0);
+  if (pl.n_ptiles > 0) {
+    std::vector<std::pair<double, int>> items;
+    for (int b = 0; b < B; ++b) {
+      const ReqPlan& r = pl.req[b];
+      if (!r.stage2) continue;
+      int nt = (r.m + sub::kTile - 1) / sub::kTile;
+      for (int t = 0; t < nt; ++t) {
+        int rows = std::min(sub::kTile, r.m - t * sub::kTile);
+        double pp = (double)r.p;
+        items.push_back({pp * pp * (1.0 + 1.5 * rows / sub::kTile) + 64.0 * r.m, r.ptile_off + t});
+      }
+    }
+    std::stable_sort(items.begin(), items.end(), [](const std::pair<double, int>& a, const std::pair<double, int>& b2) { return a.first > b2.first; });
+    std::vector<double> load(pl.pow_grid, 0.0);
+    std::vector<std::vector<int>> lists(pl.pow_grid);
+    for (const auto& it : items) {
+      int best = 0;
+      for (int g = 1; g < pl.pow_grid; ++g) if (load[g] < load[best]) best = g;
+      load[best] += it.first;
+      lists[best].push_back(it.second);
+    }
+    int off = 0;
+    int* items_out = pl.sched.data() + pl.pow_grid + 1;
+    for (int g = 0; g < pl.pow_grid; ++g) {
+      pl.sched[g] = off;
+      for (int v : lists[g]) items_out[off++] = v;
+    }
+    pl.sched[pl.pow_grid] = off;
+  }
+
   // Stage plan + gemm table in pinned memory and upload.
   if (ctx->stage_free) CUDA_TRY(cudaEventSynchronize(ctx->stage_free));
   ReqPlan* h_plan = reinterpret_cast<ReqPlan*>(ctx->h_stage);
@@ -259,6 +296,11 @@ int get_plan(covspec_ctx* ctx, const covspec_problem* p, cudaStream_t stream) {
   if (s2 > 0)
     CUDA_TRY(cudaMemcpyAsync(ctx->d_tables, h_tab, sizeof(GemmProb) * (size_t)T_COUNT * mb,
                              cudaMemcpyHostToDevice, stream));
+  if (pl.n_ptiles > 0) {
+    int* h_sched = reinterpret_cast<int*>(ctx->h_stage + ctx->stage_sched_off);
+    memcpy(h_sched, pl.sched.data(), sizeof(int) * pl.sched.size());
+    CUDA_TRY(cudaMemcpyAsync(ctx->d_sched, h_sched, sizeof(int) * pl.sched.size(), cudaMemcpyHostToDevice, stream));
+  }
   CUDA_TRY(cudaEventRecord(ctx->stage_free, stream));
   pl.valid = true;
   return COVSPEC_OK;
@@ -506,10 +548,10 @@ int select_impl(covspec_ctx* ctx, const covspec_problem* p, const float* s_fused
     sub::basis_init_kernel<<<gb, 256, 0, s>>>(ctx->d_plan, ctx->Yp[0][0], ctx->Yp[0][1], ctx->Yp[1][0],
                                               ctx->Yp[1][1], ctx->ld);
     LAUNCH_CHECK(ctx);
-    int grid = std::min(pl.n_ptiles, ctx->num_sms);
+    int grid = pl.pow_grid;
     for (int pass = 0; pass <= cfg.eig_iters; ++pass) {
       sub::PowerParams pp{};
-      pp.plan = ctx->d_plan; pp.batch = B; pp.n_items = pl.n_ptiles;
+      pp.plan = ctx->d_plan; pp.batch = B; pp.n_items = pl.n_ptiles; pp.sched = ctx->d_sched;
       pp.identity = pass == 0;
       pp.lbuf = ctx->Lbuf;
       int in = pass & 1, out = in ^ 1;
@@ -645,6 +687,8 @@ int covspec_prune_init(const covspec_config* cfg, covspec_ctx** out) {
   long long o_status = carve(256);
   long long o_plan = carve(sizeof(ReqPlan) * c.max_batch);
   long long o_tab = carve(sizeof(GemmProb) * (long long)T_COUNT * c.max_batch);
+  long long sched_ints = 1024 + ctx->cap_ptiles;   // offsets of up to 1023 CTAs + one entry per tile
+  long long o_sched = carve(4 * sched_ints);
   long long o_qn = carve(4ll * c.max_total_txt * ctx->P);
   long long o_kp = carve(4ll * ctx->kp_rows * ctx->P);
   long long o_sq = carve(4ll * c.max_total_vis), o_sa = carve(4ll * c.max_total_vis);
@@ -672,6 +716,7 @@ int covspec_prune_init(const covspec_config* cfg, covspec_ctx** out) {
   ctx->status = reinterpret_cast<int*>(w + o_status);
   ctx->d_plan = reinterpret_cast<ReqPlan*>(w + o_plan);
   ctx->d_tables = reinterpret_cast<GemmProb*>(w + o_tab);
+  ctx->d_sched = reinterpret_cast<int*>(w + o_sched);
   ctx->Qn = reinterpret_cast<float*>(w + o_qn);
   ctx->Kp = reinterpret_cast<float*>(w + o_kp);
   ctx->sq = reinterpret_cast<float*>(w + o_sq);
@@ -692,6 +737,8 @@ int covspec_prune_init(const covspec_config* cfg, covspec_ctx** out) {
   ctx->Ub = reinterpret_cast<float*>(w + o_ub);
   ctx->stage_bytes = round_up(sizeof(ReqPlan) * c.max_batch, 256) +
                      sizeof(GemmProb) * (long long)T_COUNT * c.max_batch;
+  ctx->stage_sched_off = round_up(ctx->stage_bytes, 256);
+  ctx->stage_bytes = ctx->stage_sched_off + 4 * sched_ints;
   bool ok = cudaMemset(ctx->status, 0, 256) == cudaSuccess &&
             cudaMallocHost(&ctx->h_stage, (size_t)ctx->stage_bytes) == cudaSuccess &&
             cudaEventCreateWithFlags(&ctx->stage_free, cudaEventDisableTiming) == cudaSuccess;

@@ -285,6 +285,8 @@ struct PowerParams {
   const ReqPlan* plan;
   int batch;
   int n_items;              // 128-row tiles over all stage-2 requests
+  const int* sched;         // [gridDim.x + 1] offsets, then the item lists of every CTA (longest
+                            // items first, balanced on the host)
   int identity;             // first step: no triangular factor yet
   const float* lbuf;        // [batch][kLbufStride] triangular factor + reciprocal diagonal
   __nv_bfloat16* y_hi;      // output planes
@@ -475,6 +477,8 @@ power_tc_kernel(const __grid_constant__ CUtensorMap map_gh, const __grid_constan
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
+  const int s_begin = prm.sched[blockIdx.x], s_end = prm.sched[blockIdx.x + 1];
+  const int* s_items = prm.sched + gridDim.x + 1;
   auto decode = [&](int item, int& b, ReqPlan& rp, int& tile) {
     b = find_request(item, prm.batch, [&](int q) { return prm.plan[q].ptile_off; });
     rp = prm.plan[b];
@@ -485,7 +489,8 @@ power_tc_kernel(const __grid_constant__ CUtensorMap map_gh, const __grid_constan
     if (lane == 0) {
       uint32_t it = 0, n = 0;
       bool ok = true;
-      for (int item = blockIdx.x; item < prm.n_items && ok; item += gridDim.x, ++n) {
+      for (int si = s_begin; si < s_end && ok; ++si, ++n) {
+        const int item = s_items[si];
         int b, tile; ReqPlan rp;
         decode(item, b, rp, tile);
         // the previous item's staged block lives in the ring until its epilogue is done
@@ -509,7 +514,8 @@ power_tc_kernel(const __grid_constant__ CUtensorMap map_gh, const __grid_constan
     if (lane == 0) {
       uint32_t it = 0, n = 0;
       bool ok = true;
-      for (int item = blockIdx.x; item < prm.n_items && ok; item += gridDim.x, ++n) {
+      for (int si = s_begin; si < s_end && ok; ++si, ++n) {
+        const int item = s_items[si];
         int b, tile; ReqPlan rp;
         decode(item, b, rp, tile);
         const uint32_t idesc = umma_idesc(kTile, (rp.p + 15) & ~15);
@@ -545,7 +551,8 @@ power_tc_kernel(const __grid_constant__ CUtensorMap map_gh, const __grid_constan
     uint32_t n = 0;
     int cached_b = -1;
     bool ok = true;
-    for (int item = blockIdx.x; item < prm.n_items; item += gridDim.x, ++n) {
+    for (int si = s_begin; si < s_end; ++si, ++n) {
+      const int item = s_items[si];
       int b, tile; ReqPlan rp;
       decode(item, b, rp, tile);
       const int p = rp.p, P = (p + 7) & ~7;
