@@ -47,11 +47,45 @@ __device__ __forceinline__ unsigned block_exclusive_scan(unsigned v, unsigned* w
 // emission: every element above the k-th value, plus the lowest-index elements equal to it until k
 // are taken.  out[0..k) receives the selected positions in ascending order, mapped through `remap`
 // when given.  `all_equal` treats every key as equal (selects the first k positions).
+constexpr int kRankSelectMax = 1024;   // up to this many keys the selection ranks every key directly
+
 __device__ void block_topk(const float* __restrict__ keys, int n, int k, bool all_equal,
                            const int* __restrict__ remap, int* __restrict__ out, int* status) {
   __shared__ unsigned hist[256];
   __shared__ unsigned sel_prefix, sel_k;
   __shared__ unsigned warp_tot[33];
+  __shared__ unsigned skeys[kRankSelectMax];
+  if (n <= kRankSelectMax) {
+    // Small segments: rank of key i = number of keys that precede it in (larger value, lower index)
+    // order, counted against the whole segment held in shared memory (every thread reads the same
+    // key at the same time: a broadcast); key i is selected when its rank is below k.  Positions
+    // are emitted in ascending order through a block scan of the selection flags.
+    bool bad = false;
+    for (int i = threadIdx.x; i < n; i += blockDim.x) {
+      float v = keys[i];
+      bad |= !all_equal && !(fabsf(v) <= 3.402823466e38f);
+      skeys[i] = all_equal ? 0u : order_key(v);
+    }
+    if (bad) atomicOr(status, kStatusNonFinite);
+    __syncthreads();
+    unsigned run = 0u;
+    for (int base = 0; base < n; base += blockDim.x) {
+      int i = base + threadIdx.x;
+      unsigned sel = 0u;
+      if (i < n) {
+        unsigned ki = skeys[i];
+        int rank = 0;
+        for (int j = 0; j < i; ++j) rank += skeys[j] >= ki;       // equal keys with a lower index come first
+        for (int j = i + 1; j < n; ++j) rank += skeys[j] > ki;
+        sel = rank < k;
+      }
+      unsigned tot;
+      unsigned ex = block_exclusive_scan(sel, warp_tot, &tot);
+      if (sel) out[run + ex] = remap ? remap[i] : i;
+      run += tot;
+    }
+    return;
+  }
   unsigned prefix = 0u, mask = 0u, kk = (unsigned)k;
   if (!all_equal) {
     bool bad = false;
