@@ -145,6 +145,14 @@ int covspec_prune(covspec_ctx* ctx, const covspec_problem* p, void* out_hidden, 
  * COVSPEC_ERR_NOCONVERGE) and clears it. */
 int covspec_get_device_status(covspec_ctx* ctx, void* stream);
 
+/* Self-test of the kernels' bounded waits (no step of the paper).  Every wait inside the
+ * tensor-core kernels gives up after a fixed number of polls, raises COVSPEC_ERR_TIMEOUT in the
+ * device status word and lets the kernel return, so that a protocol fault cannot hang the GPU.
+ * This call launches one thread that waits, with the same routine and a small limit, on a barrier
+ * nothing signals; afterwards covspec_get_device_status() reports COVSPEC_ERR_TIMEOUT (and clears
+ * it).  Asynchronous on `stream`; takes well under a millisecond. */
+int covspec_selftest_wait_timeout(covspec_ctx* ctx, void* stream);
+
 /* Optional per-stage timing of covspec_prune with CUDA events recorded on the call's stream.
  * covspec_profile_begin reserves events for up to max_calls prune calls; covspec_profile_end
  * waits for them, writes the summed milliseconds of each stage into stage_ms[n_stages] (stage

@@ -25,7 +25,7 @@ EXPORTS = [
     "covspec_compact", "covspec_prune", "covspec_get_device_status",
     "covspec_last_launch_count", "covspec_strerror", "covspec_last_cuda_error",
     "covspec_profile_begin", "covspec_profile_end", "covspec_profile_stage_count",
-    "covspec_profile_stage_name", "covspec_query_score_static",
+    "covspec_profile_stage_name", "covspec_query_score_static", "covspec_selftest_wait_timeout",
 ]
 STATIC_MAX_BATCH = 256
 STATIC_MAX_QUERY_ELEMS = 1 << 20
@@ -89,6 +89,7 @@ def load_library():
     lib.covspec_compact.argtypes = [vp, C.POINTER(Problem), vp, ip, vp, vp, vp]
     lib.covspec_prune.argtypes = [vp, C.POINTER(Problem), vp, vp, ip, vp]
     lib.covspec_get_device_status.argtypes = [vp, vp]
+    lib.covspec_selftest_wait_timeout.argtypes = [vp, vp]
     lib.covspec_last_launch_count.argtypes = [vp]
     lib.covspec_strerror.argtypes = [C.c_int]
     lib.covspec_strerror.restype = C.c_char_p
@@ -309,6 +310,12 @@ class Pruner:
             raise CovspecError(st, "covspec_profile_end")
         names = [self.lib.covspec_profile_stage_name(i).decode() for i in range(n)]
         return dict(zip(names, list(ms))), calls.value
+
+    def selftest_wait_timeout(self):
+        """covspec_selftest_wait_timeout: makes one bounded wait run out on purpose."""
+        st = self.lib.covspec_selftest_wait_timeout(self._ctx, _stream())
+        if st:
+            raise CovspecError(st, "covspec_selftest_wait_timeout")
 
     def device_status(self) -> int:
         return int(self.lib.covspec_get_device_status(self._ctx, _stream()))

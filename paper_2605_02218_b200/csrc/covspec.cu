@@ -922,6 +922,14 @@ int covspec_get_device_status(covspec_ctx* ctx, void* stream) {
   return COVSPEC_OK;
 }
 
+int covspec_selftest_wait_timeout(covspec_ctx* ctx, void* stream) {
+  if (!ctx) return COVSPEC_ERR_ARG;
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  tc::wait_timeout_selftest_kernel<<<1, 32, 0, s>>>(ctx->status, 4096u);
+  CUDA_TRY(cudaGetLastError());
+  return COVSPEC_OK;
+}
+
 int covspec_last_launch_count(const covspec_ctx* ctx) { return ctx ? ctx->launches : 0; }
 
 const char* covspec_strerror(int status) {

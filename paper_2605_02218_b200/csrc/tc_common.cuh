@@ -41,14 +41,18 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-// Bounded wait.  Returns false when the limit expired or another role already gave up.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
-  for (uint32_t i = 0; i < kSpinLimit; ++i) {
+// Bounded wait.  Returns false when `limit` polls expired or another role already gave up.
+__device__ __forceinline__ bool mbar_wait_limited(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                                  uint32_t limit) {
+  for (uint32_t i = 0; i < limit; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((i & 255u) == 255u && *abort_flag) return false;
   }
   *abort_flag = 1;
   return false;
+}
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+  return mbar_wait_limited(bar, parity, abort_flag, kSpinLimit);
 }
 
 __device__ __forceinline__ void tma_load_2d(uint32_t smem_dst, const CUtensorMap* map, int x, int y,
@@ -140,6 +144,23 @@ __device__ __forceinline__ void tmem_dealloc(uint32_t base, int cols) {
 // Named barrier among the first `n` threads' warps (id 1..15; 0 is __syncthreads).
 __device__ __forceinline__ void named_barrier(int id, int n) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n) : "memory");
+}
+
+// Self-test of the bounded wait: one thread waits on a barrier that nothing signals; the wait gives
+// up after `limit` polls and the time-out is recorded in the status word, exactly as the kernels do.
+__global__ void wait_timeout_selftest_kernel(int* status, uint32_t limit) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    mbar_init(&bar, 1);
+    abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    bool ok = mbar_wait_limited(&bar, 0, &abort_flag, limit);
+    if (!ok && abort_flag) atomicOr(status, kStatusTimeout);
+  }
 }
 
 }  // namespace tc

@@ -168,6 +168,24 @@ def test_device_status_reports_nonfinite():
     assert len(np.unique(k)) == 8 and k.min() >= 0 and k.max() < 64
 
 
+def test_bounded_wait_reports_timeout():
+    # A wait on a barrier that nothing signals runs out after its poll limit: the kernel returns,
+    # the status word says so, and the context keeps working.
+    from paper_2605_02218_b200 import api
+    wl = workloads.make_workload("timeout", seed=34, dtype=torch.bfloat16, batch=1, n_vis=200, n_txt=4,
+                                 d=128, n_heads=1, rank=8, keep=20).to("cuda:0")
+    pr = api.Pruner.for_workload(wl)
+    m = pr.marshal(wl)
+    ref = pr.prune(m)
+    assert pr.device_status() == 0
+    pr.selftest_wait_timeout()
+    assert pr.device_status() == -9
+    assert pr.device_status() == 0        # reading clears it
+    again = pr.prune(m)
+    assert torch.equal(ref[1], again[1]) and torch.equal(ref[0], again[0])
+    assert pr.device_status() == 0
+
+
 def test_capacity_and_argument_errors():
     from paper_2605_02218_b200 import api
     wl = workloads.make_workload("cap", seed=33, dtype=torch.bfloat16, batch=2, n_vis=100, n_txt=4,
