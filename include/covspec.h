@@ -145,6 +145,30 @@ int covspec_prune(covspec_ctx* ctx, const covspec_problem* p, void* out_hidden, 
  * COVSPEC_ERR_NOCONVERGE) and clears it. */
 int covspec_get_device_status(covspec_ctx* ctx, void* stream);
 
+/* Device-side gating and correction over the vocabulary (Sec. III-B.1 and III-C.2), one call for
+ * `rows` decoding positions; needs no context and no workspace.
+ *  logit_dtype   COVSPEC_F32, COVSPEC_BF16 or COVSPEC_F16 (the paper sends logits as float16)
+ *  z_draft       device [rows, ld] draft logits z_d (Eq. 1); ld >= vocab, ld * element size a
+ *                multiple of 16 bytes, base 16-byte aligned
+ *  z_target      device [rows, ld] target logits z_t of the position (Eq. 3)
+ *  drafted       device [rows] int32 drafted token ids in [0, vocab) or NULL
+ *  uniforms      device [rows] float32 in [0, 1): the random numbers of the correction draw
+ *  gamma         margin threshold of Eq. 17
+ *  margin        device [rows] float32 (out): p_(1) - p_(2) of softmax(z_d)         (Eq. 2, 16)
+ *  gate          device [rows] int32   (out): 1 if margin < gamma else 0               (Eq. 17)
+ *  accept        device [rows] float32 (out, may be NULL): min(1, p_t(y)/p_d(y))        (Eq. 4, 5);
+ *                1 when drafted is NULL
+ *  resid_mass    device [rows] float32 (out, may be NULL): sum_w max(p_t(w) - p_d(w), 0)
+ *  token         device [rows] int32   (out): the first token whose cumulative residual
+ *                probability (Eq. 6, vocabulary order) exceeds uniforms[row]; drawn from p_t when
+ *                the residual is identically zero
+ * Returns COVSPEC_ERR_ARG / COVSPEC_ERR_SHAPE / COVSPEC_ERR_CUDA on the host before launching. */
+#define COVSPEC_F16 2
+int covspec_correct(int logit_dtype, int rows, int vocab, long long ld, const void* z_draft,
+                    const void* z_target, const int* drafted, const float* uniforms, float gamma,
+                    float* margin, int* gate, float* accept, float* resid_mass, int* token,
+                    void* stream);
+
 /* Self-test of the kernels' bounded waits (no step of the paper).  Every wait inside the
  * tensor-core kernels gives up after a fixed number of polls, raises COVSPEC_ERR_TIMEOUT in the
  * device status word and lets the kernel return, so that a protocol fault cannot hang the GPU.

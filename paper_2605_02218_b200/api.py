@@ -15,7 +15,7 @@ import torch
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libcovspec.so")
 
-COVSPEC_F32, COVSPEC_BF16 = 0, 1
+COVSPEC_F32, COVSPEC_BF16, COVSPEC_F16 = 0, 1, 2
 NORM_MODES = {"minmax": 0, "zscore": 1, "none": 2}
 HEAD_REDUCE = {"max": 0, "mean": 1}
 
@@ -26,6 +26,7 @@ EXPORTS = [
     "covspec_last_launch_count", "covspec_strerror", "covspec_last_cuda_error",
     "covspec_profile_begin", "covspec_profile_end", "covspec_profile_stage_count",
     "covspec_profile_stage_name", "covspec_query_score_static", "covspec_selftest_wait_timeout",
+    "covspec_correct",
 ]
 STATIC_MAX_BATCH = 256
 STATIC_MAX_QUERY_ELEMS = 1 << 20
@@ -90,6 +91,8 @@ def load_library():
     lib.covspec_prune.argtypes = [vp, C.POINTER(Problem), vp, vp, ip, vp]
     lib.covspec_get_device_status.argtypes = [vp, vp]
     lib.covspec_selftest_wait_timeout.argtypes = [vp, vp]
+    lib.covspec_correct.argtypes = [C.c_int, C.c_int, C.c_int, C.c_longlong, vp, vp, vp, vp, C.c_float,
+                                    vp, vp, vp, vp, vp, vp]
     lib.covspec_last_launch_count.argtypes = [vp]
     lib.covspec_strerror.argtypes = [C.c_int]
     lib.covspec_strerror.restype = C.c_char_p
@@ -344,3 +347,30 @@ def query_score_static(X: torch.Tensor, Q: torch.Tensor, vis_offsets, txt_offset
     if st:
         raise CovspecError(st, "covspec_query_score_static")
     return out
+
+
+_LOGIT_DTYPES = {torch.float32: COVSPEC_F32, torch.bfloat16: COVSPEC_BF16, torch.float16: COVSPEC_F16}
+
+
+def correct(z_draft: torch.Tensor, z_target: torch.Tensor, uniforms: torch.Tensor, gamma: float,
+            drafted: Optional[torch.Tensor] = None, vocab: Optional[int] = None):
+    """covspec_correct: gating (Eq. 16-17), acceptance probability (Eq. 5) and the residual
+    correction draw (Eq. 6) for every row of two logit matrices [rows, ld] (ld >= vocab).
+    Returns (margin, gate, accept, resid_mass, token) device tensors."""
+    lib = load_library()
+    assert z_draft.is_cuda and z_draft.is_contiguous() and z_target.is_contiguous()
+    assert z_draft.shape == z_target.shape and z_draft.dtype == z_target.dtype
+    rows, ld = z_draft.shape
+    vocab = ld if vocab is None else vocab
+    dev = z_draft.device
+    margin = torch.empty(rows, dtype=torch.float32, device=dev)
+    gate = torch.empty(rows, dtype=torch.int32, device=dev)
+    accept = torch.empty(rows, dtype=torch.float32, device=dev)
+    mass = torch.empty(rows, dtype=torch.float32, device=dev)
+    token = torch.empty(rows, dtype=torch.int32, device=dev)
+    st = lib.covspec_correct(_LOGIT_DTYPES[z_draft.dtype], rows, vocab, ld, _ptr(z_draft), _ptr(z_target),
+                             _ptr(drafted), _ptr(uniforms), float(gamma), _ptr(margin), _ptr(gate),
+                             _ptr(accept), _ptr(mass), _ptr(token), _stream())
+    if st:
+        raise CovspecError(st, "covspec_correct")
+    return margin, gate, accept, mass, token

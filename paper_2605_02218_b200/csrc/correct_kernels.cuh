@@ -1,0 +1,258 @@
+// Device-side gating and correction over the vocabulary (Eq. 2, 4, 5, 6, 16, 17; Sec. III-C.2):
+// from the draft logits and the target logits of one position, the draft distribution's top-2 margin
+// and gate, the acceptance probability of the drafted token, the residual distribution
+// max(p_t - p_d, 0) / mass and a token drawn from it by inverse CDF with a uniform number supplied by
+// the caller.
+//
+// One block per position; HBM-bound.  Both logit rows (2 * W * elem bytes, ~600 KB at W = 152 k in
+// 16 bits) are read from HBM once; the second sweep (residual mass) and the short third one (the
+// cumulative sum inside the one warp segment that contains the sample) find them in L2.  Each warp
+// owns a contiguous segment of the row and reads it with coalesced 16-byte vectors, so the order of
+// the cumulative sum is (segment, vector, lane, element).
+#pragma once
+#include <cuda_fp16.h>
+
+#include "common.cuh"
+
+namespace covspec {
+namespace corr {
+
+constexpr int kThreads = 1024;
+constexpr int kWarps = kThreads / 32;
+
+__device__ __forceinline__ float cvt(float v) { return v; }
+__device__ __forceinline__ float cvt(__half v) { return __half2float(v); }
+__device__ __forceinline__ float cvt(__nv_bfloat16 v) { return __bfloat162float(v); }
+
+template <typename T> struct Vec;           // 16-byte vector of logits
+template <> struct Vec<float> { static constexpr int N = 4; };
+template <> struct Vec<__half> { static constexpr int N = 8; };
+template <> struct Vec<__nv_bfloat16> { static constexpr int N = 8; };
+
+// Loads the N consecutive logits that start at element `i` (a multiple of N) of `row`; elements at
+// or beyond `w` read as -inf (probability zero).  The row base is 16-byte aligned.
+template <typename T>
+__device__ __forceinline__ void load_vec(const T* __restrict__ row, int i, int w, float (&v)[Vec<T>::N]) {
+  constexpr int N = Vec<T>::N;
+  if (i + N <= w) {
+    uint4 raw = *reinterpret_cast<const uint4*>(row + i);
+    const T* e = reinterpret_cast<const T*>(&raw);
+#pragma unroll
+    for (int k = 0; k < N; ++k) v[k] = cvt(e[k]);
+  } else {
+#pragma unroll
+    for (int k = 0; k < N; ++k) v[k] = i + k < w ? cvt(row[i + k]) : -INFINITY;
+  }
+}
+
+// Running (max, sum of exp(z - max)) pair of a softmax denominator.
+struct MaxSum {
+  float m, s;
+  __device__ __forceinline__ void add(float z) {
+    if (z > m) { s = s * __expf(m - z) + 1.f; m = z; }
+    else s += __expf(z - m);
+  }
+  __device__ __forceinline__ void merge(const MaxSum& o) {
+    if (o.m > m) { s = s * __expf(m - o.m) + o.s; m = o.m; }
+    else if (o.m > -INFINITY) s += o.s * __expf(o.m - m);
+  }
+};
+__device__ __forceinline__ MaxSum shfl_xor(const MaxSum& a, int o) {
+  MaxSum r;
+  r.m = __shfl_xor_sync(0xffffffffu, a.m, o);
+  r.s = __shfl_xor_sync(0xffffffffu, a.s, o);
+  return r;
+}
+
+// Probability of one logit given the row maximum and the reciprocal denominator.  The product is
+// rounded on its own (no fused multiply-add with the subtraction that follows), so that identical
+// draft and target rows give a residual of exactly zero.
+__device__ __forceinline__ float prob(float z, float zmax, float inv_sum) {
+  return __fmul_rn(__expf(z - zmax), inv_sum);
+}
+
+// Two largest values of a multiset.
+struct Top2 {
+  float a, b;   // a >= b
+  __device__ __forceinline__ void add(float z) {
+    if (z > a) { b = a; a = z; } else if (z > b) b = z;
+  }
+  __device__ __forceinline__ void merge(const Top2& o) { add(o.a); add(o.b); }
+};
+
+// rows: positions; w: vocabulary size; ldz: elements between consecutive rows (multiple of 16 bytes).
+template <typename T>
+__global__ void __launch_bounds__(kThreads)
+correct_kernel(const T* __restrict__ zd, const T* __restrict__ zt, long long ldz, int w,
+               const int* __restrict__ drafted, const float* __restrict__ uniforms, float gamma,
+               float* __restrict__ margin, int* __restrict__ gate, float* __restrict__ accept,
+               float* __restrict__ resid_mass, int* __restrict__ token) {
+  constexpr int N = Vec<T>::N;
+  __shared__ MaxSum sh_d[kWarps], sh_t[kWarps];
+  __shared__ Top2 sh_top[kWarps];
+  __shared__ float sh_mass[kWarps];
+  __shared__ float bc[6];
+  __shared__ int sh_token;
+  const int row = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const T* rd = zd + (size_t)row * ldz;
+  const T* rt = zt + (size_t)row * ldz;
+  // contiguous segment of this warp, in whole vectors
+  const int nvec = (w + N - 1) / N;
+  const int vec_per_warp = (nvec + kWarps - 1) / kWarps;
+  const int v0 = warp * vec_per_warp, v1 = min(nvec, v0 + vec_per_warp);
+
+  // ---- sweep 1: softmax denominators of both rows (Eq. 2, 4), two largest draft logits (Eq. 16) ----
+  MaxSum md{-INFINITY, 0.f}, mt{-INFINITY, 0.f};
+  Top2 top{-INFINITY, -INFINITY};
+  for (int v = v0 + lane; v < v1; v += 32) {
+    float a[N], b[N];
+    load_vec(rd, v * N, w, a);
+    load_vec(rt, v * N, w, b);
+#pragma unroll
+    for (int k = 0; k < N; ++k) {
+      if (a[k] > -INFINITY) { md.add(a[k]); top.add(a[k]); }
+      if (b[k] > -INFINITY) mt.add(b[k]);
+    }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    md.merge(shfl_xor(md, o));
+    mt.merge(shfl_xor(mt, o));
+    Top2 other{__shfl_xor_sync(0xffffffffu, top.a, o), __shfl_xor_sync(0xffffffffu, top.b, o)};
+    top.merge(other);
+  }
+  if (lane == 0) { sh_d[warp] = md; sh_t[warp] = mt; sh_top[warp] = top; }
+  __syncthreads();
+  if (warp == 0) {
+    md = sh_d[lane]; mt = sh_t[lane]; top = sh_top[lane];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      md.merge(shfl_xor(md, o));
+      mt.merge(shfl_xor(mt, o));
+      Top2 other{__shfl_xor_sync(0xffffffffu, top.a, o), __shfl_xor_sync(0xffffffffu, top.b, o)};
+      top.merge(other);
+    }
+    if (lane == 0) {
+      bc[0] = md.m; bc[1] = 1.f / md.s; bc[2] = mt.m; bc[3] = 1.f / mt.s;
+      float m = (1.f - (top.b > -INFINITY ? __expf(top.b - top.a) : 0.f)) * __expf(top.a - md.m) / md.s;
+      margin[row] = m;
+      gate[row] = m < gamma ? 1 : 0;                                       // Eq. 17
+      if (accept != nullptr) {
+        float al = 1.f;
+        if (drafted != nullptr) {
+          int y = drafted[row];
+          float pd = __expf(cvt(rd[y]) - md.m) / md.s, pt = __expf(cvt(rt[y]) - mt.m) / mt.s;
+          al = pd > 0.f ? fminf(1.f, pt / pd) : 1.f;                       // Eq. 5
+        }
+        accept[row] = al;
+      }
+    }
+  }
+  __syncthreads();
+  const float max_d = bc[0], inv_d = bc[1], max_t = bc[2], inv_t = bc[3];
+
+  // ---- sweep 2: residual mass per warp segment (Eq. 6 denominator) ----
+  // use_pt: the residual is identically zero (the two distributions coincide): draw from p_t.
+  for (int use_pt = 0; use_pt < 2; ++use_pt) {
+    float part = 0.f;
+    for (int v = v0 + lane; v < v1; v += 32) {
+      float a[N], b[N];
+      load_vec(rd, v * N, w, a);
+      load_vec(rt, v * N, w, b);
+#pragma unroll
+      for (int k = 0; k < N; ++k) {
+        float pt = prob(b[k], max_t, inv_t), pd = prob(a[k], max_d, inv_d);
+        part += use_pt ? pt : fmaxf(pt - pd, 0.f);
+      }
+    }
+    part = warp_sum(part);
+    if (lane == 0) sh_mass[warp] = part;
+    __syncthreads();
+    float mass = 0.f;
+    for (int q = 0; q < kWarps; ++q) mass += sh_mass[q];                  // same order in every thread
+    if (!use_pt && tid == 0 && resid_mass != nullptr) resid_mass[row] = mass;
+    if (mass > 0.f || use_pt) {
+      // ---- sweep 3: the warp whose segment contains x * mass walks it in order ----
+      const float target = uniforms[row] * mass;
+      float before = 0.f;
+      int seg = -1;
+      for (int q = 0; q < kWarps; ++q) {
+        if (seg < 0 && before + sh_mass[q] > target) seg = q;
+        if (seg < 0) before += sh_mass[q];
+      }
+      if (tid == 0) sh_token = -1;
+      __syncthreads();
+      float tgt = target;
+      if (seg < 0) {
+        // rounding left x * mass at or above the total: the last token with positive probability,
+        // i.e. the walk below never crosses and reports the last positive entry of this segment
+        seg = kWarps - 1;
+        while (seg > 0 && !(sh_mass[seg] > 0.f)) --seg;
+        tgt = INFINITY;
+      }
+      if (warp == seg) {
+        float run = before;
+        int found = -1, last_pos = -1;
+        for (int vb = v0; vb < v1; vb += 32) {
+          int v = vb + lane;
+          float r[N];
+          float lsum = 0.f;
+          if (v < v1) {
+            float a[N], b[N];
+            load_vec(rd, v * N, w, a);
+            load_vec(rt, v * N, w, b);
+#pragma unroll
+            for (int k = 0; k < N; ++k) {
+              float pt = prob(b[k], max_t, inv_t), pd = prob(a[k], max_d, inv_d);
+              r[k] = use_pt ? pt : fmaxf(pt - pd, 0.f);
+              lsum += r[k];
+            }
+          } else {
+#pragma unroll
+            for (int k = 0; k < N; ++k) r[k] = 0.f;
+          }
+          // exclusive prefix over lanes
+          float inc = lsum;
+#pragma unroll
+          for (int o = 1; o < 32; o <<= 1) {
+            float t = __shfl_up_sync(0xffffffffu, inc, o);
+            if (lane >= o) inc += t;
+          }
+          float acc = run + inc - lsum;
+          int mine = -1, mylast = -1;
+#pragma unroll
+          for (int k = 0; k < N; ++k) {
+            if (r[k] > 0.f) mylast = v * N + k;
+            acc += r[k];
+            if (mine < 0 && r[k] > 0.f && acc > tgt) mine = v * N + k;
+          }
+          // first lane that crossed; last positive element seen so far
+          unsigned hit = __ballot_sync(0xffffffffu, mine >= 0);
+          unsigned pos = __ballot_sync(0xffffffffu, mylast >= 0);
+          if (pos) last_pos = __shfl_sync(0xffffffffu, mylast, 31 - __clz(pos));
+          if (hit) { found = __shfl_sync(0xffffffffu, mine, __ffs(hit) - 1); break; }
+          run += __shfl_sync(0xffffffffu, inc, 31);
+        }
+        if (lane == 0) sh_token = found >= 0 ? found : last_pos;
+      }
+      __syncthreads();
+      if (tid == 0) {
+        int tk = sh_token;
+        if (tk < 0) {
+          // the chosen segment held no positive entry at all (possible only through rounding):
+          // scan back for the last positive probability in the whole row
+          for (int i = w - 1; i >= 0 && tk < 0; --i) {
+            float pt = prob(cvt(rt[i]), max_t, inv_t), pd = prob(cvt(rd[i]), max_d, inv_d);
+            if ((use_pt ? pt : pt - pd) > 0.f) tk = i;
+          }
+        }
+        token[row] = tk;
+      }
+      break;
+    }
+    __syncthreads();
+  }
+}
+
+}  // namespace corr
+}  // namespace covspec

@@ -12,6 +12,7 @@
 #include <vector>
 
 #include "common.cuh"
+#include "correct_kernels.cuh"
 #include "eig_kernels.cuh"
 #include "gemm_simt.cuh"
 #include "relevance_tc.cuh"
@@ -919,6 +920,33 @@ int covspec_get_device_status(covspec_ctx* ctx, void* stream) {
   if (h & kStatusTimeout) return COVSPEC_ERR_TIMEOUT;
   if (h & kStatusNonFinite) return COVSPEC_ERR_NONFINITE;
   if (h & kStatusNoConverge) return COVSPEC_ERR_NOCONVERGE;
+  return COVSPEC_OK;
+}
+
+int covspec_correct(int logit_dtype, int rows, int vocab, long long ld, const void* z_draft,
+                    const void* z_target, const int* drafted, const float* uniforms, float gamma,
+                    float* margin, int* gate, float* accept, float* resid_mass, int* token,
+                    void* stream) {
+  if (!z_draft || !z_target || !uniforms || !margin || !gate || !token) return COVSPEC_ERR_ARG;
+  if (logit_dtype != COVSPEC_F32 && logit_dtype != COVSPEC_BF16 && logit_dtype != COVSPEC_F16)
+    return COVSPEC_ERR_ARG;
+  int esize = logit_dtype == COVSPEC_F32 ? 4 : 2;
+  if (rows < 1 || vocab < 2 || ld < vocab || (ld * esize) % 16 != 0) return COVSPEC_ERR_SHAPE;
+  if ((reinterpret_cast<uintptr_t>(z_draft) | reinterpret_cast<uintptr_t>(z_target)) & 15) return COVSPEC_ERR_ARG;
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  if (logit_dtype == COVSPEC_F32)
+    corr::correct_kernel<float><<<rows, corr::kThreads, 0, s>>>(
+        static_cast<const float*>(z_draft), static_cast<const float*>(z_target), ld, vocab, drafted,
+        uniforms, gamma, margin, gate, accept, resid_mass, token);
+  else if (logit_dtype == COVSPEC_BF16)
+    corr::correct_kernel<__nv_bfloat16><<<rows, corr::kThreads, 0, s>>>(
+        static_cast<const __nv_bfloat16*>(z_draft), static_cast<const __nv_bfloat16*>(z_target), ld,
+        vocab, drafted, uniforms, gamma, margin, gate, accept, resid_mass, token);
+  else
+    corr::correct_kernel<__half><<<rows, corr::kThreads, 0, s>>>(
+        static_cast<const __half*>(z_draft), static_cast<const __half*>(z_target), ld, vocab, drafted,
+        uniforms, gamma, margin, gate, accept, resid_mass, token);
+  CUDA_TRY(cudaGetLastError());
   return COVSPEC_OK;
 }
 

@@ -224,3 +224,24 @@ def make_config(name: str, device="cpu", **overrides) -> Workload:
     kw = dict(CONFIGS[name])
     kw.update(overrides)
     return make_workload(name, device=device, **kw)
+
+
+def make_logits(*, seed=0, rows=64, vocab=151674, dtype=torch.float16, spread=3.0, disagreement=1.0,
+                device="cpu"):
+    """Seeded draft / target logit rows for the device-side correction step: draft logits
+    spread * N(0, 1), target logits = draft + disagreement * N(0, 1) (the two models mostly agree),
+    uniform numbers in [0, 1) for the correction draw and uniformly drawn drafted token ids.  Rows are
+    padded to a multiple of 8 elements (16-byte rows); the padding holds zeros and is not part of the
+    vocabulary.  Returns a dict of tensors and sizes; draws only, none of the method's arithmetic."""
+    gen = torch.Generator(device=device)
+    gen.manual_seed(seed)
+    ld = (vocab + 7) // 8 * 8
+    zd = torch.zeros(rows, ld, dtype=torch.float32, device=device)
+    zt = torch.zeros(rows, ld, dtype=torch.float32, device=device)
+    base = spread * torch.randn(rows, vocab, generator=gen, device=device)
+    zd[:, :vocab] = base
+    zt[:, :vocab] = base + disagreement * torch.randn(rows, vocab, generator=gen, device=device)
+    uniforms = torch.rand(rows, generator=gen, device=device, dtype=torch.float32)
+    drafted = torch.randint(0, vocab, (rows,), generator=gen, device=device, dtype=torch.int32)
+    return dict(z_draft=zd.to(dtype), z_target=zt.to(dtype), uniforms=uniforms, drafted=drafted,
+                rows=rows, vocab=vocab, ld=ld)
