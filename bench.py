@@ -32,7 +32,7 @@ from paper_2605_02218_b200 import workloads
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one visual-side relevance_tc_kernel launch (ncu,
 # profiles/relevance_tc_kernel_c2.md); None where no capture of the current kernel exists.
-NCU_TRAFFIC_BYTES = {"c2": 55.675e6}
+NCU_TRAFFIC_BYTES = {"c2": 55.675e6, "correct_per_row": 343.9e6 / 512}   # profiles/correct_kernel_vocab152k.md
 
 METRIC = "visual_tokens_pruned_per_s"
 UNIT = "tokens/s"
@@ -190,6 +190,62 @@ def run_reference(args, rank):
     print(json.dumps(line))
 
 
+def run_correction(args):
+    """Secondary measurement (not the headline metric): covspec_correct, the device-side gating and
+    residual-correction kernel (Eq. 5, 6, 16, 17), on float16 logit rows of a 151,674-token
+    vocabulary.  HBM-bound: both logit rows are read once from HBM."""
+    from paper_2605_02218_b200 import api, build
+    from oracle import correction_oracle
+    build.build()
+    torch.cuda.set_device(0)
+    rows, vocab = args.corr_rows, 151674
+    data = workloads.make_logits(seed=11, rows=rows, vocab=vocab, dtype=torch.float16, device="cuda:0")
+    call = lambda: api.correct(data["z_draft"], data["z_target"], data["uniforms"], 0.02, data["drafted"], vocab=vocab)
+    for _ in range(max(args.warmup, 3)):
+        call()
+    torch.cuda.synchronize()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(0) as clk:
+        ev0.record()
+        for _ in range(args.steps):
+            call()
+        ev1.record()
+        torch.cuda.synchronize()
+    ms = ev0.elapsed_time(ev1) / args.steps
+    bytes_alg = 2.0 * rows * vocab * 2                       # both logit rows, once
+    peaks = _peaks()
+    gbs = bytes_alg / (ms * 1e-3) / 1e9
+    # The kernel evaluates 4.25 exponentials per vocabulary entry (softmax denominators with one
+    # rescale per 8-element vector, then both probabilities again for the residual); the special
+    # function units deliver 16 per clock per SM.
+    exps = 4.25 * rows * vocab
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    xu_peak = 16.0 * sms * 1.965                             # G exp/s at the 1965 MHz maximum clock
+    gexp = exps / (ms * 1e-3) / 1e9
+    zd = data["z_draft"][:8, :vocab].cpu().double().numpy(); zt = data["z_target"][:8, :vocab].cpu().double().numpy()
+    xs = data["uniforms"][:8].cpu().numpy()
+    t0 = time.perf_counter(); n = 0
+    while time.perf_counter() - t0 < 10.0:
+        correction_oracle.correct_position(zd[n % 8], zt[n % 8], float(xs[n % 8]), 0.02, y=3)
+        n += 1
+    dt = time.perf_counter() - t0
+    print(json.dumps(dict(
+        metric="positions_corrected_per_s", value=rows / (ms * 1e-3), unit="positions/s", n_gpus=1,
+        steps=args.steps, warmup=max(args.warmup, 3), ms_per_step=ms, higher_is_better=True,
+        dtype="f32", data="synthetic",
+        config=dict(workload=f"covspec_correct: {rows} positions x {vocab} logits, float16, draft + target rows",
+                    l2="inputs (%.0f MB) larger than L2" % (bytes_alg / 1e6)),
+        gpu_launches=args.steps, clocks=clk.summary(),
+        roofline=dict(bound="alu", achieved=gexp, peak=xu_peak, unit="Gexp/s", frac=gexp / xu_peak,
+                      traffic=NCU_TRAFFIC_BYTES.get("correct_per_row", 0) * rows or None,
+                      kernel="correct_kernel<__half>",
+                      peak_source="16 exp/clk/SM x %d SMs x 1.965 GHz" % sms,
+                      hbm=dict(achieved=gbs, peak=peaks["hbm"], unit="GB/s", frac=gbs / peaks["hbm"],
+                               bytes_per_launch=bytes_alg)),
+        cpu_baseline=dict(value=n / dt, unit="positions/s", cores=1, kind="oracle",
+                          sample=f"{n} positions of the same rows, {dt:.1f} s"))))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -201,6 +257,9 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--ref-batch", type=int, default=16)
     ap.add_argument("--ref-budget", type=float, default=20.0)
+    ap.add_argument("--kernel", default="prune", choices=["prune", "correct"],
+                    help="prune: the headline path (default); correct: the gating / correction kernel")
+    ap.add_argument("--corr-rows", type=int, default=1024)
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", 0))
@@ -208,6 +267,10 @@ def main():
     world = int(os.environ.get("WORLD_SIZE", 1))
     if args.impl == "reference":
         run_reference(args, rank)
+        return
+    if args.kernel == "correct":
+        if rank == 0:
+            run_correction(args)
         return
 
     from paper_2605_02218_b200 import api, build

@@ -82,7 +82,7 @@ struct Top2 {
 
 // rows: positions; w: vocabulary size; ldz: elements between consecutive rows (multiple of 16 bytes).
 template <typename T>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, 1)
 correct_kernel(const T* __restrict__ zd, const T* __restrict__ zt, long long ldz, int w,
                const int* __restrict__ drafted, const float* __restrict__ uniforms, float gamma,
                float* __restrict__ margin, int* __restrict__ gate, float* __restrict__ accept,
@@ -104,14 +104,23 @@ correct_kernel(const T* __restrict__ zd, const T* __restrict__ zt, long long ldz
   // ---- sweep 1: softmax denominators of both rows (Eq. 2, 4), two largest draft logits (Eq. 16) ----
   MaxSum md{-INFINITY, 0.f}, mt{-INFINITY, 0.f};
   Top2 top{-INFINITY, -INFINITY};
+#pragma unroll 2
   for (int v = v0 + lane; v < v1; v += 32) {
     float a[N], b[N];
     load_vec(rd, v * N, w, a);
     load_vec(rt, v * N, w, b);
+    // one rescale per vector: every vector holds at least one element of the vocabulary, so its
+    // maximum is finite and exp(-inf - max) = 0 takes care of the padding
+    float va = a[0], vb = b[0];
+#pragma unroll
+    for (int k = 1; k < N; ++k) { va = fmaxf(va, a[k]); vb = fmaxf(vb, b[k]); }
+    if (va > md.m) { md.s *= __expf(md.m - va); md.m = va; }
+    if (vb > mt.m) { mt.s *= __expf(mt.m - vb); mt.m = vb; }
 #pragma unroll
     for (int k = 0; k < N; ++k) {
-      if (a[k] > -INFINITY) { md.add(a[k]); top.add(a[k]); }
-      if (b[k] > -INFINITY) mt.add(b[k]);
+      md.s += __expf(a[k] - md.m);
+      mt.s += __expf(b[k] - mt.m);
+      top.add(a[k]);
     }
   }
 #pragma unroll
@@ -124,7 +133,8 @@ correct_kernel(const T* __restrict__ zd, const T* __restrict__ zt, long long ldz
   if (lane == 0) { sh_d[warp] = md; sh_t[warp] = mt; sh_top[warp] = top; }
   __syncthreads();
   if (warp == 0) {
-    md = sh_d[lane]; mt = sh_t[lane]; top = sh_top[lane];
+    if (lane < kWarps) { md = sh_d[lane]; mt = sh_t[lane]; top = sh_top[lane]; }
+    else { md = MaxSum{-INFINITY, 0.f}; mt = md; top = Top2{-INFINITY, -INFINITY}; }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
       md.merge(shfl_xor(md, o));
@@ -155,6 +165,7 @@ correct_kernel(const T* __restrict__ zd, const T* __restrict__ zt, long long ldz
   // use_pt: the residual is identically zero (the two distributions coincide): draw from p_t.
   for (int use_pt = 0; use_pt < 2; ++use_pt) {
     float part = 0.f;
+#pragma unroll 2
     for (int v = v0 + lane; v < v1; v += 32) {
       float a[N], b[N];
       load_vec(rd, v * N, w, a);
