@@ -169,6 +169,21 @@ int covspec_correct(int logit_dtype, int rows, int vocab, long long ld, const vo
                     float* margin, int* gate, float* accept, float* resid_mass, int* token,
                     void* stream);
 
+/* Fan-out of the parallel branching, Eq. 23: F_j = ceil(F_0 * rho^j), 0 < rho < 1, evaluated in
+ * double (a product within 1e-9 of an integer counts as that integer).  Host only. */
+int covspec_fanout(int f0, double rho, int j);
+
+/* Bonus-token candidates (Sec. III-C.1): for every position the F_j largest draft logits, excluding
+ * the token drafted at that position; ties go to the lower token id.  No context, no workspace.
+ *  z_draft       device [rows, ld], layout and alignment as in covspec_correct
+ *  drafted       device [rows] int32 drafted token ids, or NULL (nothing excluded)
+ *  cand_offsets  device [rows+1] int32 prefix sums of the fan-outs F_j (built by the caller)
+ *  max_fanout    largest F_j (host); must be <= vocab - 1
+ *  cand          device [cand_offsets[rows]] int32 (out): candidate token ids, ascending per position */
+int covspec_branch_candidates(int logit_dtype, int rows, int vocab, long long ld, const void* z_draft,
+                              const int* drafted, const int* cand_offsets, int max_fanout, int* cand,
+                              void* stream);
+
 /* Self-test of the kernels' bounded waits (no step of the paper).  Every wait inside the
  * tensor-core kernels gives up after a fixed number of polls, raises COVSPEC_ERR_TIMEOUT in the
  * device status word and lets the kernel return, so that a protocol fault cannot hang the GPU.

@@ -66,3 +66,17 @@ def correct_position(z_d, z_t, x, gamma, y=None):
     if y is not None:
         out["accept"] = accept_probability(p_t, p_d, int(y))
     return out
+
+
+def fanout(f0, rho, j):
+    """Eq. 23: F_j = ceil(F_0 * rho^j)."""
+    import math
+    return int(math.ceil(f0 * rho ** j - 1e-9))
+
+
+def bonus_candidates(z_d, y, f):
+    """Sec. III-C.1: the f largest draft logits, the drafted token y excluded (y None: nothing
+    excluded); equal logits are taken in order of increasing token id; ids returned ascending."""
+    z = np.asarray(z_d, dtype=np.float64)
+    order = sorted((w for w in range(len(z)) if w != y), key=lambda w: (-z[w], w))
+    return np.array(sorted(order[:f]), dtype=np.int64)

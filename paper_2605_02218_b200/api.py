@@ -26,7 +26,7 @@ EXPORTS = [
     "covspec_last_launch_count", "covspec_strerror", "covspec_last_cuda_error",
     "covspec_profile_begin", "covspec_profile_end", "covspec_profile_stage_count",
     "covspec_profile_stage_name", "covspec_query_score_static", "covspec_selftest_wait_timeout",
-    "covspec_correct",
+    "covspec_correct", "covspec_fanout", "covspec_branch_candidates",
 ]
 STATIC_MAX_BATCH = 256
 STATIC_MAX_QUERY_ELEMS = 1 << 20
@@ -91,6 +91,8 @@ def load_library():
     lib.covspec_prune.argtypes = [vp, C.POINTER(Problem), vp, vp, ip, vp]
     lib.covspec_get_device_status.argtypes = [vp, vp]
     lib.covspec_selftest_wait_timeout.argtypes = [vp, vp]
+    lib.covspec_fanout.argtypes = [C.c_int, C.c_double, C.c_int]
+    lib.covspec_branch_candidates.argtypes = [C.c_int, C.c_int, C.c_int, C.c_longlong, vp, vp, vp, C.c_int, vp, vp]
     lib.covspec_correct.argtypes = [C.c_int, C.c_int, C.c_int, C.c_longlong, vp, vp, vp, vp, C.c_float,
                                     vp, vp, vp, vp, vp, vp]
     lib.covspec_last_launch_count.argtypes = [vp]
@@ -374,3 +376,31 @@ def correct(z_draft: torch.Tensor, z_target: torch.Tensor, uniforms: torch.Tenso
     if st:
         raise CovspecError(st, "covspec_correct")
     return margin, gate, accept, mass, token
+
+
+def fanout(f0: int, rho: float, j: int) -> int:
+    """covspec_fanout: F_j = ceil(F_0 * rho^j) (Eq. 23)."""
+    v = load_library().covspec_fanout(int(f0), float(rho), int(j))
+    if v < 0:
+        raise CovspecError(v, "covspec_fanout")
+    return v
+
+
+def branch_candidates(z_draft: torch.Tensor, fanouts, drafted: Optional[torch.Tensor] = None,
+                      vocab: Optional[int] = None):
+    """covspec_branch_candidates: the F_j largest draft logits of every row, the drafted token
+    excluded.  `fanouts`: one int per row.  Returns (cand int32 device tensor, offsets numpy)."""
+    lib = load_library()
+    rows, ld = z_draft.shape
+    vocab = ld if vocab is None else vocab
+    f = np.asarray(fanouts, dtype=np.int64)
+    assert len(f) == rows
+    off = np.concatenate([[0], np.cumsum(f)]).astype(np.int32)
+    d_off = torch.from_numpy(off).to(z_draft.device)
+    cand = torch.empty(max(int(off[-1]), 1), dtype=torch.int32, device=z_draft.device)
+    st = lib.covspec_branch_candidates(_LOGIT_DTYPES[z_draft.dtype], rows, vocab, ld, _ptr(z_draft),
+                                       _ptr(drafted), _ptr(d_off), int(f.max()) if rows else 0,
+                                       _ptr(cand), _stream())
+    if st:
+        raise CovspecError(st, "covspec_branch_candidates")
+    return cand[:int(off[-1])], off

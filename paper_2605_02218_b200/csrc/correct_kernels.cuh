@@ -13,6 +13,7 @@
 #include <cuda_fp16.h>
 
 #include "common.cuh"
+#include "select_kernels.cuh"
 
 namespace covspec {
 namespace corr {
@@ -263,6 +264,23 @@ correct_kernel(const T* __restrict__ zd, const T* __restrict__ zt, long long ldz
     }
     __syncthreads();
   }
+}
+
+// Bonus-token candidates of the parallel branching (Sec. III-C.1, Eq. 23): for every position the
+// F_j largest draft logits, the token drafted at that position excluded; ties go to the lower
+// token id; ids are written in ascending order at cand[cand_offsets[row] ...].  One block per
+// position (segmented radix select over the logit row, which stays in L2 between its passes).
+template <typename T>
+__global__ void __launch_bounds__(1024)
+branch_candidates_kernel(const T* __restrict__ zd, long long ldz, int w, const int* __restrict__ drafted,
+                         const int* __restrict__ cand_offsets, int* __restrict__ cand) {
+  const int row = blockIdx.x;
+  const int off = cand_offsets[row], f = cand_offsets[row + 1] - off;
+  if (f <= 0) return;
+  const T* r = zd + (size_t)row * ldz;
+  const int y = drafted != nullptr ? drafted[row] : -1;
+  block_topk_by([&](int i) { return i == y ? -INFINITY : cvt(r[i]); }, w, min(f, w), false, nullptr,
+                cand + off, nullptr);
 }
 
 }  // namespace corr

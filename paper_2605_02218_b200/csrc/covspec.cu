@@ -950,6 +950,34 @@ int covspec_correct(int logit_dtype, int rows, int vocab, long long ld, const vo
   return COVSPEC_OK;
 }
 
+int covspec_fanout(int f0, double rho, int j) {
+  if (f0 < 0 || j < 0 || !(rho > 0.0 && rho < 1.0)) return COVSPEC_ERR_ARG;
+  return (int)ceil((double)f0 * pow(rho, (double)j) - 1e-9);
+}
+
+int covspec_branch_candidates(int logit_dtype, int rows, int vocab, long long ld, const void* z_draft,
+                              const int* drafted, const int* cand_offsets, int max_fanout, int* cand,
+                              void* stream) {
+  if (!z_draft || !cand_offsets || !cand) return COVSPEC_ERR_ARG;
+  if (logit_dtype != COVSPEC_F32 && logit_dtype != COVSPEC_BF16 && logit_dtype != COVSPEC_F16)
+    return COVSPEC_ERR_ARG;
+  int esize = logit_dtype == COVSPEC_F32 ? 4 : 2;
+  if (rows < 1 || vocab < 2 || ld < vocab || (ld * esize) % 16 != 0) return COVSPEC_ERR_SHAPE;
+  if (max_fanout < 0 || max_fanout > vocab - 1) return COVSPEC_ERR_SHAPE;
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  if (logit_dtype == COVSPEC_F32)
+    corr::branch_candidates_kernel<float><<<rows, 1024, 0, s>>>(static_cast<const float*>(z_draft), ld, vocab,
+                                                                drafted, cand_offsets, cand);
+  else if (logit_dtype == COVSPEC_BF16)
+    corr::branch_candidates_kernel<__nv_bfloat16><<<rows, 1024, 0, s>>>(
+        static_cast<const __nv_bfloat16*>(z_draft), ld, vocab, drafted, cand_offsets, cand);
+  else
+    corr::branch_candidates_kernel<__half><<<rows, 1024, 0, s>>>(static_cast<const __half*>(z_draft), ld, vocab,
+                                                                 drafted, cand_offsets, cand);
+  CUDA_TRY(cudaGetLastError());
+  return COVSPEC_OK;
+}
+
 int covspec_selftest_wait_timeout(covspec_ctx* ctx, void* stream) {
   if (!ctx) return COVSPEC_ERR_ARG;
   cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);

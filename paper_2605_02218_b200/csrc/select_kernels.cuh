@@ -49,8 +49,10 @@ __device__ __forceinline__ unsigned block_exclusive_scan(unsigned v, unsigned* w
 // when given.  `all_equal` treats every key as equal (selects the first k positions).
 constexpr int kRankSelectMax = 1024;   // up to this many keys the selection ranks every key directly
 
-__device__ void block_topk(const float* __restrict__ keys, int n, int k, bool all_equal,
-                           const int* __restrict__ remap, int* __restrict__ out, int* status) {
+// `load(i)` returns key i as a float; `status` may be nullptr (non-finite keys are then not reported).
+template <typename LoadF>
+__device__ void block_topk_by(LoadF load, int n, int k, bool all_equal,
+                              const int* __restrict__ remap, int* __restrict__ out, int* status) {
   __shared__ unsigned hist[256];
   __shared__ unsigned sel_prefix, sel_k;
   __shared__ unsigned warp_tot[33];
@@ -62,11 +64,11 @@ __device__ void block_topk(const float* __restrict__ keys, int n, int k, bool al
     // are emitted in ascending order through a block scan of the selection flags.
     bool bad = false;
     for (int i = threadIdx.x; i < n; i += blockDim.x) {
-      float v = keys[i];
+      float v = load(i);
       bad |= !all_equal && !(fabsf(v) <= 3.402823466e38f);
       skeys[i] = all_equal ? 0u : order_key(v);
     }
-    if (bad) atomicOr(status, kStatusNonFinite);
+    if (bad && status != nullptr) atomicOr(status, kStatusNonFinite);
     __syncthreads();
     unsigned run = 0u;
     for (int base = 0; base < n; base += blockDim.x) {
@@ -93,7 +95,7 @@ __device__ void block_topk(const float* __restrict__ keys, int n, int k, bool al
       for (int i = threadIdx.x; i < 256; i += blockDim.x) hist[i] = 0u;
       __syncthreads();
       for (int i = threadIdx.x; i < n; i += blockDim.x) {
-        float v = keys[i];
+        float v = load(i);
         if (shift == 24) bad |= !(fabsf(v) <= 3.402823466e38f);
         unsigned key = order_key(v);
         if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
@@ -114,7 +116,7 @@ __device__ void block_topk(const float* __restrict__ keys, int n, int k, bool al
       kk = sel_k;
       mask |= 255u << shift;
     }
-    if (bad) atomicOr(status, kStatusNonFinite);
+    if (bad && status != nullptr) atomicOr(status, kStatusNonFinite);
   }
   // Ordered emission.  kk = how many elements equal to the threshold are taken.
   unsigned run_gt = 0u, run_eq = 0u;
@@ -124,7 +126,7 @@ __device__ void block_topk(const float* __restrict__ keys, int n, int k, bool al
     if (i < n) {
       if (all_equal) eq = 1u;
       else {
-        unsigned key = order_key(keys[i]);
+        unsigned key = order_key(load(i));
         gt = key > prefix; eq = key == prefix;
       }
     }
@@ -138,6 +140,11 @@ __device__ void block_topk(const float* __restrict__ keys, int n, int k, bool al
     run_gt += tot & 0xffffu;
     run_eq += tot >> 16;
   }
+}
+
+__device__ __forceinline__ void block_topk(const float* __restrict__ keys, int n, int k, bool all_equal,
+                                           const int* __restrict__ remap, int* __restrict__ out, int* status) {
+  block_topk_by([&](int i) { return keys[i]; }, n, k, all_equal, remap, out, status);
 }
 
 // Preselection: one block per request, the M best fused scores -> presel (ascending token index).

@@ -94,3 +94,24 @@ def test_sampling_frequencies_follow_the_residual():
 def test_correct_position_bundles_the_definitions():
     out = C.correct_position(GOLD["z_d"], GOLD["z_t"], 0.75, 0.35, y=2)
     assert out["token"] == 3 and out["gate"] == 1 and out["accept"] == pytest.approx(0.4)
+
+
+def test_fanout_sequence():
+    # Eq. 23 by hand: F_0 = 8, rho = 0.5 -> 8, 4, 2, 1, ceil(0.5) = 1; F_0 = 5, rho = 0.7 -> 5, 4, 3, 2, 2
+    assert [C.fanout(8, 0.5, j) for j in range(5)] == [8, 4, 2, 1, 1]
+    assert [C.fanout(5, 0.7, j) for j in range(5)] == [5, 4, 3, 2, 2]
+    assert C.fanout(3, 0.999999, 0) == 3
+
+
+def test_bonus_candidates_hand_and_brute_force():
+    z = [0.5, 2.0, 2.0, -1.0, 3.0, 2.0]
+    assert C.bonus_candidates(z, 4, 2).tolist() == [1, 2]        # 3.0 is drafted; ties 2.0 -> lowest ids
+    assert C.bonus_candidates(z, None, 3).tolist() == [1, 2, 4]
+    assert C.bonus_candidates(z, 1, 3).tolist() == [2, 4, 5]
+    rng = np.random.default_rng(5)
+    zr = np.round(rng.normal(size=40), 1)                         # many ties
+    for y in (None, 0, 17):
+        got = C.bonus_candidates(zr, y, 7)
+        assert len(set(got.tolist())) == 7 and (y is None or y not in got)
+        rest = [w for w in range(40) if w not in got and w != y]
+        assert min(zr[got]) >= max(zr[rest])                      # nothing outside beats anything inside

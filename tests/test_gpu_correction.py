@@ -88,3 +88,22 @@ def test_argument_errors():
     with pytest.raises(api.CovspecError) as e:
         api.correct(z, z, u, 0.1)
     assert e.value.status == -2
+
+
+@pytest.mark.parametrize("dtype", [torch.float16, torch.float32])
+def test_branch_candidates(dtype):
+    from paper_2605_02218_b200 import api
+    for vocab, rows in [(37, 6), (5003, 8), (151674, 4)]:
+        data = workloads.make_logits(seed=vocab + 1, rows=rows, vocab=vocab, dtype=dtype, device="cuda:0")
+        fan = [api.fanout(8, 0.6, j) for j in range(rows)]
+        assert fan == [C.fanout(8, 0.6, j) for j in range(rows)]
+        if vocab == 5003:
+            fan[0] = 1500                                         # beyond the direct-ranking size
+        cand, off = api.branch_candidates(data["z_draft"], fan, data["drafted"], vocab=vocab)
+        torch.cuda.synchronize()
+        cand = cand.cpu().numpy()
+        zd = data["z_draft"].cpu().double().numpy()[:, :vocab]
+        ys = data["drafted"].cpu().numpy()
+        for i in range(rows):
+            want = C.bonus_candidates(zd[i], int(ys[i]), min(fan[i], vocab - 1))
+            assert np.array_equal(cand[off[i]:off[i + 1]], want), (vocab, i)
