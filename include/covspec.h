@@ -184,6 +184,23 @@ int covspec_branch_candidates(int logit_dtype, int rows, int vocab, long long ld
                               const int* drafted, const int* cand_offsets, int max_fanout, int* cand,
                               void* stream);
 
+/* Scalar host-side formulas of the link model and the draft-length controller.  No device work.
+ *  covspec_uplink_bits       Eq. 7: N_draft * b_id + N_logit_draft * b_logit
+ *  covspec_downlink_bits     Eq. 8: b_acc + b_bonus if all drafted tokens were accepted, else
+ *                            b_rej + vocab * b_logit_tar
+ *  covspec_comm_latency      Eq. 9 / 19: bits / (B log2(1 + 10^(SNR/10))), B in Hz, result in s
+ *  covspec_ema_update        Eq. 18: n_acc updates with a = 1, then k - n_acc updates with a = 0
+ *  covspec_draft_length      Eq. 20-22: phi from (p_hat, T_rej), k <- clip(round(k s^phi), k_min, k_max),
+ *                            halves rounded away from zero; returns the new k (negative status on
+ *                            invalid arguments: s <= 1, k_min > k_max, k < 1) */
+double covspec_uplink_bits(long long n_draft, int b_id, long long n_logit_draft, int b_logit);
+double covspec_downlink_bits(int all_accepted, int b_acc, int b_bonus, int b_rej, long long vocab,
+                             int b_logit_tar);
+double covspec_comm_latency(double bits, double bandwidth_hz, double snr_db);
+double covspec_ema_update(double p_hat, double eta, int k, int n_acc);
+int covspec_draft_length(int k, double p_hat, double t_rej, double p_low, double p_up, double t_ref,
+                         double s, int k_min, int k_max);
+
 /* Self-test of the kernels' bounded waits (no step of the paper).  Every wait inside the
  * tensor-core kernels gives up after a fixed number of polls, raises COVSPEC_ERR_TIMEOUT in the
  * device status word and lets the kernel return, so that a protocol fault cannot hang the GPU.

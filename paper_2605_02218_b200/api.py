@@ -27,6 +27,8 @@ EXPORTS = [
     "covspec_profile_begin", "covspec_profile_end", "covspec_profile_stage_count",
     "covspec_profile_stage_name", "covspec_query_score_static", "covspec_selftest_wait_timeout",
     "covspec_correct", "covspec_fanout", "covspec_branch_candidates",
+    "covspec_uplink_bits", "covspec_downlink_bits", "covspec_comm_latency", "covspec_ema_update",
+    "covspec_draft_length",
 ]
 STATIC_MAX_BATCH = 256
 STATIC_MAX_QUERY_ELEMS = 1 << 20
@@ -92,6 +94,15 @@ def load_library():
     lib.covspec_get_device_status.argtypes = [vp, vp]
     lib.covspec_selftest_wait_timeout.argtypes = [vp, vp]
     lib.covspec_fanout.argtypes = [C.c_int, C.c_double, C.c_int]
+    lib.covspec_uplink_bits.argtypes = [C.c_longlong, C.c_int, C.c_longlong, C.c_int]
+    lib.covspec_uplink_bits.restype = C.c_double
+    lib.covspec_downlink_bits.argtypes = [C.c_int, C.c_int, C.c_int, C.c_int, C.c_longlong, C.c_int]
+    lib.covspec_downlink_bits.restype = C.c_double
+    lib.covspec_comm_latency.argtypes = [C.c_double, C.c_double, C.c_double]
+    lib.covspec_comm_latency.restype = C.c_double
+    lib.covspec_ema_update.argtypes = [C.c_double, C.c_double, C.c_int, C.c_int]
+    lib.covspec_ema_update.restype = C.c_double
+    lib.covspec_draft_length.argtypes = [C.c_int] + [C.c_double] * 6 + [C.c_int, C.c_int]
     lib.covspec_branch_candidates.argtypes = [C.c_int, C.c_int, C.c_int, C.c_longlong, vp, vp, vp, C.c_int, vp, vp]
     lib.covspec_correct.argtypes = [C.c_int, C.c_int, C.c_int, C.c_longlong, vp, vp, vp, vp, C.c_float,
                                     vp, vp, vp, vp, vp, vp]

@@ -950,6 +950,40 @@ int covspec_correct(int logit_dtype, int rows, int vocab, long long ld, const vo
   return COVSPEC_OK;
 }
 
+double covspec_uplink_bits(long long n_draft, int b_id, long long n_logit_draft, int b_logit) {
+  return (double)n_draft * b_id + (double)n_logit_draft * b_logit;
+}
+
+double covspec_downlink_bits(int all_accepted, int b_acc, int b_bonus, int b_rej, long long vocab,
+                             int b_logit_tar) {
+  return all_accepted ? (double)b_acc + b_bonus : (double)b_rej + (double)vocab * b_logit_tar;
+}
+
+double covspec_comm_latency(double bits, double bandwidth_hz, double snr_db) {
+  return bits / (bandwidth_hz * log2(1.0 + pow(10.0, snr_db / 10.0)));
+}
+
+double covspec_ema_update(double p_hat, double eta, int k, int n_acc) {
+  if (n_acc < 0) n_acc = 0;
+  if (n_acc > k) n_acc = k;
+  for (int i = 0; i < n_acc; ++i) p_hat = (1.0 - eta) * p_hat + eta;
+  for (int i = n_acc; i < k; ++i) p_hat = (1.0 - eta) * p_hat;
+  return p_hat;
+}
+
+int covspec_draft_length(int k, double p_hat, double t_rej, double p_low, double p_up, double t_ref,
+                         double s, int k_min, int k_max) {
+  if (k < 1 || !(s > 1.0) || k_min > k_max || k_min < 1) return COVSPEC_ERR_ARG;
+  int phi = 0;
+  if (p_hat <= p_low) phi = -1;
+  else if (p_hat >= p_up && t_rej <= t_ref) phi = 1;
+  double x = phi < 0 ? (double)k / s : phi > 0 ? (double)k * s : (double)k;
+  long long r = (long long)floor(x + 0.5);
+  if (r > k_max) r = k_max;
+  if (r < k_min) r = k_min;
+  return (int)r;
+}
+
 int covspec_fanout(int f0, double rho, int j) {
   if (f0 < 0 || j < 0 || !(rho > 0.0 && rho < 1.0)) return COVSPEC_ERR_ARG;
   return (int)ceil((double)f0 * pow(rho, (double)j) - 1e-9);
