@@ -404,37 +404,30 @@ energy_kernel(const ReqPlan* __restrict__ plan, const float* __restrict__ q,
   const float* usrc = ub + (size_t)blockIdx.y * kPMax * kPMax;
   for (int e = tid; e < w * nbot; e += blockDim.x) us[e] = usrc[e];
   __syncthreads();
+  __shared__ float rowbuf[8][2 * kPMax];                 // this warp's rows of Y' and Q
+  float* ys = rowbuf[warp];
+  float* qs = ys + kPMax;
   for (int rr = warp; rr < nrows; rr += 8) {
     const float* yrow = yn + ((size_t)rp.presel_off + row0 + rr) * kPMax;
     const float* qrow = q + ((size_t)rp.presel_off + row0 + rr) * kPMax;
-    // total over all p basis vectors; the window part of both rows stays in registers
+    // total over all p basis vectors; both rows are staged for the window sums
     float total = 0.f;
-    float yw[(kPMax + 31) / 32], qw[(kPMax + 31) / 32];
-#pragma unroll
-    for (int t = 0; t < (kPMax + 31) / 32; ++t) {
-      int c = lane + 32 * t;
-      float yv = c < p ? yrow[c] : 0.f, qv = c < p ? qrow[c] : 0.f;
+    __syncwarp();
+    for (int c = lane; c < p; c += 32) {
+      float yv = yrow[c], qv = qrow[c];
+      ys[c] = yv; qs[c] = qv;
       total += yv * qv;
-      yw[t] = yv; qw[t] = qv;
     }
     total = warp_sum(total);
-    // discarded Ritz pairs: lanes over k, window components broadcast from the owning lane
+    __syncwarp();
+    // discarded Ritz pairs: lanes over k, window components broadcast from shared memory
     float sub_ = 0.f;
-    for (int k0 = 0; k0 < nbot; k0 += 32) {
-      int k = k0 + lane;
+    for (int k = lane; k < nbot; k += 32) {
       float ya = 0.f, qa = 0.f;
-#pragma unroll
-      for (int t = 0; t < (kPMax + 31) / 32; ++t) {
-        int cbase = 32 * t;
-        if (cbase + 31 < w0 || cbase >= p) continue;    // chunk entirely outside the window
-        for (int l = 0; l < 32; ++l) {
-          int c = cbase + l;
-          float yv = __shfl_sync(0xffffffffu, yw[t], l), qv = __shfl_sync(0xffffffffu, qw[t], l);
-          if (c >= w0 && c < p && k < nbot) {
-            float u = us[(c - w0) * nbot + k];
-            ya += yv * u; qa += qv * u;
-          }
-        }
+      for (int j = 0; j < w; ++j) {
+        float u = us[j * nbot + k];
+        ya += ys[w0 + j] * u;
+        qa += qs[w0 + j] * u;
       }
       sub_ += ya * qa;
     }
