@@ -4,9 +4,11 @@
 //   Kp = X_tile * Wk[heads]^T           tcgen05.mma kind::f16, 128 x 256 accumulator in TMEM,
 //                                       operands streamed by TMA through a shared-memory ring
 //   per token and head: ||Kp||^2        epilogue warps read TMEM, keep the norm in float32 and
-//                                       restage Kp as bf16 hi + lo K-major tiles in shared memory
+//                                       restage Kp, 64 features at a time, as bf16 hi + lo K-major
+//                                       tiles in shared memory
 //   logits = Kp * Qn[head]^T            second tcgen05.mma against the unit-length query elements,
-//                                       as hi*hi + lo*hi + hi*lo so that bf16 staging costs ~2^-16
+//                                       as hi*hi + lo*hi + hi*lo so that bf16 staging costs ~2^-16,
+//                                       accumulated over the two halves of the head in TMEM
 //   S^query = max_j,h logits / ||Kp||   row max in registers, atomic max into the score array
 // so the projected embeddings never leave the SM.  MODE 1 reuses the main loop for the query side:
 // Qp = Q * Wq^T, normalised per head and written as bf16 for MODE 0 to consume.
@@ -25,18 +27,23 @@ constexpr int kTileM = 128;            // tokens per tile (UMMA M)
 constexpr int kTileN = 256;            // projected features per pass: one pair of heads (UMMA N)
 constexpr int kHeadDim = 128;
 constexpr int kBK = 64;                // bf16 elements per k-chunk = one 128-byte swizzle row
-constexpr int kStages = 3;
+// The ring is bound by how far ahead of their use the loads are issued (2 -> 3 stages: -25 %), so
+// the projection is restaged half a head (64 features) at a time: its staging area shrinks from
+// 64 KB to 32 KB and a fourth stage fits.
+constexpr int kStages = 4;
 constexpr int kTT = 64;                // query elements per logits tile (UMMA N of the 2nd product)
+constexpr int kHalf = 64;              // features restaged at a time (one 128-byte swizzle row)
+constexpr int kLogitSlots = 4;         // logits tiles that accumulate across the two halves
 constexpr int kBytesA = kTileM * kBK * 2;          // 16 KB
 constexpr int kBytesB = kTileN * kBK * 2;          // 32 KB
 constexpr int kBytesStage = kBytesA + kBytesB;
-constexpr int kBytesKp = kTileM * kHeadDim * 2;    // 32 KB: two k-blocks of [128 x 64]; hi and lo
-constexpr int kBytesQ = kTT * kHeadDim * 2;        // 16 KB: two k-blocks of [64 x 64]; hi and lo
-// The query tiles (hi + lo = 32 KB) travel through the same ring slots as the main-loop chunks.
+constexpr int kBytesKp = kTileM * kHalf * 2;       // 16 KB: [128 x 64] of one half head; hi and lo
+constexpr int kBytesQ = kTT * kHalf * 2;           // 8 KB: [64 x 64] of one half head; hi and lo
+// The query sub-tiles (hi + lo = 16 KB) travel through the same ring slots as the main-loop chunks.
 constexpr int kSmemBytes = kStages * kBytesStage + 2 * kBytesKp + 1024 /*barriers*/ +
                            1024 /*alignment slack*/;
 constexpr int kTmemCols = 512;
-constexpr int kLogitCol = 256;         // logits tiles live at columns 256 + 64 * buffer
+constexpr int kLogitCol = 256;         // logits tiles live at columns 256 + 64 * slot
 
 struct Params {
   const ReqPlan* plan;
@@ -72,8 +79,8 @@ relevance_tc_kernel(const __grid_constant__ CUtensorMap map_a,   // X (MODE 0) o
   uint64_t* acc_empty = acc_full + 1;
   uint64_t* kp_ready = acc_full + 2;
   uint64_t* kp_free = acc_full + 3;
-  uint64_t* logit_full = acc_full + 8;   // [2]
-  uint64_t* logit_empty = acc_full + 10; // [2]
+  uint64_t* logit_full = acc_full + 4;   // [kLogitSlots]
+  uint64_t* logit_empty = acc_full + 8;  // [kLogitSlots]
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_full + 12);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
@@ -85,7 +92,7 @@ relevance_tc_kernel(const __grid_constant__ CUtensorMap map_a,   // X (MODE 0) o
     mbar_init(acc_empty, 128);
     mbar_init(kp_ready, 128);
     mbar_init(kp_free, 1);
-    for (int i = 0; i < 2; ++i) {
+    for (int i = 0; i < kLogitSlots; ++i) {
       mbar_init(&logit_full[i], 1); mbar_init(&logit_empty[i], 128);
     }
     *abort_flag = 0;
@@ -145,22 +152,24 @@ relevance_tc_kernel(const __grid_constant__ CUtensorMap map_a,   // X (MODE 0) o
             tma_load_2d(dst + kBytesA, &map_b, kc * kBK, hp * kTileN, &full[s]);
           }
           if (MODE == 0 && ok) {
-            // query tiles of this head pair use the next ring slots: [hi kb0][hi kb1][lo kb0][lo kb1]
+            // query sub-tiles of this head pair use the next ring slots, in the order the MMA issuer
+            // consumes them: head, group of up to kLogitSlots tiles, half, tile; one slot holds the
+            // [64 x 64] hi block followed by the lo block
             int heads = min(2, prm.n_heads - 2 * hp);
             int ntt = (T + kTT - 1) / kTT;
             for (int h = 0; h < heads && ok; ++h)
-              for (int tt = 0; tt < ntt; ++tt, ++it) {
-                int s = it % kStages;
-                uint32_t ph = (it / kStages) & 1u;
-                if (!(ok = mbar_wait(&empty[s], ph ^ 1u, abort_flag))) break;
-                mbar_expect_tx(&full[s], 2 * kBytesQ);
-                uint32_t dst = smem_u32(stage_base + s * kBytesStage);
-                int col = (2 * hp + h) * kHeadDim, y = txt0 + tt * kTT;
-                tma_load_2d(dst, &map_q, col, y, &full[s]);
-                tma_load_2d(dst + kBytesQ / 2, &map_q, col + kBK, y, &full[s]);
-                tma_load_2d(dst + kBytesQ, &map_ql, col, y, &full[s]);
-                tma_load_2d(dst + kBytesQ + kBytesQ / 2, &map_ql, col + kBK, y, &full[s]);
-              }
+              for (int g0 = 0; g0 < ntt && ok; g0 += kLogitSlots)
+                for (int half = 0; half < 2 && ok; ++half)
+                  for (int tt = g0; tt < min(ntt, g0 + kLogitSlots); ++tt, ++it) {
+                    int s = it % kStages;
+                    uint32_t ph = (it / kStages) & 1u;
+                    if (!(ok = mbar_wait(&empty[s], ph ^ 1u, abort_flag))) break;
+                    mbar_expect_tx(&full[s], 2 * kBytesQ);
+                    uint32_t dst = smem_u32(stage_base + s * kBytesStage);
+                    int col = (2 * hp + h) * kHeadDim + half * kHalf, y = txt0 + tt * kTT;
+                    tma_load_2d(dst, &map_q, col, y, &full[s]);
+                    tma_load_2d(dst + kBytesQ, &map_ql, col, y, &full[s]);
+                  }
           }
         }
       }
@@ -171,7 +180,8 @@ relevance_tc_kernel(const __grid_constant__ CUtensorMap map_a,   // X (MODE 0) o
     if (lane == 0) {
       const uint32_t idesc1 = umma_idesc(kTileM, kTileN);
       const uint32_t idesc2 = umma_idesc(kTileM, kTT);
-      uint32_t it = 0, acc_it = 0, kp_it = 0, qi = 0;
+      uint32_t it = 0, acc_it = 0, kp_it = 0;
+      uint32_t slot_uses[kLogitSlots] = {0u, 0u, 0u, 0u};
       bool ok = true;
       for (int item = blockIdx.x; item < prm.n_items && ok; item += gridDim.x) {
         int row0, nrows, txt0, T, hp_begin, hp_end;
@@ -196,33 +206,36 @@ relevance_tc_kernel(const __grid_constant__ CUtensorMap map_a,   // X (MODE 0) o
           if (MODE == 0) {
             int heads = min(2, prm.n_heads - 2 * hp);
             int ntt = (T + kTT - 1) / kTT;
-            for (int h = 0; h < heads && ok; ++h, ++kp_it) {
-              if (!(ok = mbar_wait(kp_ready, kp_it & 1u, abort_flag))) break;
-              for (int tt = 0; tt < ntt; ++tt, ++qi, ++it) {
-                int s = it % kStages;
-                int buf = qi & 1;
-                if (!(ok = mbar_wait(&full[s], (it / kStages) & 1u, abort_flag))) break;
-                if (!(ok = mbar_wait(&logit_empty[buf], ((qi >> 1) & 1u) ^ 1u, abort_flag))) break;
-                tc_fence_after();
-                uint32_t kp_addr = smem_u32(kp_smem), q_addr = smem_u32(stage_base + s * kBytesStage);
-                // logits = Kp_hi Qn_hi^T + Kp_lo Qn_hi^T + Kp_hi Qn_lo^T
+            for (int h = 0; h < heads && ok; ++h)
+              for (int g0 = 0; g0 < ntt && ok; g0 += kLogitSlots) {
+                const int ng = min(ntt, g0 + kLogitSlots) - g0;
+                for (int half = 0; half < 2 && ok; ++half, ++kp_it) {
+                  // the epilogue has restaged features [64 half, 64 half + 64) of this head
+                  if (!(ok = mbar_wait(kp_ready, kp_it & 1u, abort_flag))) break;
+                  for (int slot = 0; slot < ng; ++slot, ++it) {
+                    int s = it % kStages;
+                    if (!(ok = mbar_wait(&full[s], (it / kStages) & 1u, abort_flag))) break;
+                    if (half == 0 &&
+                        !(ok = mbar_wait(&logit_empty[slot], (slot_uses[slot] & 1u) ^ 1u, abort_flag))) break;
+                    tc_fence_after();
+                    uint32_t kp_addr = smem_u32(kp_smem), q_addr = smem_u32(stage_base + s * kBytesStage);
+                    // logits += Kp_hi Qn_hi^T + Kp_lo Qn_hi^T + Kp_hi Qn_lo^T over this half's 64 features
 #pragma unroll
-                for (int term = 0; term < 3; ++term) {
-                  uint32_t a0 = kp_addr + (term == 1 ? kBytesKp : 0);
-                  uint32_t b0 = q_addr + (term == 2 ? kBytesQ : 0);
+                    for (int term = 0; term < 3; ++term) {
+                      uint64_t adesc = umma_desc(kp_addr + (term == 1 ? kBytesKp : 0));
+                      uint64_t bdesc = umma_desc(q_addr + (term == 2 ? kBytesQ : 0));
 #pragma unroll
-                  for (int ks = 0; ks < kHeadDim / 16; ++ks) {
-                    uint64_t adesc = umma_desc(a0 + (ks >> 2) * (kBytesKp / 2)) + 2 * (ks & 3);
-                    uint64_t bdesc = umma_desc(b0 + (ks >> 2) * (kBytesQ / 2)) + 2 * (ks & 3);
-                    umma_bf16(tmem_base + kLogitCol + buf * kTT, adesc, bdesc, idesc2, (term | ks) != 0);
+                      for (int ks = 0; ks < kHalf / 16; ++ks)
+                        umma_bf16(tmem_base + kLogitCol + slot * kTT, adesc + 2 * ks, bdesc + 2 * ks, idesc2,
+                                  (half | term | ks) != 0);
+                    }
+                    umma_commit(&empty[s]);
+                    if (half == 1) { umma_commit(&logit_full[slot]); ++slot_uses[slot]; }
                   }
+                  if (!ok) break;
+                  umma_commit(kp_free);
                 }
-                umma_commit(&empty[s]);
-                umma_commit(&logit_full[buf]);
               }
-              if (!ok) break;
-              umma_commit(kp_free);
-            }
           }
         }
       }
@@ -232,7 +245,8 @@ relevance_tc_kernel(const __grid_constant__ CUtensorMap map_a,   // X (MODE 0) o
     // ---------------------------------------------------------------- epilogue (warps 0-3)
     const int r = warp * 32 + lane;                        // token row inside the tile = TMEM lane
     const uint32_t t_lane = tmem_base + ((uint32_t)(warp * 32) << 16);
-    uint32_t acc_it = 0, kp_it = 0, qi = 0;
+    uint32_t acc_it = 0, kp_it = 0;
+    uint32_t slot_uses[kLogitSlots] = {0u, 0u, 0u, 0u};
     bool ok = true;
     for (int item = blockIdx.x; item < prm.n_items && ok; item += gridDim.x) {
       int row0, nrows, txt0, T, hp_begin, hp_end;
@@ -243,59 +257,69 @@ relevance_tc_kernel(const __grid_constant__ CUtensorMap map_a,   // X (MODE 0) o
         if (!(ok = mbar_wait(acc_full, acc_it & 1u, abort_flag))) break;
         tc_fence_after();
         int heads = min(2, prm.n_heads - 2 * hp);
-        for (int h = 0; h < heads && ok; ++h, ++kp_it) {
+        for (int h = 0; h < heads && ok; ++h) {
           float ss = 0.f;
           if (MODE == 0) {
-            if (!(ok = mbar_wait(kp_free, (kp_it & 1u) ^ 1u, abort_flag))) break;
-#pragma unroll 1
-            for (int c4 = 0; c4 < 4; ++c4) {
-              float v[32];
-              tmem_ld32(t_lane + h * kHeadDim + c4 * 32, v);
-              uint32_t pk[16], pl[16];
-#pragma unroll
-              for (int e = 0; e < 16; ++e) {
-                float a = v[2 * e], b = v[2 * e + 1];
-                ss += a * a + b * b;
-                __nv_bfloat162 hi = __floats2bfloat162_rn(a, b);
-                pk[e] = *reinterpret_cast<uint32_t*>(&hi);
-                pl[e] = pack_bf16(a - __low2float(hi), b - __high2float(hi));
-              }
-              uint8_t* rowp = kp_smem + (c4 >> 1) * (kBytesKp / 2) + r * 128;
-#pragma unroll
-              for (int q = 0; q < 4; ++q) {
-                int chunk = ((c4 & 1) * 4 + q) ^ (r & 7);
-                *reinterpret_cast<uint4*>(rowp + chunk * 16) =
-                    make_uint4(pk[4 * q], pk[4 * q + 1], pk[4 * q + 2], pk[4 * q + 3]);
-                *reinterpret_cast<uint4*>(rowp + kBytesKp + chunk * 16) =
-                    make_uint4(pl[4 * q], pl[4 * q + 1], pl[4 * q + 2], pl[4 * q + 3]);
-              }
-            }
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-            tc_fence_before();
-            mbar_arrive(kp_ready);
-            if (h == heads - 1) mbar_arrive(acc_empty);    // the accumulator is fully drained
-            nonfinite |= !(ss <= 3.402823466e38f);
+            const int ntt = (T + kTT - 1) / kTT;
             float inv = 0.f;
-            if (ss > 1.17549435e-38f) { inv = rsqrtf(ss); inv = inv * (1.5f - 0.5f * ss * inv * inv); }
-            int ntt = (T + kTT - 1) / kTT;
-            for (int tt = 0; tt < ntt; ++tt, ++qi) {
-              int buf = qi & 1;
-              if (!(ok = mbar_wait(&logit_full[buf], (qi >> 1) & 1u, abort_flag))) break;
-              tc_fence_after();
+            for (int g0 = 0; g0 < ntt && ok; g0 += kLogitSlots) {
+              const int ng = min(ntt, g0 + kLogitSlots) - g0;
+              for (int half = 0; half < 2 && ok; ++half, ++kp_it) {
+                // restage features [64 half, 64 half + 64) of this head as bf16 hi + lo
+                if (!(ok = mbar_wait(kp_free, (kp_it & 1u) ^ 1u, abort_flag))) break;
 #pragma unroll 1
-              for (int c2 = 0; c2 < 2; ++c2) {
-                float v[32];
-                tmem_ld32(t_lane + kLogitCol + buf * kTT + c2 * 32, v);
-                int jbase = tt * kTT + c2 * 32;
+                for (int c2 = 0; c2 < 2; ++c2) {
+                  float v[32];
+                  tmem_ld32(t_lane + h * kHeadDim + half * kHalf + c2 * 32, v);
+                  uint32_t pk[16], pl[16];
 #pragma unroll
-                for (int e = 0; e < 32; ++e)
-                  if (jbase + e < T) {
-                    nonfinite |= v[e] != v[e];
-                    best = fmaxf(best, v[e] * inv);
+                  for (int e = 0; e < 16; ++e) {
+                    float a = v[2 * e], b = v[2 * e + 1];
+                    if (g0 == 0) ss += a * a + b * b;
+                    __nv_bfloat162 hi = __floats2bfloat162_rn(a, b);
+                    pk[e] = *reinterpret_cast<uint32_t*>(&hi);
+                    pl[e] = pack_bf16(a - __low2float(hi), b - __high2float(hi));
                   }
+                  uint8_t* rowp = kp_smem + r * 128;
+#pragma unroll
+                  for (int q = 0; q < 4; ++q) {
+                    int chunk = (c2 * 4 + q) ^ (r & 7);
+                    *reinterpret_cast<uint4*>(rowp + chunk * 16) =
+                        make_uint4(pk[4 * q], pk[4 * q + 1], pk[4 * q + 2], pk[4 * q + 3]);
+                    *reinterpret_cast<uint4*>(rowp + kBytesKp + chunk * 16) =
+                        make_uint4(pl[4 * q], pl[4 * q + 1], pl[4 * q + 2], pl[4 * q + 3]);
+                  }
+                }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                tc_fence_before();
+                mbar_arrive(kp_ready);
+                // the accumulator is fully drained after the last restaging of the last head
+                if (h == heads - 1 && half == 1 && g0 + kLogitSlots >= ntt) mbar_arrive(acc_empty);
               }
-              tc_fence_before();
-              mbar_arrive(&logit_empty[buf]);
+              if (!ok) break;
+              if (g0 == 0) {
+                nonfinite |= !(ss <= 3.402823466e38f);
+                if (ss > 1.17549435e-38f) { inv = rsqrtf(ss); inv = inv * (1.5f - 0.5f * ss * inv * inv); }
+              }
+              for (int slot = 0; slot < ng; ++slot) {
+                if (!(ok = mbar_wait(&logit_full[slot], slot_uses[slot] & 1u, abort_flag))) break;
+                ++slot_uses[slot];
+                tc_fence_after();
+#pragma unroll 1
+                for (int c2 = 0; c2 < 2; ++c2) {
+                  float v[32];
+                  tmem_ld32(t_lane + kLogitCol + slot * kTT + c2 * 32, v);
+                  int jbase = (g0 + slot) * kTT + c2 * 32;
+#pragma unroll
+                  for (int e = 0; e < 32; ++e)
+                    if (jbase + e < T) {
+                      nonfinite |= v[e] != v[e];
+                      best = fmaxf(best, v[e] * inv);
+                    }
+                }
+                tc_fence_before();
+                mbar_arrive(&logit_empty[slot]);
+              }
             }
           } else {
             // MODE 1: unit-length bf16 head slice of the projected query element to global memory.
