@@ -41,6 +41,9 @@ SMALL = [
     # video-like near-duplicate frames: low-rank dependency dominates
     dict(seed=17, dtype=torch.bfloat16, batch=2, n_vis=1536, n_txt=16, d=256, n_heads=2, rank=16,
          kind="video", keep=128),
+    # more query elements than the four logits tiles one pass of the relevance kernel holds
+    dict(seed=18, dtype=torch.bfloat16, batch=2, n_vis=(130, 400), n_txt=(257, 330), d=128, n_heads=3,
+         rank=8, keep_ratio=0.2),
 ]
 
 
