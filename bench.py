@@ -32,7 +32,7 @@ from paper_2605_02218_b200 import workloads
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one visual-side relevance_tc_kernel launch (ncu,
 # profiles/relevance_tc_kernel_c2.md); None where no capture of the current kernel exists.
-NCU_TRAFFIC_BYTES = {"c2": 55.675e6, "correct_per_row": 343.9e6 / 512}   # profiles/correct_kernel_vocab152k.md
+NCU_TRAFFIC_BYTES = {"c2": 55.62e6, "correct_per_row": 343.9e6 / 512}   # profiles/correct_kernel_vocab152k.md
 
 METRIC = "visual_tokens_pruned_per_s"
 UNIT = "tokens/s"
