@@ -136,6 +136,15 @@ int covspec_select(covspec_ctx* ctx, const covspec_problem* p, const float* s_fu
 int covspec_compact(covspec_ctx* ctx, const covspec_problem* p, const int* keep_idx,
                     const int* keep_offsets, void* out_hidden, int* out_pos, void* stream);
 
+/* The same gather for any other per-token tensor that must follow the kept tokens (the K or V rows of
+ * a layer when the pruning is applied after a prefill, position ids, ...): src is laid out like X,
+ * one row of row_bytes (a multiple of 16; both bases 16-byte aligned) per visual token;
+ * out[keep_offsets[b] + k, :] = src[vis_offsets[b] + keep_idx[..], :], bit copies.  The paper selects
+ * before the draft prefill, so its own pipeline has only the hidden states to compact. */
+int covspec_compact_rows(covspec_ctx* ctx, const covspec_problem* p, const int* keep_idx,
+                         const int* keep_offsets, const void* src, long long row_bytes, void* out,
+                         void* stream);
+
 /* The whole path, Eq. 10 through the compacted buffer, in one call.  out_hidden device
  * [sum B_vis, d]; keep_idx device [sum B_vis]; keep_offsets host [batch+1] (may be NULL). */
 int covspec_prune(covspec_ctx* ctx, const covspec_problem* p, void* out_hidden, int* keep_idx,

@@ -22,7 +22,7 @@ HEAD_REDUCE = {"max": 0, "mean": 1}
 EXPORTS = [
     "covspec_default_config", "covspec_budgets", "covspec_plan_sizes", "covspec_prune_init",
     "covspec_prune_destroy", "covspec_workspace_bytes", "covspec_score", "covspec_select",
-    "covspec_compact", "covspec_prune", "covspec_get_device_status",
+    "covspec_compact", "covspec_compact_rows", "covspec_prune", "covspec_get_device_status",
     "covspec_last_launch_count", "covspec_strerror", "covspec_last_cuda_error",
     "covspec_profile_begin", "covspec_profile_end", "covspec_profile_stage_count",
     "covspec_profile_stage_name", "covspec_query_score_static", "covspec_selftest_wait_timeout",
@@ -91,6 +91,7 @@ def load_library():
     lib.covspec_select.argtypes = [vp, C.POINTER(Problem), fp, vp, ip, vp, fp, vp]
     lib.covspec_compact.argtypes = [vp, C.POINTER(Problem), vp, ip, vp, vp, vp]
     lib.covspec_prune.argtypes = [vp, C.POINTER(Problem), vp, vp, ip, vp]
+    lib.covspec_compact_rows.argtypes = [vp, C.POINTER(Problem), vp, ip, vp, C.c_longlong, vp, vp]
     lib.covspec_get_device_status.argtypes = [vp, vp]
     lib.covspec_selftest_wait_timeout.argtypes = [vp, vp]
     lib.covspec_fanout.argtypes = [C.c_int, C.c_double, C.c_int]
@@ -295,6 +296,20 @@ class Pruner:
         if st:
             raise CovspecError(st, "covspec_compact")
         return out, pos
+
+    def compact_rows(self, m: _Marshalled, keep_idx: torch.Tensor, keep_offsets: np.ndarray,
+                     src: torch.Tensor):
+        """covspec_compact_rows: gathers the kept tokens' rows of another per-token tensor
+        (first dimension = visual tokens, like X)."""
+        assert src.is_cuda and src.is_contiguous() and src.shape[0] == int(m.vis[-1])
+        ko, ko_p = _i32(keep_offsets)
+        row_bytes = src[0].numel() * src.element_size()
+        out = torch.empty((int(ko[-1]),) + tuple(src.shape[1:]), dtype=src.dtype, device=src.device)
+        st = self.lib.covspec_compact_rows(self._ctx, C.byref(m.problem), _ptr(keep_idx), ko_p, _ptr(src),
+                                           row_bytes, _ptr(out), _stream())
+        if st:
+            raise CovspecError(st, "covspec_compact_rows")
+        return out
 
     def prune(self, m: _Marshalled, out: Optional[torch.Tensor] = None,
               keep_idx: Optional[torch.Tensor] = None):

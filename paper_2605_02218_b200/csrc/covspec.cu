@@ -841,6 +841,25 @@ int covspec_compact(covspec_ctx* ctx, const covspec_problem* p, const int* keep_
   return compact_impl(ctx, p, keep_idx, out_hidden, out_pos, s);
 }
 
+int covspec_compact_rows(covspec_ctx* ctx, const covspec_problem* p, const int* keep_idx,
+                         const int* keep_offsets, const void* src, long long row_bytes, void* out,
+                         void* stream) {
+  if (!ctx || !p || !keep_idx || !keep_offsets || !src || !out) return COVSPEC_ERR_ARG;
+  if (row_bytes < 16 || row_bytes % 16 != 0 || row_bytes / 16 > 0x7fffffffll) return COVSPEC_ERR_SHAPE;
+  if ((reinterpret_cast<uintptr_t>(src) | reinterpret_cast<uintptr_t>(out)) & 15) return COVSPEC_ERR_ARG;
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  ctx->launches = 0;
+  int st = get_plan(ctx, p, s);
+  if (st) return st;
+  if (memcmp(keep_offsets, ctx->plan.keep_offsets.data(), sizeof(int) * (p->batch + 1)))
+    return COVSPEC_ERR_SHAPE;
+  gather_rows_kernel<<<(unsigned)ctx->plan.total_keep, 256, 0, s>>>(
+      reinterpret_cast<const uint4*>(src), keep_idx, ctx->d_plan, p->batch, 0, (int)(row_bytes / 16),
+      reinterpret_cast<uint4*>(out), nullptr);
+  LAUNCH_CHECK(ctx);
+  return COVSPEC_OK;
+}
+
 int covspec_prune(covspec_ctx* ctx, const covspec_problem* p, void* out_hidden, int* keep_idx,
                   int* keep_offsets, void* stream) {
   if (!ctx || !p || !out_hidden || !keep_idx) return COVSPEC_ERR_ARG;

@@ -171,6 +171,27 @@ def test_device_status_reports_nonfinite():
     assert len(np.unique(k)) == 8 and k.min() >= 0 and k.max() < 64
 
 
+def test_compact_rows_follows_the_keep_set():
+    # K / V rows (or any per-token tensor) gathered with the same kept indices, bit for bit
+    from paper_2605_02218_b200 import api
+    wl = workloads.make_workload("kv", seed=35, dtype=torch.bfloat16, batch=3, n_vis=(90, 300), n_txt=5,
+                                 d=64, n_heads=0, rank=4, keep_ratio=0.25).to("cuda:0")
+    pr = api.Pruner.for_workload(wl)
+    m = pr.marshal(wl)
+    out, keep_idx, ko = pr.prune(m)
+    kv = torch.randn(wl.total_vis, 2, 3, 40, device="cuda:0").to(torch.bfloat16)     # [token, k/v, head, dim]
+    pos = torch.arange(wl.total_vis, device="cuda:0", dtype=torch.int32).repeat_interleave(4).view(-1, 4).contiguous()
+    got_kv = pr.compact_rows(m, keep_idx, ko, kv)
+    got_pos = pr.compact_rows(m, keep_idx, ko, pos)
+    pr.check_device_status()
+    k = keep_idx.cpu().numpy().astype(np.int64)
+    rows = np.concatenate([k[ko[b]:ko[b + 1]] + int(wl.vis_offsets[b]) for b in range(wl.batch)])
+    idx = torch.from_numpy(rows).to("cuda:0")
+    assert torch.equal(got_kv, kv[idx]) and torch.equal(got_pos, pos[idx])
+    with pytest.raises(api.CovspecError):
+        pr.compact_rows(m, keep_idx, ko, kv[:, 0, 0, :3].contiguous())              # 6-byte rows
+
+
 def test_bounded_wait_reports_timeout():
     # A wait on a barrier that nothing signals runs out after its poll limit: the kernel returns,
     # the status word says so, and the context keeps working.
