@@ -208,3 +208,46 @@ def energy_ambiguity(Z_M, r, delta=1e-3):
         return np.zeros(Z_M.shape[1])
     near = (np.abs(lam - lam[r - 1]) <= delta * lam[0]) | (np.abs(lam - lam[r]) <= delta * lam[0])
     return np.sum((Vt[near].T ** 2) * lam[near][None, :], axis=1)
+
+
+# ----------------------------------------------------------------------------------------------
+# Variant (not in the paper): greedy pivoted low-rank selection
+# ----------------------------------------------------------------------------------------------
+def greedy_lowrank_select(Z_M, B, follow=None, tol=0.0):
+    """Alternative to Eq. 14-15 that the library offers as `lowrank_mode = 1`: pick, B times, the
+    preselected token whose representation has the largest residual energy after projecting out
+    the span of the tokens already picked, then update the residuals (pivoted Cholesky of
+    G = Z_M^T Z_M: argmax of the residual diagonal, rank-1 update).  Ties go to the lower index; a
+    picked token is never picked again.
+
+    Returns (picks in order, residual energy of every pick at the time it was picked).  With
+    `follow` (a pick sequence from another implementation) the same loop takes that sequence
+    instead of its own argmax and returns, as a third value, whether every followed pick was within
+    tol * max(diag G) of the largest residual at its step (several orders are valid at near-ties)."""
+    Z = np.asarray(Z_M, dtype=np.float64)
+    G = Z.T @ Z
+    M = G.shape[0]
+    e = np.diag(G).copy()
+    scale = e.max() if M else 0.0
+    C = np.zeros((0, M))
+    picked = np.zeros(M, dtype=bool)
+    picks, energies, valid = [], [], True
+    for k in range(B):
+        cand = np.where(picked, -np.inf, e)
+        best = int(np.argmax(cand))                      # first index of the maximum
+        if follow is not None:
+            p = int(follow[k])
+            if picked[p] or cand[p] < cand[best] - tol * scale:
+                valid = False
+        else:
+            p = best
+        picks.append(p)
+        energies.append(float(e[p]))
+        picked[p] = True
+        if e[p] > 0.0:
+            c = (G[:, p] - C.T @ C[:, p]) / np.sqrt(e[p])
+            C = np.vstack([C, c[None, :]])
+            e = e - c * c
+    if follow is not None:
+        return np.array(picks), np.array(energies), valid
+    return np.array(picks), np.array(energies)

@@ -366,3 +366,40 @@ def test_forced_preselect_and_ambiguity():
     Zt = np.zeros((4, 3))
     Zt[0, 0], Zt[1, 1], Zt[2, 2] = 3.0, 2.0, 2.0
     np.testing.assert_allclose(O.energy_ambiguity(Zt, 2), [0.0, 4.0, 4.0])
+
+
+# ------------------------------------------------------------------ greedy pivoted variant
+def test_greedy_lowrank_hand_and_properties():
+    # columns e1*3, e1*2, e2*1, (e1+e2): norms^2 9, 4, 1, 2.  First pick 0 (9).  Residuals after
+    # projecting out e1: 0, 0, 1, 1 -> tie between 2 and 3 goes to the lower index 2.
+    Z = np.array([[3.0, 2.0, 0.0, 1.0], [0.0, 0.0, 1.0, 1.0]])
+    picks, en = O.greedy_lowrank_select(Z, 2)
+    assert picks.tolist() == [0, 2] and np.allclose(en, [9.0, 1.0])
+    rng = np.random.default_rng(11)
+    Z = rng.normal(size=(20, 12))
+    picks, en = O.greedy_lowrank_select(Z, 6)
+    assert len(set(picks.tolist())) == 6
+    assert np.all(np.diff(en) <= 1e-12)                  # residual energies never grow
+    # the energies are the squared pivots of a QR with column pivoting: their product is the squared
+    # volume of the picked columns
+    sub = Z[:, picks]
+    assert np.isclose(np.prod(en), np.linalg.det(sub.T @ sub), rtol=1e-9)
+    # each pick is the brute-force argmax of the distance to the span of the previous picks
+    for k in range(1, 6):
+        Q, _ = np.linalg.qr(Z[:, picks[:k]])
+        resid = ((Z - Q @ (Q.T @ Z)) ** 2).sum(0)
+        resid[picks[:k]] = -1
+        assert int(np.argmax(resid)) == picks[k]
+    # following its own sequence is valid; following a bad one is not
+    assert O.greedy_lowrank_select(Z, 6, follow=picks)[2]
+    bad = picks.copy(); bad[0] = int(np.argmin((Z ** 2).sum(0)))
+    assert not O.greedy_lowrank_select(Z, 6, follow=bad)[2]
+
+
+def test_greedy_lowrank_exhausted_rank():
+    # rank 2 data, 4 picks: after two picks every residual is ~0 and the remaining picks are the
+    # lowest unpicked indices
+    rng = np.random.default_rng(12)
+    Z = rng.normal(size=(2, 6))
+    picks, en = O.greedy_lowrank_select(Z, 4)
+    assert len(set(picks.tolist())) == 4 and np.all(np.abs(en[2:]) < 1e-12 * en[0])
