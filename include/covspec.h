@@ -76,6 +76,10 @@ typedef struct {
   int relevance_path;  /* 0: Eq. 10 on the tensor cores (tcgen05) whenever the configuration allows
                           (bf16, 128-wide heads, max over heads, d >= 64), else the CUDA-core path;
                           1: always the CUDA-core path                                            */
+  int lowrank_mode;    /* 0: energy in the top-r singular subspace (Eq. 14-15, the paper's criterion);
+                          1: greedy pivoted selection (not in the paper): pick B_vis times the token with
+                             the largest residual energy after projecting out the picked ones; needs
+                             M <= 16384 and B_vis <= 8192 per request                              */
 } covspec_config;
 
 /* One batch of requests (Sec. III-A notation in brackets). */

@@ -42,7 +42,7 @@ class Config(C.Structure):
         ("rank_cap", C.c_int), ("eig_iters", C.c_int), ("eig_oversample", C.c_int),
         ("max_batch", C.c_int), ("max_total_vis", C.c_longlong), ("max_total_txt", C.c_longlong),
         ("max_vis_per_req", C.c_int), ("max_presel_per_req", C.c_int),
-        ("max_total_presel", C.c_longlong), ("relevance_path", C.c_int),
+        ("max_total_presel", C.c_longlong), ("relevance_path", C.c_int), ("lowrank_mode", C.c_int),
     ]
 
 

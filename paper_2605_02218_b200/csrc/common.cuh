@@ -26,6 +26,7 @@ struct ReqPlan {
   int ptile_off;           // first 128-row tile of the request's subspace-iteration block
   int win;                 // basis vectors in the Rayleigh-Ritz window next to the cut at r
   long long g_off;         // float offset of the request's float32 Gram matrix (float32 inputs only)
+  long long c_off;         // float offset of the request's factor columns (greedy low-rank mode)
 };
 
 // One dense product C[m x n] = A[m x k] * op(B) handled by the tiled SIMT kernel.

@@ -15,6 +15,7 @@
 #include "correct_kernels.cuh"
 #include "eig_kernels.cuh"
 #include "gemm_simt.cuh"
+#include "greedy_kernels.cuh"
 #include "relevance_tc.cuh"
 #include "subspace_tc.cuh"
 #include "score_kernels.cuh"
@@ -97,6 +98,8 @@ struct covspec_ctx {
   float* Yf[2] = {nullptr, nullptr};     // float32 blocks before / after the last power step
   double* partial = nullptr;
   float *Lbuf = nullptr, *Ub = nullptr;
+  float* Cg = nullptr;                   // factor columns of the greedy low-rank mode
+  long long cg_cap = 0;
   CUtensorMap map_zg, map_gh, map_gl, map_y[2][2];
   // pinned staging for the plan upload
   char* h_stage = nullptr;
@@ -149,6 +152,7 @@ int validate_cfg(const covspec_config* c) {
   if (!(c->presel_factor >= 1.f) || !(c->rank_frac > 0.f) || c->rank_cap < 1) return COVSPEC_ERR_ARG;
   if (c->eig_iters < 1 || c->eig_oversample < 0) return COVSPEC_ERR_ARG;
   if (c->rank_cap + c->eig_oversample > kPMax) return COVSPEC_ERR_UNSUPPORTED;
+  if (c->lowrank_mode < 0 || c->lowrank_mode > 1) return COVSPEC_ERR_ARG;
   return COVSPEC_OK;
 }
 
@@ -191,7 +195,7 @@ int get_plan(covspec_ctx* ctx, const covspec_problem* p, cudaStream_t stream) {
   pl.n_stage2 = 0; pl.t_max = 0; pl.p_max = 0; pl.m_max = 0; pl.n_tiles = 0;
   pl.n_gram_tiles = 0; pl.n_ptiles = 0;
   pl.win_max = 0; pl.nbot_max = 0;
-  long long g_off = 0;
+  long long g_off = 0, c_off = 0;
   int n_max = 0;
   bool f32 = cfg.dtype == COVSPEC_F32;
   for (int b = 0; b < B; ++b) {
@@ -208,6 +212,7 @@ int get_plan(covspec_ctx* ctx, const covspec_problem* p, cudaStream_t stream) {
     r.gram_tile_off = pl.n_gram_tiles;
     r.ptile_off = pl.n_ptiles;
     r.g_off = g_off;
+    r.c_off = c_off;
     if (r.stage2) {
       r.p = r.r + cfg.eig_oversample;
       if (r.p > r.m) r.p = r.m;
@@ -216,6 +221,10 @@ int get_plan(covspec_ctx* ctx, const covspec_problem* p, cudaStream_t stream) {
       pl.n_gram_tiles += nt * (nt + 1) / 2;
       pl.n_ptiles += nt;
       if (f32) g_off += (long long)r.m * r.ldm;
+      if (cfg.lowrank_mode == 1) {
+        if (r.m > kGreedyMaxM || r.b_vis > kGreedyMaxB) return COVSPEC_ERR_UNSUPPORTED;
+        c_off += (long long)r.b_vis * r.m;
+      }
       r.win = r.p - r.r + std::min(32, r.r);
       if (r.win > r.p) r.win = r.p;
       pl.win_max = std::max(pl.win_max, r.win);
@@ -232,7 +241,7 @@ int get_plan(covspec_ctx* ctx, const covspec_problem* p, cudaStream_t stream) {
   pl.total_vis = p->vis_offsets[B]; pl.total_txt = p->txt_offsets[B];
   pl.total_keep = pl.keep_offsets[B]; pl.total_presel = pl.presel_offsets[B];
   if (pl.total_vis > cfg.max_total_vis || pl.total_txt > cfg.max_total_txt ||
-      n_max > cfg.max_vis_per_req || g_off > ctx->g_cap || pl.m_max > ctx->cfg.max_presel_per_req ||
+      n_max > cfg.max_vis_per_req || g_off > ctx->g_cap || c_off > ctx->cg_cap || pl.m_max > ctx->cfg.max_presel_per_req ||
       pl.total_presel > ctx->cfg.max_total_presel || pl.n_ptiles > ctx->cap_ptiles)
     return COVSPEC_ERR_WORKSPACE;
 
@@ -546,6 +555,16 @@ int select_impl(covspec_ctx* ctx, const covspec_problem* p, const float* s_fused
     }
     prof_mark(ctx, ST_GRAM, 1, s);
     prof_mark(ctx, ST_EIG, 0, s);
+    if (cfg.lowrank_mode == 1) {
+      // greedy pivoted selection instead of the subspace energies; it writes its own `energy`
+      greedy_select_kernel<<<B, kGreedyThreads, 0, s>>>(ctx->d_plan, ctx->Ghi, ctx->Glo, ctx->ld, ctx->Cg, energy);
+      LAUNCH_CHECK(ctx);
+      prof_mark(ctx, ST_EIG, 1, s);
+      prof_mark(ctx, ST_FINAL, 0, s);
+      final_select_kernel<<<B, 1024, 0, s>>>(energy, presel, ctx->d_plan, keep_idx, ctx->status);
+      LAUNCH_CHECK(ctx);
+      return COVSPEC_OK;
+    }
     sub::basis_init_kernel<<<gb, 256, 0, s>>>(ctx->d_plan, ctx->Yp[0][0], ctx->Yp[0][1], ctx->Yp[1][0],
                                               ctx->Yp[1][1], ctx->ld);
     LAUNCH_CHECK(ctx);
@@ -630,6 +649,7 @@ void covspec_default_config(covspec_config* c) {
   c->eig_iters = 5;
   c->eig_oversample = 32;
   c->relevance_path = 0;
+  c->lowrank_mode = 0;
 }
 
 int covspec_budgets(const covspec_config* cfg, int n, int keep, int* b_vis, int* m, int* r) {
@@ -706,6 +726,8 @@ int covspec_prune_init(const covspec_config* cfg, covspec_ctx** out) {
   long long o_part = carve(8ll * ctx->cap_ptiles * sub::kTriMax);
   long long o_lbuf = carve(4ll * c.max_batch * sub::kLbufStride);
   long long o_ub = carve(4ll * c.max_batch * kPMax * kPMax);
+  ctx->cg_cap = c.lowrank_mode == 1 ? (long long)c.max_total_presel * c.max_presel_per_req : 0;
+  long long o_cg = carve(4ll * ctx->cg_cap);
   ctx->ws_bytes = off;
   cudaError_t e = cudaMalloc(&ctx->ws, (size_t)off);
   if (e != cudaSuccess) {
@@ -736,6 +758,7 @@ int covspec_prune_init(const covspec_config* cfg, covspec_ctx** out) {
   ctx->partial = reinterpret_cast<double*>(w + o_part);
   ctx->Lbuf = reinterpret_cast<float*>(w + o_lbuf);
   ctx->Ub = reinterpret_cast<float*>(w + o_ub);
+  ctx->Cg = reinterpret_cast<float*>(w + o_cg);
   ctx->stage_bytes = round_up(sizeof(ReqPlan) * c.max_batch, 256) +
                      sizeof(GemmProb) * (long long)T_COUNT * c.max_batch;
   ctx->stage_sched_off = round_up(ctx->stage_bytes, 256);

@@ -171,6 +171,45 @@ def test_device_status_reports_nonfinite():
     assert len(np.unique(k)) == 8 and k.min() >= 0 and k.max() < 64
 
 
+@pytest.mark.parametrize("kw", [
+    dict(seed=41, dtype=torch.bfloat16, batch=3, n_vis=(120, 500), n_txt=6, d=136, n_heads=0, rank=12, keep_ratio=0.2),
+    dict(seed=42, dtype=torch.float32, batch=2, n_vis=(60, 200), n_txt=4, d=72, n_heads=0, rank=6, keep=25),
+    dict(seed=43, dtype=torch.bfloat16, batch=2, n_vis=1536, n_txt=8, d=256, n_heads=2, rank=16, kind="video", keep=128),
+], ids=lambda kw: f"seed{kw['seed']}")
+def test_greedy_lowrank_mode(kw):
+    # lowrank_mode = 1: the pick sequence must be a valid run of the pivoted selection (each pick
+    # within 1e-4 of the largest residual of its step: several orders are valid at near-ties) and
+    # the keep-set must be exactly the picked tokens.
+    from oracle import covspec_oracle as O
+    from paper_2605_02218_b200 import api
+    wl = workloads.make_workload(f"greedy{kw['seed']}", **kw)
+    dev = wl.to("cuda:0")
+    pr = api.Pruner.for_workload(dev, lowrank_mode=1)
+    m = pr.marshal(dev)
+    sq, sa, sf = pr.score(m)
+    keep_idx, ko, presel, po, energy = pr.select(m, sf)
+    out, keep2, ko2 = pr.prune(m)
+    pr.check_device_status()
+    assert torch.equal(keep_idx, keep2)
+    keep_idx, presel, energy = keep_idx.cpu().numpy(), presel.cpu().numpy(), energy.cpu().numpy()
+    exact = 0
+    for b in range(wl.batch):
+        v0 = int(wl.vis_offsets[b])
+        ps, en, kp = presel[po[b]:po[b + 1]], energy[po[b]:po[b + 1]], keep_idx[ko[b]:ko[b + 1]]
+        B = len(kp)
+        if B >= len(ps):
+            assert np.array_equal(kp, ps)
+            continue
+        order = np.argsort(-en, kind="stable")[:B]                   # energy = B - k for the k-th pick
+        assert np.array_equal(np.sort(en)[::-1][:B], np.arange(B, 0, -1)) and (np.sort(en)[:len(ps) - B] == 0).all()
+        assert np.array_equal(np.sort(ps[order]), kp)
+        Z = parity.f64(wl.X[v0:v0 + int(np.diff(wl.vis_offsets)[b])])[ps].T
+        picks, _, valid = O.greedy_lowrank_select(Z, B, follow=order, tol=1e-4)
+        assert valid, f"request {b}: a pick was not (nearly) the largest residual"
+        exact += int(np.array_equal(O.greedy_lowrank_select(Z, B)[0], order))
+    print(f"\n[parity] {wl.name}: pick sequences identical to the oracle in {exact} of {wl.batch} requests")
+
+
 def test_compact_rows_follows_the_keep_set():
     # K / V rows (or any per-token tensor) gathered with the same kept indices, bit for bit
     from paper_2605_02218_b200 import api
