@@ -225,7 +225,7 @@ int get_plan(covspec_ctx* ctx, const covspec_problem* p, cudaStream_t stream) {
         if (r.m > kGreedyMaxM || r.b_vis > kGreedyMaxB) return COVSPEC_ERR_UNSUPPORTED;
         c_off += (long long)r.b_vis * r.m;
       }
-      r.win = r.p - r.r + std::min(32, r.r);
+      r.win = r.p - r.r + std::min(16, r.r);
       if (r.win > r.p) r.win = r.p;
       pl.win_max = std::max(pl.win_max, r.win);
       pl.nbot_max = std::max(pl.nbot_max, r.p - r.r);

@@ -16,8 +16,8 @@
 //                  vectors minus the part of the p - r smallest Ritz pairs,
 //                  c_i = sum_j Y'_ij Q_ij - sum_k (Y'_i,win u_k)(Q_i,win u_k).
 // Only the Ritz pairs next to the cut at r have to be resolved individually: basis vectors more
-// than 32 places above the cut are separated from the discarded ones by the same eigenvalue ratios
-// that drive the subspace iteration itself, so the window has p - r + min(32, r) vectors (all p when
+// than 16 places above the cut are separated from the discarded ones by the same eigenvalue ratios
+// that drive the subspace iteration itself, so the window has p - r + min(16, r) vectors (all p when
 // the problem is small).
 #pragma once
 #include "subspace_tc.cuh"
