@@ -98,7 +98,7 @@ typedef struct {
 } covspec_problem;
 
 /* Defaults: lambda 0.5, min-max, head max, presel_factor 2, rank_frac 0.5, rank_cap 128,
- * eig_iters 5, eig_oversample 32, act_layers 4; capacities zero (the caller must set them). */
+ * eig_iters 5, eig_oversample 16, act_layers 4; capacities zero (the caller must set them). */
 void covspec_default_config(covspec_config* cfg);
 
 /* Host-only integer logic of the budgets (paper: r < min(M,d), B_vis < M <= N).  `keep` is the

@@ -647,7 +647,7 @@ void covspec_default_config(covspec_config* c) {
   c->rank_frac = 0.5f;
   c->rank_cap = 128;
   c->eig_iters = 5;
-  c->eig_oversample = 32;
+  c->eig_oversample = 16;
   c->relevance_path = 0;
   c->lowrank_mode = 0;
 }
