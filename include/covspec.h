@@ -80,6 +80,8 @@ typedef struct {
                           1: greedy pivoted selection (not in the paper): pick B_vis times the token with
                              the largest residual energy after projecting out the picked ones; needs
                              M <= 16384 and B_vis <= 8192 per request                              */
+  int ritz_window;     /* basis vectors above the cut at r that take part in the final Rayleigh-Ritz
+                          step together with the eig_oversample ones below it (default 16; >= p: all) */
 } covspec_config;
 
 /* One batch of requests (Sec. III-A notation in brackets). */

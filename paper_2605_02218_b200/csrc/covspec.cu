@@ -153,6 +153,7 @@ int validate_cfg(const covspec_config* c) {
   if (c->eig_iters < 1 || c->eig_oversample < 0) return COVSPEC_ERR_ARG;
   if (c->rank_cap + c->eig_oversample > kPMax) return COVSPEC_ERR_UNSUPPORTED;
   if (c->lowrank_mode < 0 || c->lowrank_mode > 1) return COVSPEC_ERR_ARG;
+  if (c->ritz_window < 0) return COVSPEC_ERR_ARG;
   return COVSPEC_OK;
 }
 
@@ -225,7 +226,7 @@ int get_plan(covspec_ctx* ctx, const covspec_problem* p, cudaStream_t stream) {
         if (r.m > kGreedyMaxM || r.b_vis > kGreedyMaxB) return COVSPEC_ERR_UNSUPPORTED;
         c_off += (long long)r.b_vis * r.m;
       }
-      r.win = r.p - r.r + std::min(16, r.r);
+      r.win = r.p - r.r + std::min(cfg.ritz_window, r.r);
       if (r.win > r.p) r.win = r.p;
       pl.win_max = std::max(pl.win_max, r.win);
       pl.nbot_max = std::max(pl.nbot_max, r.p - r.r);
@@ -650,6 +651,7 @@ void covspec_default_config(covspec_config* c) {
   c->eig_oversample = 16;
   c->relevance_path = 0;
   c->lowrank_mode = 0;
+  c->ritz_window = 16;
 }
 
 int covspec_budgets(const covspec_config* cfg, int n, int keep, int* b_vis, int* m, int* r) {
