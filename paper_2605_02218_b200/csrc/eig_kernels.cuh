@@ -31,18 +31,18 @@ using sub::kXsLd;
 using sub::lt_row_offset;
 using sub::tri_index;
 
-// 1 / sqrt(x) in float64: float32 estimate (~22 bits) refined by two Newton steps written as short
-// dependency chains (the factorisation's critical path runs through this once per column); the
-// library routine outside the float32 range.
+// 1 / sqrt(x) in float64.  The factorisation's critical path runs through this once per column, so
+// the chain of dependent float64 operations is kept short: the float32 estimate is first refined
+// in float32 (to ~2^-23), then one Newton step in float64 squares that error (~1e-13).  The library
+// routine is used outside the float32 range.
 __device__ __forceinline__ double rsqrt_f64(double x) {
   if (!(x > 1e-37 && x < 1e37)) return 1.0 / sqrt(x);
-  double y = (double)rsqrtf((float)x);
-  double hx = 0.5 * x;
-  double e = fma(-hx * y, y, 0.5);        // (1 - x y^2) / 2
-  y = fma(y, e, y);
-  e = fma(-hx * y, y, 0.5);
-  y = fma(y, e, y);
-  return y;
+  float xf = (float)x;
+  float yf = rsqrtf(xf);
+  yf = yf * (1.5f - 0.5f * xf * yf * yf);
+  double y = (double)yf;
+  double e = fma(-0.5 * x * y, y, 0.5);   // (1 - x y^2) / 2
+  return fma(y, e, y);
 }
 
 // Blocked right-looking Cholesky factorisation of an n x n float64 matrix kept in shared memory as
