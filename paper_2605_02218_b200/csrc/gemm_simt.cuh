@@ -47,40 +47,51 @@ gemm_simt_kernel(const GemmProb* __restrict__ table, int nprob, GemmProb single,
   int a_row = tid >> 2, a_k = (tid & 3) * 4;           // A tile: 64 rows x 16 k
   int bkn_k = tid >> 4, bkn_n = (tid & 15) * 4;        // B tile when [k x n]: 16 k x 64 n
 
-  for (int k0 = 0; k0 < pr.k; k0 += kGemmBK) {
+  // The next k-tile is fetched into registers while the current one is multiplied, so that the
+  // global-memory latency overlaps the arithmetic (the problems here are small: few blocks, and a
+  // loop that waited for every tile would be latency-bound).
+  auto fetch = [&](int k0, float (&va)[4], float (&vb)[4]) {
+#pragma unroll
+    for (int e = 0; e < 4; ++e) { va[e] = 0.f; vb[e] = 0.f; }
+    if (k0 >= pr.k) return;
     {
-      float v[4] = {0.f, 0.f, 0.f, 0.f};
       int r = row0 + a_row, kk = k0 + a_k;
       if (r < pr.m) {
         const TA* src = A + (size_t)r * pr.lda + kk;
-        if (kk + 3 < pr.k) load4(src, v);
-        else for (int e = 0; e < 4; ++e) if (kk + e < pr.k) v[e] = to_float(src[e]);
+        if (kk + 3 < pr.k) load4(src, va);
+        else for (int e = 0; e < 4; ++e) if (kk + e < pr.k) va[e] = to_float(src[e]);
       }
-#pragma unroll
-      for (int e = 0; e < 4; ++e) As[a_k + e][a_row] = (AccT)v[e];
     }
     if (!B_KN) {
-      float v[4] = {0.f, 0.f, 0.f, 0.f};
       int r = col0 + a_row, kk = k0 + a_k;
       if (r < pr.n) {
         const TB* src = B + (size_t)r * pr.ldb + kk;
-        if (kk + 3 < pr.k) load4(src, v);
-        else for (int e = 0; e < 4; ++e) if (kk + e < pr.k) v[e] = to_float(src[e]);
+        if (kk + 3 < pr.k) load4(src, vb);
+        else for (int e = 0; e < 4; ++e) if (kk + e < pr.k) vb[e] = to_float(src[e]);
       }
-#pragma unroll
-      for (int e = 0; e < 4; ++e) Bs[a_k + e][a_row] = (AccT)v[e];
     } else {
-      float v[4] = {0.f, 0.f, 0.f, 0.f};
       int kk = k0 + bkn_k, c = col0 + bkn_n;
       if (kk < pr.k) {
         const TB* src = B + (size_t)kk * pr.ldb + c;
-        if (c + 3 < pr.n) load4(src, v);
-        else for (int e = 0; e < 4; ++e) if (c + e < pr.n) v[e] = to_float(src[e]);
+        if (c + 3 < pr.n) load4(src, vb);
+        else for (int e = 0; e < 4; ++e) if (c + e < pr.n) vb[e] = to_float(src[e]);
       }
+    }
+  };
+  float va[4], vb[4];
+  fetch(0, va, vb);
+  for (int k0 = 0; k0 < pr.k; k0 += kGemmBK) {
 #pragma unroll
-      for (int e = 0; e < 4; ++e) Bs[bkn_k][bkn_n + e] = (AccT)v[e];
+    for (int e = 0; e < 4; ++e) As[a_k + e][a_row] = (AccT)va[e];
+    if (!B_KN) {
+#pragma unroll
+      for (int e = 0; e < 4; ++e) Bs[a_k + e][a_row] = (AccT)vb[e];
+    } else {
+#pragma unroll
+      for (int e = 0; e < 4; ++e) Bs[bkn_k][bkn_n + e] = (AccT)vb[e];
     }
     __syncthreads();
+    fetch(k0 + kGemmBK, va, vb);
 #pragma unroll
     for (int kk = 0; kk < kGemmBK; ++kk) {
       AccT a[4], b[4];
