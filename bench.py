@@ -173,7 +173,9 @@ def run_reference(args, rank):
         cpu_baseline(wl.request(0), budget_s=0, min_s=0)
     t_total, tok_total, samples = 0.0, 0, []
     for _ in range(args.steps):
-        r = cpu_baseline(wl, budget_s=args.ref_budget, min_s=min(10.0, args.ref_budget))
+        # every step is a bounded sample; the whole run stays within a few minutes
+        per_step = max(0.5, min(10.0, args.ref_budget, 150.0 / max(args.steps, 1)))
+        r = cpu_baseline(wl, budget_s=max(per_step, 1.5 * per_step), min_s=per_step)
         t_total += r["seconds"]
         tok_total += r["value"] * r["seconds"]
         samples.append(r["sample"])
