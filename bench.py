@@ -5,7 +5,8 @@
 
 One step = one pass of the whole hot path (Eq. 10 through the compacted buffer) over one batch.
 `value` is whole-job visual tokens pruned per second with inputs resident in HBM; `e2e` repeats the
-measurement with host (pinned) inputs copied in and the results copied out inside the timed region.
+measurement with host (pinned) inputs copied in and the results copied out inside the timed region
+(two sets of device input buffers, so that the copy of the next step overlaps the kernels of this one).
 N > 1 (launched with torch.distributed.run): requests are independent, so every rank prunes its own
 batch of the same shape (different seed) with no collective on the data path (weak scaling); the
 time is the maximum over ranks.
@@ -334,30 +335,52 @@ def main():
     host = wl0.to("cpu")
     pin = lambda t: t.pin_memory()
     hX, hQ, hHs = pin(host.X), pin(host.Q), [pin(h) for h in host.Hs]
-    dX, dQ, dHs = torch.empty_like(wl0.X), torch.empty_like(wl0.Q), [torch.empty_like(h) for h in wl0.Hs]
-    m_e2e = pr.marshal(X=dX, Q=dQ, vis_offsets=wl0.vis_offsets, txt_offsets=wl0.txt_offsets,
-                       Wq=wl0.Wq, Wk=wl0.Wk, Hs=dHs, keep=wl0.keep)
+    # Two sets of device input buffers: the copy of step i+1 (on a copy stream) overlaps the kernels
+    # of step i.  Every step still copies all of its inputs in and its results out.
+    n_buf = 2
+    dXs = [torch.empty_like(wl0.X) for _ in range(n_buf)]
+    dQs = [torch.empty_like(wl0.Q) for _ in range(n_buf)]
+    dHss = [[torch.empty_like(h) for h in wl0.Hs] for _ in range(n_buf)]
+    m_e2e = [pr.marshal(X=dXs[i], Q=dQs[i], vis_offsets=wl0.vis_offsets, txt_offsets=wl0.txt_offsets,
+                        Wq=wl0.Wq, Wk=wl0.Wk, Hs=dHss[i], keep=wl0.keep) for i in range(n_buf)]
     h_out = torch.empty((n_keep, wl0.d), dtype=wl0.dtype).pin_memory()
     h_keep = torch.empty(n_keep, dtype=torch.int32).pin_memory()
     h2d = hX.nbytes + hQ.nbytes + sum(h.nbytes for h in hHs)
     d2h = h_out.nbytes + h_keep.nbytes
+    copy_stream = torch.cuda.Stream(device=dev)
+    main_stream = torch.cuda.current_stream(dev)
+    copied = [torch.cuda.Event() for _ in range(n_buf)]      # inputs of the set are on the device
+    consumed = [torch.cuda.Event() for _ in range(n_buf)]    # the kernels that read the set are done
+    for ev in consumed:
+        ev.record(main_stream)
 
-    def step_e2e():
-        dX.copy_(hX, non_blocking=True)
-        dQ.copy_(hQ, non_blocking=True)
-        for a, b in zip(dHs, hHs):
-            a.copy_(b, non_blocking=True)
-        pr.prune(m_e2e, outs[0], keeps[0])
-        h_out.copy_(outs[0], non_blocking=True)
-        h_keep.copy_(keeps[0], non_blocking=True)
+    def upload(i):
+        j = i % n_buf
+        with torch.cuda.stream(copy_stream):
+            copy_stream.wait_event(consumed[j])
+            dXs[j].copy_(hX, non_blocking=True)
+            dQs[j].copy_(hQ, non_blocking=True)
+            for a_, b_ in zip(dHss[j], hHs):
+                a_.copy_(b_, non_blocking=True)
+            copied[j].record(copy_stream)
+
+    def run_e2e(n_steps):
+        upload(0)
+        for i in range(n_steps):
+            j = i % n_buf
+            if i + 1 < n_steps:
+                upload(i + 1)
+            main_stream.wait_event(copied[j])
+            pr.prune(m_e2e[j], outs[0], keeps[0])
+            consumed[j].record(main_stream)
+            h_out.copy_(outs[0], non_blocking=True)
+            h_keep.copy_(keeps[0], non_blocking=True)
 
     e2e_steps = max(3, min(args.steps, 20))
-    for _ in range(3):
-        step_e2e()
+    run_e2e(3)
     barrier()
     ev0.record()
-    for _ in range(e2e_steps):
-        step_e2e()
+    run_e2e(e2e_steps)
     ev1.record()
     barrier()
     ms_e2e = ev0.elapsed_time(ev1) / e2e_steps
