@@ -349,7 +349,8 @@ ritz_kernel(const ReqPlan* __restrict__ plan, const double* __restrict__ partial
   __syncthreads();
   if (tid < nact) {
     bool converged;
-    if (w <= 64) converged = jacobi_sweeps<16>(C, ldc, w, s1, max_sweeps, nact, &s_flag);
+    if (w <= 32) converged = jacobi_sweeps<8>(C, ldc, w, s1, max_sweeps, nact, &s_flag);
+    else if (w <= 64) converged = jacobi_sweeps<16>(C, ldc, w, s1, max_sweeps, nact, &s_flag);
     else if (w <= 96) converged = jacobi_sweeps<24>(C, ldc, w, s1, max_sweeps, nact, &s_flag);
     else converged = jacobi_sweeps<(kPMax + 3) / 4>(C, ldc, w, s1, max_sweeps, nact, &s_flag);
     if (!converged && tid == 0) atomicOr(status, kStatusNoConverge);
