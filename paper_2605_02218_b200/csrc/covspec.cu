@@ -521,16 +521,18 @@ int score_impl(covspec_ctx* ctx, const covspec_problem* p, float* s_query, float
 // ---- preselect, Eq. 13-15, final select ---------------------------------------------------------
 template <typename T>
 int select_impl(covspec_ctx* ctx, const covspec_problem* p, const float* s_fused, int* keep_idx,
-                int* presel_out, float* energy_out, cudaStream_t s) {
+                int* presel_out, float* energy_out, cudaStream_t s, bool presel_done = false) {
   const covspec_config& cfg = ctx->cfg;
   const Plan& pl = ctx->plan;
   int B = p->batch;
   int* presel = presel_out ? presel_out : ctx->presel;
   float* energy = energy_out ? energy_out : ctx->energy;
-  prof_mark(ctx, ST_PRESELECT, 0, s);
-  preselect_kernel<<<B, 1024, 0, s>>>(s_fused, ctx->d_plan, presel, ctx->status);
-  LAUNCH_CHECK(ctx);
-  prof_mark(ctx, ST_PRESELECT, 1, s);
+  if (!presel_done) {
+    prof_mark(ctx, ST_PRESELECT, 0, s);
+    preselect_kernel<<<B, 1024, 0, s>>>(s_fused, ctx->d_plan, presel, ctx->status);
+    LAUNCH_CHECK(ctx);
+    prof_mark(ctx, ST_PRESELECT, 1, s);
+  }
   if (pl.n_stage2 > 0) {
     prof_mark(ctx, ST_GRAM, 0, s);
     int vec16 = cfg.d * ctx->esize / 16;
@@ -900,14 +902,15 @@ int covspec_prune(covspec_ctx* ctx, const covspec_problem* p, void* out_hidden, 
   st = bf ? score_impl<__nv_bfloat16>(ctx, p, nullptr, nullptr, fused, false, s)
           : score_impl<float>(ctx, p, nullptr, nullptr, fused, false, s);
   if (st) return st;
+  // Eq. 12 and the preselection share one launch in the fused call
   prof_mark(ctx, ST_FUSE, 0, s);
-  fuse_kernel<<<p->batch, 1024, 0, s>>>(ctx->sq, ctx->cfg.act_layers > 0 ? ctx->sa : nullptr,
-                                        ctx->d_plan, ctx->cfg.lambda, ctx->cfg.norm_mode, fused,
-                                        ctx->status);
+  fuse_preselect_kernel<<<p->batch, 1024, 0, s>>>(ctx->sq, ctx->cfg.act_layers > 0 ? ctx->sa : nullptr,
+                                                  ctx->d_plan, ctx->cfg.lambda, ctx->cfg.norm_mode, fused,
+                                                  ctx->presel, ctx->status);
   LAUNCH_CHECK(ctx);
   prof_mark(ctx, ST_FUSE, 1, s);
-  st = bf ? select_impl<__nv_bfloat16>(ctx, p, fused, keep_idx, nullptr, nullptr, s)
-          : select_impl<float>(ctx, p, fused, keep_idx, nullptr, nullptr, s);
+  st = bf ? select_impl<__nv_bfloat16>(ctx, p, fused, keep_idx, nullptr, nullptr, s, true)
+          : select_impl<float>(ctx, p, fused, keep_idx, nullptr, nullptr, s, true);
   if (st) return st;
   st = compact_impl(ctx, p, keep_idx, out_hidden, nullptr, s);
   if (ctx->prof_cap && ctx->prof_calls < ctx->prof_cap) ++ctx->prof_calls;

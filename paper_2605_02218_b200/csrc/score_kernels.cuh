@@ -169,14 +169,11 @@ __device__ __forceinline__ NormParams norm_params(const float* s, int n, int mod
   return np;
 }
 
-// Eq. 12.  One block per request: normalise both scores to a common scale, fuse with lambda.
+// Eq. 12 for one request (whole block): normalise both scores to a common scale, fuse with lambda.
 // s_act == nullptr (no activity stack): the fused score is the normalised query score.
-__global__ void __launch_bounds__(1024)
-fuse_kernel(const float* __restrict__ s_query, const float* __restrict__ s_act,
-            const ReqPlan* __restrict__ plan, float lambda, int mode, float* __restrict__ s_fused,
-            int* status) {
-  __shared__ float scratch[32];
-  ReqPlan rp = plan[blockIdx.x];
+__device__ __forceinline__ void fuse_request(const ReqPlan& rp, const float* __restrict__ s_query,
+                                             const float* __restrict__ s_act, float lambda, int mode,
+                                             float* __restrict__ s_fused, float* scratch, int* status) {
   const float* sq = s_query + rp.vis_off;
   NormParams nq = norm_params(sq, rp.n, mode, scratch, status);
   if (s_act == nullptr) {
@@ -189,6 +186,15 @@ fuse_kernel(const float* __restrict__ s_query, const float* __restrict__ s_act,
   for (int i = threadIdx.x; i < rp.n; i += blockDim.x)
     s_fused[rp.vis_off + i] =
         lambda * ((sq[i] - nq.shift) * nq.scale) + (1.f - lambda) * ((sa[i] - na.shift) * na.scale);
+}
+
+// Eq. 12.  One block per request.
+__global__ void __launch_bounds__(1024)
+fuse_kernel(const float* __restrict__ s_query, const float* __restrict__ s_act,
+            const ReqPlan* __restrict__ plan, float lambda, int mode, float* __restrict__ s_fused,
+            int* status) {
+  __shared__ float scratch[32];
+  fuse_request(plan[blockIdx.x], s_query, s_act, lambda, mode, s_fused, scratch, status);
 }
 
 }  // namespace covspec

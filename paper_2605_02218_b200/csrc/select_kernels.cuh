@@ -2,6 +2,7 @@
 // and the row gather used for Z_M (Eq. 13) and for the compacted output.
 #pragma once
 #include "common.cuh"
+#include "score_kernels.cuh"
 
 namespace covspec {
 
@@ -152,6 +153,19 @@ __global__ void __launch_bounds__(1024)
 preselect_kernel(const float* __restrict__ s_fused, const ReqPlan* __restrict__ plan,
                  int* __restrict__ presel, int* status) {
   ReqPlan rp = plan[blockIdx.x];
+  block_topk(s_fused + rp.vis_off, rp.n, rp.m, false, nullptr, presel + rp.presel_off, status);
+}
+
+// Eq. 12 and the preselection in one launch (the fused call): the block that fused a request's
+// scores selects its M best right away.
+__global__ void __launch_bounds__(1024)
+fuse_preselect_kernel(const float* __restrict__ s_query, const float* __restrict__ s_act,
+                      const ReqPlan* __restrict__ plan, float lambda, int mode,
+                      float* __restrict__ s_fused, int* __restrict__ presel, int* status) {
+  __shared__ float scratch[32];
+  ReqPlan rp = plan[blockIdx.x];
+  fuse_request(rp, s_query, s_act, lambda, mode, s_fused, scratch, status);
+  __syncthreads();                                  // the block's own global writes are visible to it
   block_topk(s_fused + rp.vis_off, rp.n, rp.m, false, nullptr, presel + rp.presel_off, status);
 }
 
