@@ -46,9 +46,11 @@ typedef enum {
   COVSPEC_ERR_WORKSPACE = -4,   /* problem exceeds the capacities given at init               */
   COVSPEC_ERR_CUDA = -5,        /* a CUDA runtime call failed (see covspec_last_cuda_error)   */
   COVSPEC_ERR_NONFINITE = -6,   /* device status: a score was NaN or Inf                      */
-  COVSPEC_ERR_NOCONVERGE = -7,  /* device status: small eigen-solve hit its sweep limit       */
-  COVSPEC_ERR_STATIC_CAPACITY = -8, /* covspec_query_score_static: beyond its fixed scratch size */
-  COVSPEC_ERR_TIMEOUT = -9      /* device status: a bounded wait inside a kernel expired      */
+  COVSPEC_ERR_NOCONVERGE = -7,  /* device status: the subspace iteration behind Eq. 14 had not
+                                   settled within the tolerance after its last step, or the small
+                                   eigen-solve hit its sweep limit                             */
+  COVSPEC_ERR_TIMEOUT = -8,     /* device status: a bounded wait inside a kernel expired      */
+  COVSPEC_ERR_STATIC_CAPACITY = -9 /* covspec_query_score_static: beyond its fixed scratch size */
 } covspec_status;
 
 /* Static configuration.  Fill with covspec_default_config() and override. */

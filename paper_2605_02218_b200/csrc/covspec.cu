@@ -560,7 +560,7 @@ int select_impl(covspec_ctx* ctx, const covspec_problem* p, const float* s_fused
     prof_mark(ctx, ST_EIG, 0, s);
     if (cfg.lowrank_mode == 1) {
       // greedy pivoted selection instead of the subspace energies; it writes its own `energy`
-      greedy_select_kernel<<<B, kGreedyThreads, 0, s>>>(ctx->d_plan, ctx->Ghi, ctx->Glo, ctx->ld, ctx->Cg, energy);
+      greedy_select_kernel<<<B, kGreedyThreads, 0, s>>>(ctx->d_plan, ctx->Ghi, ctx->Glo, ctx->ld, ctx->Cg, energy, ctx->status);
       LAUNCH_CHECK(ctx);
       prof_mark(ctx, ST_EIG, 1, s);
       prof_mark(ctx, ST_FINAL, 0, s);
@@ -1124,16 +1124,43 @@ int static_scratch_ptr(unsigned char** out) {
   return COVSPEC_OK;
 }
 
+// The per-request plan reaches the scratch array as kernel arguments (by value, 64 requests per
+// launch), not through a host-to-device copy: nothing of the call keeps pointing at host memory
+// after the call has returned.
+struct StaticPlanChunk {
+  int4 e[64];        // vis_off, n, txt_off, t
+  int first, count;
+};
+
+__global__ void static_plan_kernel(ReqPlan* __restrict__ plan, const StaticPlanChunk chunk) {
+  int i = threadIdx.x;
+  if (i >= chunk.count) return;
+  ReqPlan rp{};
+  rp.vis_off = chunk.e[i].x; rp.n = chunk.e[i].y; rp.txt_off = chunk.e[i].z; rp.t = chunk.e[i].w;
+  plan[chunk.first + i] = rp;
+}
+
 template <typename T>
-int query_score_static_impl(int d, int batch, const ReqPlan* h_plan, const void* X, const void* Q,
-                            long long rows_x, int rows_q, float* s_query, cudaStream_t s) {
+int query_score_static_impl(int d, int batch, const int* vis_offsets, const int* txt_offsets,
+                            const void* X, const void* Q, float* s_query, cudaStream_t s) {
   unsigned char* scratch = nullptr;
   int st = static_scratch_ptr(&scratch);
   if (st) return st;
   ReqPlan* d_plan = reinterpret_cast<ReqPlan*>(scratch);
   float* Qn = reinterpret_cast<float*>(scratch + kStaticPlanBytes);
-  // The copy source is ordinary host memory: the runtime stages it before the call returns.
-  CUDA_TRY(cudaMemcpyAsync(d_plan, h_plan, sizeof(ReqPlan) * batch, cudaMemcpyHostToDevice, s));
+  for (int b0 = 0; b0 < batch; b0 += 64) {
+    StaticPlanChunk chunk{};
+    chunk.first = b0; chunk.count = std::min(64, batch - b0);
+    for (int i = 0; i < chunk.count; ++i) {
+      int b = b0 + i;
+      chunk.e[i] = make_int4(vis_offsets[b], vis_offsets[b + 1] - vis_offsets[b], txt_offsets[b],
+                             txt_offsets[b + 1] - txt_offsets[b]);
+    }
+    static_plan_kernel<<<1, 64, 0, s>>>(d_plan, chunk);
+    CUDA_TRY(cudaGetLastError());
+  }
+  long long rows_x = vis_offsets[batch];
+  int rows_q = txt_offsets[batch];
   qnorm_kernel<T><<<(rows_q + 7) / 8, 256, 0, s>>>(reinterpret_cast<const T*>(Q), Qn, rows_q, 1, d);
   CUDA_TRY(cudaGetLastError());
   cosmax_kernel<T><<<(unsigned)((rows_x + 7) / 8), 256, 0, s>>>(
@@ -1152,19 +1179,12 @@ extern "C" int covspec_query_score_static(int dtype, int d, int batch, const voi
   if (d < 8 || d % 8) return COVSPEC_ERR_UNSUPPORTED;
   if (vis_offsets[0] != 0 || txt_offsets[0] != 0) return COVSPEC_ERR_SHAPE;
   if (batch > kStaticMaxBatch) return COVSPEC_ERR_STATIC_CAPACITY;
-  ReqPlan h_plan[kStaticMaxBatch];
-  memset(h_plan, 0, sizeof(ReqPlan) * batch);
-  for (int b = 0; b < batch; ++b) {
+  for (int b = 0; b < batch; ++b)
     if (vis_offsets[b + 1] <= vis_offsets[b] || txt_offsets[b + 1] <= txt_offsets[b])
       return COVSPEC_ERR_SHAPE;
-    h_plan[b].vis_off = vis_offsets[b]; h_plan[b].n = vis_offsets[b + 1] - vis_offsets[b];
-    h_plan[b].txt_off = txt_offsets[b]; h_plan[b].t = txt_offsets[b + 1] - txt_offsets[b];
-  }
   if ((long long)txt_offsets[batch] * d > kStaticMaxQueryElems) return COVSPEC_ERR_STATIC_CAPACITY;
   cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
   return dtype == COVSPEC_BF16
-             ? query_score_static_impl<__nv_bfloat16>(d, batch, h_plan, X, Q, vis_offsets[batch],
-                                                      txt_offsets[batch], s_query, s)
-             : query_score_static_impl<float>(d, batch, h_plan, X, Q, vis_offsets[batch],
-                                              txt_offsets[batch], s_query, s);
+             ? query_score_static_impl<__nv_bfloat16>(d, batch, vis_offsets, txt_offsets, X, Q, s_query, s)
+             : query_score_static_impl<float>(d, batch, vis_offsets, txt_offsets, X, Q, s_query, s);
 }

@@ -23,7 +23,7 @@ constexpr int kGreedyMaxB = 8192;                       // picks per request (ro
 __global__ void __launch_bounds__(kGreedyThreads)
 greedy_select_kernel(const ReqPlan* __restrict__ plan, const __nv_bfloat16* __restrict__ g_hi,
                      const __nv_bfloat16* __restrict__ g_lo, int ld, float* __restrict__ cbuf,
-                     float* __restrict__ energy) {
+                     float* __restrict__ energy, int* status) {
   __shared__ float cp[kGreedyMaxB];                     // c_j[p] for the current pivot p, j < k
   __shared__ float red_v[32];
   __shared__ int red_i[32];
@@ -45,14 +45,22 @@ greedy_select_kernel(const ReqPlan* __restrict__ plan, const __nv_bfloat16* __re
     int i = tid + q * kGreedyThreads;
     e[q] = i < M ? G(i, i) : -INFINITY;
   }
+  bool bad = false;
   for (int k = 0; k < B; ++k) {
     // ---- argmax of the residuals: larger value first, then lower index ----
+    // A residual that is not a number (non-finite Gram entries) ranks below every number but
+    // above the picked tokens' -inf, so that the pivot is always an unpicked token inside the
+    // request; the condition is reported through the status word.
     float bv = -INFINITY;
     int bi = 0x7fffffff;
 #pragma unroll
     for (int q = 0; q < kGreedyPer; ++q) {
       int i = tid + q * kGreedyThreads;
-      if (i < M && (e[q] > bv || (e[q] == bv && i < bi))) { bv = e[q]; bi = i; }
+      if (i < M) {
+        float v = e[q];
+        if (v != v) { v = -3.0e38f; bad = true; }
+        if (v > bv || (v == bv && i < bi)) { bv = v; bi = i; }
+      }
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
@@ -70,7 +78,10 @@ greedy_select_kernel(const ReqPlan* __restrict__ plan, const __nv_bfloat16* __re
         int oi = __shfl_xor_sync(0xffffffffu, bi, o);
         if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
       }
-      if (lane == 0) { s_p = bi; s_ep = bv; energy[rp.presel_off + bi] = (float)(B - k); }
+      if (lane == 0) {
+        if (bi >= M) { bi = 0; bv = 0.f; atomicOr(status, kStatusNonFinite); }   // every token picked: cannot happen for B < M
+        s_p = bi; s_ep = bv; energy[rp.presel_off + bi] = (float)(B - k);
+      }
     }
     __syncthreads();
     const int p = s_p;
@@ -88,11 +99,12 @@ greedy_select_kernel(const ReqPlan* __restrict__ plan, const __nv_bfloat16* __re
         float c = acc * rs;
         C[(size_t)k * M + i] = c;
         if (i == p) e[q] = -INFINITY;                   // never picked again
-        else if (e[q] > -INFINITY) e[q] -= c * c;
+        else if (!(e[q] == -INFINITY)) e[q] -= c * c;
       }
     }
     __syncthreads();
   }
+  if (bad) atomicOr(status, kStatusNonFinite);
 }
 
 }  // namespace covspec

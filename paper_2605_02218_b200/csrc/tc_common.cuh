@@ -123,8 +123,10 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&t);
 }
 
-// Float atomic max through the sign-split integer trick (the target starts at -inf).
+// Float atomic max through the sign-split integer trick (the target starts at -inf).  -0 is folded
+// onto +0 first: as an integer it would lose against the -inf fill.
 __device__ __forceinline__ void atomic_max_float(float* addr, float v) {
+  v += 0.0f;
   if (v >= 0.f) atomicMax(reinterpret_cast<int*>(addr), __float_as_int(v));
   else atomicMin(reinterpret_cast<unsigned*>(addr), __float_as_uint(v));
 }

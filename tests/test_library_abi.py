@@ -116,8 +116,8 @@ def test_host_side_rejections(lib):
 
 
 def test_strerror(lib):
-    texts = {lib.covspec_strerror(s).decode() for s in range(0, -8, -1)}
-    assert len(texts) == 8 and "unknown status" not in texts
+    texts = {lib.covspec_strerror(s).decode() for s in range(0, -10, -1)}
+    assert len(texts) == 10 and "unknown status" not in texts
     assert lib.covspec_strerror(-99).decode() == "unknown status"
 
 

@@ -151,6 +151,23 @@ def test_eq12_hand():
     np.testing.assert_allclose(O.fuse(A(g["S_query"]), A(g["S_act"]), g["lam"]), g["S"], atol=1e-15)
 
 
+def test_eq12_zscore_hand():
+    # the z-score reading divides by the population deviation; the sample deviation (n - 1) or a
+    # missing mean would fail these hand-worked values
+    g = GOLD["eq12_zscore"]
+    np.testing.assert_allclose(O.normalise(A(g["S"]), "zscore"), g["z"], atol=1e-15)
+    np.testing.assert_allclose(O.normalise(A(g["S3"]), "zscore"), g["z3"], atol=1e-15)
+    np.testing.assert_allclose(O.fuse(A(g["S3"]), A(g["S3_act"]), g["lambda"], "zscore"), g["fused3"],
+                               atol=1e-15)
+    # zero mean, unit population variance, invariant to a positive affine change; constant -> 0
+    z = O.normalise(RNG.normal(size=40) * 3 + 7, "zscore")
+    assert abs(z.mean()) < 1e-14 and abs(np.mean(z * z) - 1.0) < 1e-13
+    s = RNG.normal(size=40)
+    np.testing.assert_allclose(O.normalise(5 * s - 2, "zscore"), O.normalise(s, "zscore"), atol=1e-13)
+    np.testing.assert_allclose(O.normalise(np.full(5, 3.0), "zscore"), np.zeros(5), atol=0)
+    np.testing.assert_allclose(O.normalise(A(g["S3"]), "none"), g["S3"], atol=0)
+
+
 def test_eq12_properties():
     sq, sa = RNG.normal(size=50), np.abs(RNG.normal(size=50))
     s = O.fuse(sq, sa, 0.3)
