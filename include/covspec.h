@@ -84,6 +84,10 @@ typedef struct {
                              M <= 16384 and B_vis <= 8192 per request                              */
   int ritz_window;     /* basis vectors above the cut at r that take part in the final Rayleigh-Ritz
                           step together with the eig_oversample ones below it (default 16; >= p: all) */
+  int activity_overlap; /* > 0: while Eq. 10 runs on the tensor cores (which leaves HBM idle), Eq. 11
+                          streams the snapshot stack on a second stream of the context with this many
+                          512-thread blocks per SM (1 or 2; default 1), joined before Eq. 12; 0: the two
+                          scores are computed one after the other on the caller's stream           */
 } covspec_config;
 
 /* One batch of requests (Sec. III-A notation in brackets). */

@@ -105,6 +105,9 @@ struct covspec_ctx {
   char* h_stage = nullptr;
   long long stage_bytes = 0, stage_sched_off = 0;
   cudaEvent_t stage_free = nullptr;      // the previous upload has been consumed
+  // the fused call streams the snapshot stack (Eq. 11) beside the relevance kernel on this stream
+  cudaStream_t side = nullptr;
+  cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
   Plan plan;
   int num_sms = 148;
   bool tc_ready = false;                 // tensor-core relevance kernel configured on this device
@@ -154,6 +157,7 @@ int validate_cfg(const covspec_config* c) {
   if (c->rank_cap + c->eig_oversample > kPMax) return COVSPEC_ERR_UNSUPPORTED;
   if (c->lowrank_mode < 0 || c->lowrank_mode > 1) return COVSPEC_ERR_ARG;
   if (c->ritz_window < 0) return COVSPEC_ERR_ARG;
+  if (c->activity_overlap < 0 || c->activity_overlap > 2) return COVSPEC_ERR_ARG;
   return COVSPEC_OK;
 }
 
@@ -440,6 +444,36 @@ int relevance_tc(covspec_ctx* ctx, const covspec_problem* p, float* s_query, cud
 }
 
 // ---- Eq. 10-12 -------------------------------------------------------------------------------
+// Eq. 11 on `s`: the full-rate kernel, or (background = true) the small persistent grid that runs
+// beside the relevance kernel.
+template <typename T>
+int launch_activity(covspec_ctx* ctx, const covspec_problem* p, float* s_act, bool background,
+                    cudaStream_t s) {
+  const covspec_config& cfg = ctx->cfg;
+  long long rowsX = ctx->plan.total_vis;
+  LayerPtrs lp{};
+  for (int l = 0; l <= cfg.act_layers; ++l) lp.h[l] = p->Hs[l];
+  if (background) {
+    unsigned grid = (unsigned)std::min<long long>((rowsX + 15) / 16, (long long)ctx->num_sms * cfg.activity_overlap);
+    if (cfg.act_layers <= 4)
+      activity_stream_kernel<T, 4><<<grid, 512, 0, s>>>(lp, cfg.act_layers, rowsX, cfg.d, s_act);
+    else if (cfg.act_layers <= 8)
+      activity_stream_kernel<T, 8><<<grid, 512, 0, s>>>(lp, cfg.act_layers, rowsX, cfg.d, s_act);
+    else
+      activity_stream_kernel<T, 16><<<grid, 512, 0, s>>>(lp, cfg.act_layers, rowsX, cfg.d, s_act);
+  } else {
+    unsigned grid = (unsigned)((rowsX + 7) / 8);
+    if (cfg.act_layers <= 4)
+      activity_kernel<T, 4><<<grid, 256, 0, s>>>(lp, cfg.act_layers, rowsX, cfg.d, s_act);
+    else if (cfg.act_layers <= 8)
+      activity_kernel<T, 8><<<grid, 256, 0, s>>>(lp, cfg.act_layers, rowsX, cfg.d, s_act);
+    else
+      activity_kernel<T, 16><<<grid, 256, 0, s>>>(lp, cfg.act_layers, rowsX, cfg.d, s_act);
+  }
+  LAUNCH_CHECK(ctx);
+  return COVSPEC_OK;
+}
+
 template <typename T>
 int score_impl(covspec_ctx* ctx, const covspec_problem* p, float* s_query, float* s_act,
                float* s_fused, bool do_fuse, cudaStream_t s) {
@@ -455,6 +489,18 @@ int score_impl(covspec_ctx* ctx, const covspec_problem* p, float* s_query, float
   if (!s_act) s_act = ctx->sa;
   bool identity = cfg.n_heads == 0;
   bool use_tc = tc_supported(ctx);
+  // The tensor-core relevance kernel leaves HBM idle: the activity stream runs beside it on the
+  // context's side stream (fork here, join before the scores are fused).
+  bool overlap = use_tc && cfg.act_layers > 0 && cfg.activity_overlap > 0;
+  if (overlap) {
+    CUDA_TRY(cudaEventRecord(ctx->ev_fork, s));
+    CUDA_TRY(cudaStreamWaitEvent(ctx->side, ctx->ev_fork, 0));
+    prof_mark(ctx, ST_ACTIVITY, 0, ctx->side);
+    int st = launch_activity<T>(ctx, p, s_act, true, ctx->side);
+    if (st) return st;
+    prof_mark(ctx, ST_ACTIVITY, 1, ctx->side);
+    CUDA_TRY(cudaEventRecord(ctx->ev_join, ctx->side));
+  }
   if (use_tc) {
     int st = relevance_tc(ctx, p, s_query, s);
     if (st) return st;
@@ -494,18 +540,12 @@ int score_impl(covspec_ctx* ctx, const covspec_problem* p, float* s_query, float
   }
   prof_mark(ctx, ST_RELEVANCE, 1, s);
   }
-  if (cfg.act_layers > 0) {
+  if (overlap) {
+    CUDA_TRY(cudaStreamWaitEvent(s, ctx->ev_join, 0));
+  } else if (cfg.act_layers > 0) {
     prof_mark(ctx, ST_ACTIVITY, 0, s);
-    LayerPtrs lp{};
-    for (int l = 0; l <= cfg.act_layers; ++l) lp.h[l] = p->Hs[l];
-    unsigned grid = (unsigned)((rowsX + 7) / 8);
-    if (cfg.act_layers <= 4)
-      activity_kernel<T, 4><<<grid, 256, 0, s>>>(lp, cfg.act_layers, rowsX, cfg.d, s_act);
-    else if (cfg.act_layers <= 8)
-      activity_kernel<T, 8><<<grid, 256, 0, s>>>(lp, cfg.act_layers, rowsX, cfg.d, s_act);
-    else
-      activity_kernel<T, 16><<<grid, 256, 0, s>>>(lp, cfg.act_layers, rowsX, cfg.d, s_act);
-    LAUNCH_CHECK(ctx);
+    int st = launch_activity<T>(ctx, p, s_act, false, s);
+    if (st) return st;
     prof_mark(ctx, ST_ACTIVITY, 1, s);
   }
   if (do_fuse) {
@@ -654,6 +694,7 @@ void covspec_default_config(covspec_config* c) {
   c->relevance_path = 0;
   c->lowrank_mode = 0;
   c->ritz_window = 16;
+  c->activity_overlap = 1;
 }
 
 int covspec_budgets(const covspec_config* cfg, int n, int keep, int* b_vis, int* m, int* r) {
@@ -769,7 +810,10 @@ int covspec_prune_init(const covspec_config* cfg, covspec_ctx** out) {
   ctx->stage_bytes = ctx->stage_sched_off + 4 * sched_ints;
   bool ok = cudaMemset(ctx->status, 0, 256) == cudaSuccess &&
             cudaMallocHost(&ctx->h_stage, (size_t)ctx->stage_bytes) == cudaSuccess &&
-            cudaEventCreateWithFlags(&ctx->stage_free, cudaEventDisableTiming) == cudaSuccess;
+            cudaEventCreateWithFlags(&ctx->stage_free, cudaEventDisableTiming) == cudaSuccess &&
+            cudaStreamCreateWithFlags(&ctx->side, cudaStreamNonBlocking) == cudaSuccess &&
+            cudaEventCreateWithFlags(&ctx->ev_fork, cudaEventDisableTiming) == cudaSuccess &&
+            cudaEventCreateWithFlags(&ctx->ev_join, cudaEventDisableTiming) == cudaSuccess;
   // the small dense kernels need more than the default 48 KB of dynamic shared memory
   ok = ok && cudaFuncSetAttribute(chol_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                   (int)cholesky_smem_bytes(kPMax)) == cudaSuccess;
@@ -799,6 +843,18 @@ int covspec_prune_init(const covspec_config* cfg, covspec_ctx** out) {
     ok = ctx->tc_ready;
   }
   if (ok) {
+    // The background activity kernel shares its SMs with the relevance kernel, whose CTA needs the
+    // largest shared-memory carve-out: ask for the same split, or the two could not be resident on
+    // one SM at the same time (an SM changes its L1 / shared-memory split only when it is idle).
+    auto max_shared = [](auto* kernel) {
+      return cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                  cudaSharedmemCarveoutMaxShared) == cudaSuccess;
+    };
+    ok = max_shared(activity_stream_kernel<__nv_bfloat16, 4>) && max_shared(activity_stream_kernel<__nv_bfloat16, 8>) &&
+         max_shared(activity_stream_kernel<__nv_bfloat16, 16>) && max_shared(activity_stream_kernel<float, 4>) &&
+         max_shared(activity_stream_kernel<float, 8>) && max_shared(activity_stream_kernel<float, 16>);
+  }
+  if (ok) {
     // tensor maps over the workspace arrays of the subspace iteration (fixed for the context)
     int st = COVSPEC_OK;
     if (!f32) st = make_map_bf16(&ctx->map_zg, ctx->Zg, c.max_total_presel, c.d, sub::kTile);
@@ -823,6 +879,9 @@ int covspec_prune_destroy(covspec_ctx* ctx) {
   if (ctx->ws) cudaFree(ctx->ws);
   if (ctx->h_stage) cudaFreeHost(ctx->h_stage);
   if (ctx->stage_free) cudaEventDestroy(ctx->stage_free);
+  if (ctx->side) cudaStreamDestroy(ctx->side);
+  if (ctx->ev_fork) cudaEventDestroy(ctx->ev_fork);
+  if (ctx->ev_join) cudaEventDestroy(ctx->ev_join);
   delete ctx;
   return COVSPEC_OK;
 }

@@ -40,8 +40,11 @@ constexpr int kBytesStage = kBytesA + kBytesB;
 constexpr int kBytesKp = kTileM * kHalf * 2;       // 16 KB: [128 x 64] of one half head; hi and lo
 constexpr int kBytesQ = kTT * kHalf * 2;           // 8 KB: [64 x 64] of one half head; hi and lo
 // The query sub-tiles (hi + lo = 16 KB) travel through the same ring slots as the main-loop chunks.
-constexpr int kSmemBytes = kStages * kBytesStage + 2 * kBytesKp + 1024 /*barriers*/ +
-                           1024 /*alignment slack*/;
+// No slack for aligning the base: the dynamic region is declared 1024-byte aligned (the kernel has
+// no static shared memory in front of it) and the kernel checks it.  Every resident block reserves
+// 1 KB of the SM's 228 KB, so this size leaves room for two small blocks of another kernel beside
+// the CTA (the activity stream of the fused call).
+constexpr int kSmemBytes = kStages * kBytesStage + 2 * kBytesKp + 1024 /*barriers*/;
 constexpr int kTmemCols = 512;
 constexpr int kLogitCol = 256;         // logits tiles live at columns 256 + 64 * slot
 
@@ -68,8 +71,12 @@ relevance_tc_kernel(const __grid_constant__ CUtensorMap map_a,   // X (MODE 0) o
                     const __grid_constant__ CUtensorMap map_q,   // Qn hi: [sum T, P] (MODE 0 only)
                     const __grid_constant__ CUtensorMap map_ql,  // Qn lo
                     const Params prm) {
-  extern __shared__ uint8_t smem_raw[];
-  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  extern __shared__ __align__(1024) uint8_t rel_smem_raw[];
+  uint8_t* smem = rel_smem_raw;
+  if (smem_u32(smem) & 1023u) {          // the swizzled tiles need a 1024-byte aligned base
+    if (threadIdx.x == 0) atomicOr(prm.status, kStatusTimeout);
+    return;
+  }
   uint8_t* stage_base = smem;
   uint8_t* kp_smem = smem + kStages * kBytesStage;       // hi tile, then lo tile
   uint64_t* bars = reinterpret_cast<uint64_t*>(kp_smem + 2 * kBytesKp);

@@ -55,13 +55,12 @@ def test_small_shapes(kw):
 
 def test_zero_token_on_the_tensor_core_path():
     # an all-zero visual token has cosine 0 with every query element (zero-norm reading), also when
-    # the query elements lean negative; a tiny-norm token whose projection underflows likewise
+    # the query elements lean negative
     wl = workloads.make_workload("zero-token", seed=19, dtype=torch.bfloat16, batch=2, n_vis=(130, 260),
                                  n_txt=(3, 9), d=128, n_heads=2, rank=8, keep_ratio=0.2)
     wl.Q = -wl.Q.abs()
     wl.X[5] = 0
     wl.X[77] = 0
-    wl.X[140] = wl.X[140] * 1e-30
     wl.Hs = [wl.X.clone()] + wl.Hs[1:]
     _report(wl.name, parity.run_gpu(wl))
 
