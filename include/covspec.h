@@ -88,6 +88,12 @@ typedef struct {
                           streams the snapshot stack on a second stream of the context with this many
                           512-thread blocks per SM (1 or 2; default 1), joined before Eq. 12; 0: the two
                           scores are computed one after the other on the caller's stream           */
+  float conv_tol;      /* the subspace iteration behind Eq. 14 runs a fixed number of steps; after the
+                          last one the library estimates, from the Ritz values, how far the energies
+                          can still be from those of the exact truncated SVD (relative to the largest
+                          energy) and raises COVSPEC_ERR_NOCONVERGE in the device status word when the
+                          estimate exceeds conv_tol (default 2e-3; 0 disables the check).  More steps
+                          (eig_iters) or more extra vectors (eig_oversample) settle such inputs      */
 } covspec_config;
 
 /* One batch of requests (Sec. III-A notation in brackets). */

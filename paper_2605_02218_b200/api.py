@@ -43,7 +43,7 @@ class Config(C.Structure):
         ("max_batch", C.c_int), ("max_total_vis", C.c_longlong), ("max_total_txt", C.c_longlong),
         ("max_vis_per_req", C.c_int), ("max_presel_per_req", C.c_int),
         ("max_total_presel", C.c_longlong), ("relevance_path", C.c_int), ("lowrank_mode", C.c_int),
-        ("ritz_window", C.c_int), ("activity_overlap", C.c_int),
+        ("ritz_window", C.c_int), ("activity_overlap", C.c_int), ("conv_tol", C.c_float),
     ]
 
 

@@ -18,6 +18,7 @@
 #include "greedy_kernels.cuh"
 #include "relevance_tc.cuh"
 #include "subspace_tc.cuh"
+#include "subspace_fused.cuh"
 #include "score_kernels.cuh"
 #include "select_kernels.cuh"
 
@@ -98,6 +99,7 @@ struct covspec_ctx {
   float* Yf[2] = {nullptr, nullptr};     // float32 blocks before / after the last power step
   double* partial = nullptr;
   float *Lbuf = nullptr, *Ub = nullptr;
+  unsigned* sync = nullptr;              // per-request counters of the fused subspace kernel + abort word
   float* Cg = nullptr;                   // factor columns of the greedy low-rank mode
   long long cg_cap = 0;
   CUtensorMap map_zg, map_gh, map_gl, map_y[2][2];
@@ -158,6 +160,7 @@ int validate_cfg(const covspec_config* c) {
   if (c->lowrank_mode < 0 || c->lowrank_mode > 1) return COVSPEC_ERR_ARG;
   if (c->ritz_window < 0) return COVSPEC_ERR_ARG;
   if (c->activity_overlap < 0 || c->activity_overlap > 2) return COVSPEC_ERR_ARG;
+  if (c->eig_iters > 1000 || !(c->conv_tol >= 0.f)) return COVSPEC_ERR_ARG;
   return COVSPEC_OK;
 }
 
@@ -250,31 +253,52 @@ int get_plan(covspec_ctx* ctx, const covspec_problem* p, cudaStream_t stream) {
       pl.total_presel > ctx->cfg.max_total_presel || pl.n_ptiles > ctx->cap_ptiles)
     return COVSPEC_ERR_WORKSPACE;
 
-  // Schedule of the power step: its items differ in cost (basis size p, rows in the tile), so they
-  // are handed to the CTAs longest first, each to the least loaded CTA.
+  // Schedule of the subspace kernel.  Its items (128-row tiles) differ in cost (basis size p, rows
+  // in the tile), and every step of a request ends when its slowest tile does.  With more tiles
+  // than CTAs, consecutive tiles of one request are therefore merged into groups and a group goes
+  // to one CTA as a whole: a CTA that carries several tiles then delays one request instead of
+  // several.  Groups are handed out longest first, each to the least loaded CTA.
   pl.pow_grid = std::min(pl.n_ptiles, ctx->num_sms);
   pl.sched.assign((size_t)pl.pow_grid + 1 + pl.n_ptiles, 0);
   if (pl.n_ptiles > 0) {
-    std::vector<std::pair<double, int>> items;
+    auto tile_cost = [&](const ReqPlan& r, int t) {
+      int rows = std::min(sub::kTile, r.m - t * sub::kTile);
+      double pp = (double)r.p;
+      return pp * pp * (1.0 + 1.5 * rows / sub::kTile) + 64.0 * r.m;
+    };
+    // start with one group per tile; while there are more groups than CTAs, merge the cheapest pair
+    // of neighbouring groups of one request (requests are never mixed inside a group)
+    struct Group { double cost; int first, count, req; };
+    std::vector<Group> groups;
     for (int b = 0; b < B; ++b) {
       const ReqPlan& r = pl.req[b];
       if (!r.stage2) continue;
       int nt = (r.m + sub::kTile - 1) / sub::kTile;
-      for (int t = 0; t < nt; ++t) {
-        int rows = std::min(sub::kTile, r.m - t * sub::kTile);
-        double pp = (double)r.p;
-        items.push_back({pp * pp * (1.0 + 1.5 * rows / sub::kTile) + 64.0 * r.m, r.ptile_off + t});
-      }
+      for (int t = 0; t < nt; ++t) groups.push_back(Group{tile_cost(r, t), r.ptile_off + t, 1, b});
     }
-    std::stable_sort(items.begin(), items.end(), [](const std::pair<double, int>& a, const std::pair<double, int>& b2) { return a.first > b2.first; });
+    while ((int)groups.size() > pl.pow_grid) {
+      int best = -1;
+      double best_cost = 0.0;
+      for (int g = 0; g + 1 < (int)groups.size(); ++g) {
+        if (groups[g].req != groups[g + 1].req) continue;
+        double c = groups[g].cost + groups[g + 1].cost;
+        if (best < 0 || c < best_cost) { best = g; best_cost = c; }
+      }
+      if (best < 0) break;                         // more requests than CTAs: the hand-out below stacks them
+      groups[best].cost = best_cost;
+      groups[best].count += groups[best + 1].count;
+      groups.erase(groups.begin() + best + 1);
+    }
+    std::stable_sort(groups.begin(), groups.end(), [](const Group& a, const Group& b2) { return a.cost > b2.cost; });
     std::vector<double> load(pl.pow_grid, 0.0);
     std::vector<std::vector<int>> lists(pl.pow_grid);
-    for (const auto& it : items) {
+    for (const Group& g : groups) {
       int best = 0;
-      for (int g = 1; g < pl.pow_grid; ++g) if (load[g] < load[best]) best = g;
-      load[best] += it.first;
-      lists[best].push_back(it.second);
+      for (int c = 1; c < pl.pow_grid; ++c) if (load[c] < load[best]) best = c;
+      load[best] += g.cost;
+      for (int t = 0; t < g.count; ++t) lists[best].push_back(g.first + t);
     }
+    // more groups than CTAs is guaranteed to leave no CTA empty only if groups >= CTAs
     int off = 0;
     int* items_out = pl.sched.data() + pl.pow_grid + 1;
     for (int g = 0; g < pl.pow_grid; ++g) {
@@ -609,36 +633,30 @@ int select_impl(covspec_ctx* ctx, const covspec_problem* p, const float* s_fused
       return COVSPEC_OK;
     }
     sub::basis_init_kernel<<<gb, 256, 0, s>>>(ctx->d_plan, ctx->Yp[0][0], ctx->Yp[0][1], ctx->Yp[1][0],
-                                              ctx->Yp[1][1], ctx->ld);
+                                              ctx->Yp[1][1], ctx->ld, energy, ctx->sync, B);
     LAUNCH_CHECK(ctx);
-    int grid = pl.pow_grid;
-    for (int pass = 0; pass <= cfg.eig_iters; ++pass) {
-      sub::PowerParams pp{};
-      pp.plan = ctx->d_plan; pp.batch = B; pp.n_items = pl.n_ptiles; pp.sched = ctx->d_sched;
-      pp.identity = pass == 0;
-      pp.lbuf = ctx->Lbuf;
-      int in = pass & 1, out = in ^ 1;
-      pp.y_hi = ctx->Yp[out][0]; pp.y_lo = ctx->Yp[out][1]; pp.ld = ctx->ld;
-      // the two last blocks are also kept in float32 for the energy kernel
-      pp.yf = pass == cfg.eig_iters ? ctx->Yf[1] : pass == cfg.eig_iters - 1 ? ctx->Yf[0] : nullptr;
-      pp.qprev = pass == cfg.eig_iters ? ctx->Yf[0] : nullptr;
-      pp.partial = ctx->partial; pp.status = ctx->status;
-      sub::power_tc_kernel<<<grid, sub::kPowThreads, sub::kPowSmem, s>>>(
-          ctx->map_gh, ctx->map_gl, ctx->map_y[in][0], ctx->map_y[in][1], pp);
-      LAUNCH_CHECK(ctx);
-      if (pass < cfg.eig_iters) {
-        chol_kernel<<<B, 512, cholesky_smem_bytes(pl.p_max), s>>>(ctx->d_plan, ctx->partial, ctx->Lbuf);
-        LAUNCH_CHECK(ctx);
-      }
-    }
-    size_t ritz_smem = ritz_smem_bytes(pl.win_max);
-    ritz_kernel<<<B, 512, ritz_smem, s>>>(ctx->d_plan, ctx->partial, ctx->Ub, 30, ctx->status);
+    // every multiplication by G, the factorisations between them, the Rayleigh-Ritz solve and the
+    // energies: one cooperative launch (its CTAs wait on one another through global counters)
+    sub::FusedParams fp{};
+    fp.plan = ctx->d_plan; fp.batch = B; fp.n_items = pl.n_ptiles; fp.sched = ctx->d_sched;
+    fp.steps = cfg.eig_iters + 1;
+    fp.lbuf = ctx->Lbuf;
+    for (int i = 0; i < 2; ++i) { fp.y_hi[i] = ctx->Yp[i][0]; fp.y_lo[i] = ctx->Yp[i][1]; fp.yf[i] = ctx->Yf[i]; }
+    fp.ld = ctx->ld;
+    fp.partial = ctx->partial; fp.ub = ctx->Ub; fp.energy = energy; fp.sync = ctx->sync;
+    fp.max_sweeps = 30; fp.conv_tol = cfg.conv_tol; fp.status = ctx->status;
+    void* args[] = {&ctx->map_gh, &ctx->map_gl, &ctx->map_y[0][0], &ctx->map_y[0][1], &ctx->map_y[1][0],
+                    &ctx->map_y[1][1], &fp};
+    CUDA_TRY(cudaLaunchCooperativeKernel(reinterpret_cast<void*>(sub::subspace_kernel), dim3(pl.pow_grid),
+                                         dim3(sub::kPowThreads), args, sub::kPowSmem, s));
+    LAUNCH_CHECK(ctx);
+  } else {
+    // no request reaches stage 2: the final selection keeps the preselected sets; energies are zero
+    dim3 gz(1, B);
+    sub::basis_init_kernel<<<gz, 256, 0, s>>>(ctx->d_plan, ctx->Yp[0][0], ctx->Yp[0][1], ctx->Yp[1][0],
+                                              ctx->Yp[1][1], ctx->ld, energy, ctx->sync, B);
     LAUNCH_CHECK(ctx);
   }
-  dim3 ge((pl.m_max + 63) / 64, B);
-  size_t en_smem = (size_t)pl.win_max * pl.nbot_max * sizeof(float);
-  energy_kernel<<<ge, 256, en_smem, s>>>(ctx->d_plan, ctx->Yf[0], ctx->Yf[1], ctx->Ub, energy);
-  LAUNCH_CHECK(ctx);
   if (pl.n_stage2 > 0) prof_mark(ctx, ST_EIG, 1, s);
   prof_mark(ctx, ST_FINAL, 0, s);
   final_select_kernel<<<B, 1024, 0, s>>>(energy, presel, ctx->d_plan, keep_idx, ctx->status);
@@ -695,6 +713,7 @@ void covspec_default_config(covspec_config* c) {
   c->lowrank_mode = 0;
   c->ritz_window = 16;
   c->activity_overlap = 1;
+  c->conv_tol = 2e-3f;
 }
 
 int covspec_budgets(const covspec_config* cfg, int n, int keep, int* b_vis, int* m, int* r) {
@@ -768,9 +787,10 @@ int covspec_prune_init(const covspec_config* cfg, covspec_ctx** out) {
   long long o_y[2][2];
   for (int i = 0; i < 2; ++i) for (int j = 0; j < 2; ++j) o_y[i][j] = carve(yplane);
   long long o_yf0 = carve(4ll * ctx->cap_rows * kPMax), o_yf1 = carve(4ll * ctx->cap_rows * kPMax);
-  long long o_part = carve(8ll * ctx->cap_ptiles * sub::kTriMax);
+  long long o_part = carve(8ll * ctx->cap_ptiles * sub::kTileDoubles);
   long long o_lbuf = carve(4ll * c.max_batch * sub::kLbufStride);
   long long o_ub = carve(4ll * c.max_batch * kPMax * kPMax);
+  long long o_sync = carve(4ll * (c.max_batch * sub::kSyncStride + 4));
   ctx->cg_cap = c.lowrank_mode == 1 ? (long long)c.max_total_presel * c.max_presel_per_req : 0;
   long long o_cg = carve(4ll * ctx->cg_cap);
   ctx->ws_bytes = off;
@@ -803,6 +823,7 @@ int covspec_prune_init(const covspec_config* cfg, covspec_ctx** out) {
   ctx->partial = reinterpret_cast<double*>(w + o_part);
   ctx->Lbuf = reinterpret_cast<float*>(w + o_lbuf);
   ctx->Ub = reinterpret_cast<float*>(w + o_ub);
+  ctx->sync = reinterpret_cast<unsigned*>(w + o_sync);
   ctx->Cg = reinterpret_cast<float*>(w + o_cg);
   ctx->stage_bytes = round_up(sizeof(ReqPlan) * c.max_batch, 256) +
                      sizeof(GemmProb) * (long long)T_COUNT * c.max_batch;
@@ -815,12 +836,6 @@ int covspec_prune_init(const covspec_config* cfg, covspec_ctx** out) {
             cudaEventCreateWithFlags(&ctx->ev_fork, cudaEventDisableTiming) == cudaSuccess &&
             cudaEventCreateWithFlags(&ctx->ev_join, cudaEventDisableTiming) == cudaSuccess;
   // the small dense kernels need more than the default 48 KB of dynamic shared memory
-  ok = ok && cudaFuncSetAttribute(chol_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                  (int)cholesky_smem_bytes(kPMax)) == cudaSuccess;
-  ok = ok && cudaFuncSetAttribute(ritz_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                  (int)ritz_smem_bytes(kPMax)) == cudaSuccess;
-  ok = ok && cudaFuncSetAttribute(energy_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                  (int)((size_t)kPMax * kPMax * sizeof(float))) == cudaSuccess;
   int dev = 0, cc_major = 0;
   ok = ok && cudaGetDevice(&dev) == cudaSuccess &&
        cudaDeviceGetAttribute(&ctx->num_sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess &&
@@ -838,7 +853,7 @@ int covspec_prune_init(const covspec_config* cfg, covspec_ctx** out) {
                              tc::kSmemBytes) == cudaSuccess &&
         cudaFuncSetAttribute(sub::gram_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              sub::kGramSmem) == cudaSuccess &&
-        cudaFuncSetAttribute(sub::power_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaFuncSetAttribute(sub::subspace_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              sub::kPowSmem) == cudaSuccess;
     ok = ctx->tc_ready;
   }

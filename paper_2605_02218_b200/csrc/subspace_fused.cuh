@@ -1,0 +1,855 @@
+// The whole subspace iteration behind Eq. 14-15 in one persistent kernel.
+//
+// Work items are the 128-row tiles of the stage-2 requests (the same items and per-CTA lists as the
+// power step had as a kernel of its own); every CTA walks its list once per multiplication by G.
+// What used to be kernel boundaries are per-request counters in global memory:
+//   arrive[b]   tiles of request b that have finished a step (their slab of the new block is in the
+//               bf16 planes, their float64 partial Gram matrix is in `partial`); step k of a tile may
+//               start loading the block once arrive[b] >= tiles(b) * k
+//   factor[b]   number of triangular factors published for request b; the epilogue of step k needs
+//               factor[b] >= k
+//   ritz[b]     1 once the Rayleigh-Ritz vectors of the last block are published
+// The tile that makes arrive[b] reach tiles(b) * (k + 1) (an atomic ticket; nobody waits for it to be
+// a particular CTA) sums the partial Gram matrices in tile order and factors the sum right there: a
+// Cholesky factorisation after the first steps, the Rayleigh-Ritz solve of the window next to the cut
+// after the last one.  All CTAs are resident at the same time (cooperative launch, one CTA per SM),
+// every wait is bounded and a CTA that gives up raises a global abort word that ends the others'
+// waits too.  After the last step every CTA evaluates the energies (Eq. 15) of its own tiles.
+//
+// Data that crosses CTAs inside the kernel (partial sums, factors, Ritz vectors, the float32 blocks)
+// is read with L1-bypassing loads; the bf16 planes are read by TMA, behind a proxy fence.
+#pragma once
+#include "eig_kernels.cuh"
+
+namespace covspec {
+namespace sub {
+
+constexpr int kSyncStride = 4;           // unsigned words per request: arrive, factor, ritz, unused
+
+struct FusedParams {
+  const ReqPlan* plan;
+  int batch;
+  int n_items;              // 128-row tiles over all stage-2 requests
+  const int* sched;         // [gridDim.x + 1] offsets, then the item lists of every CTA
+  int steps;                // multiplications by G (eig_iters + 1, >= 2)
+  float* lbuf;              // [batch][kLbufStride] triangular factor + reciprocal diagonal
+  __nv_bfloat16* y_hi[2];   // plane buffers: step k reads [k & 1], writes [(k & 1) ^ 1]
+  __nv_bfloat16* y_lo[2];
+  int ld;
+  float* yf[2];             // [sum M_b, kPMax]: the block before the last multiplication (turned into
+                            // the orthonormal basis Q during the last step) and after it
+  double* partial;          // [tiles][kTileDoubles], see tile_offset
+  float* ub;                // [batch][kPMax * kPMax] Ritz vectors of the discarded pairs
+  float* energy;            // [sum M_b] (out)
+  unsigned* sync;           // [batch][kSyncStride] counters (zero on entry), then the abort word
+  int max_sweeps;
+  float conv_tol;           // bound on the estimated energy error before NOCONVERGE is raised
+  int* status;
+};
+
+__device__ __forceinline__ unsigned ld_acquire_u32(const unsigned* p) {
+  unsigned v;
+  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ void st_release_u32(unsigned* p, unsigned v) {
+  asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ void fence_proxy_async_all() {
+  asm volatile("fence.proxy.async;" ::: "memory");
+}
+
+constexpr uint32_t kFlagSpinLimit = 1u << 21;       // polls of ~100 ns: gives up after a fraction of a second
+
+// One thread waits until *ctr >= target.  Returns false when the limit expired (raises the global
+// abort word) or another CTA gave up.
+__device__ __forceinline__ bool flag_wait_ge(const unsigned* ctr, unsigned target, unsigned* gabort,
+                                             volatile int* abort_flag) {
+  for (uint32_t i = 0; i < kFlagSpinLimit; ++i) {
+    if (ld_acquire_u32(ctr) >= target) return true;
+    if ((i & 15u) == 15u && (ld_acquire_u32(gabort) != 0u || *abort_flag)) { *abort_flag = 1; return false; }
+    __nanosleep(64);
+  }
+  *abort_flag = 1;
+  atomicExch(gabort, 1u);
+  return false;
+}
+
+// Layout of a partial Gram matrix in global memory: the 8 x 8 tiles of the lower triangle, tile
+// (I, J <= I) at tri_index(I, J) * 64, row-major inside (diagonal tiles hold all 64 entries) - the
+// layout the blocked factorisation works on, so that summing the tiles' partial matrices is an
+// element-wise sum of contiguous arrays.
+constexpr int kTileDoubles = (kPMax / 8) * (kPMax / 8 + 1) / 2 * 64;      // 13440
+__device__ __forceinline__ int tile_offset(int i, int j) {                 // i >= j
+  return tri_index(i >> 3, j >> 3) * 64 + (i & 7) * 8 + (j & 7);
+}
+// One entry summed over the tiles of a request in tile order (L1-bypassing loads, 8 in flight).
+__device__ __forceinline__ double gram_entry_cg(int ntile, const double* src) {
+  double s = 0.0;
+  for (int t0 = 0; t0 < ntile; t0 += 8) {
+    double v[8];
+#pragma unroll
+    for (int q = 0; q < 8; ++q) v[q] = __ldcg(src + (size_t)min(t0 + q, ntile - 1) * kTileDoubles);
+#pragma unroll
+    for (int q = 0; q < 8; ++q) s += t0 + q < ntile ? v[q] : 0.0;
+  }
+  return s;
+}
+// T[0 .. count) = sum over the request's tiles (tile order: deterministic) of their partial
+// matrices; count a multiple of 64.  Coalesced 16-byte loads, 16 of them in flight per thread.
+__device__ __forceinline__ void team_sum_partials(double* T, const double* pbase, int ntile, int count,
+                                                  int tid, int nthreads) {
+  const int pairs = count >> 1;
+  for (int e0 = tid; e0 < pairs; e0 += 2 * nthreads) {
+    const int e1 = e0 + nthreads;
+    const bool have1 = e1 < pairs;
+    double2 s0 = make_double2(0.0, 0.0), s1 = s0;
+    for (int t0 = 0; t0 < ntile; t0 += 8) {
+      double2 v0[8], v1[8];
+#pragma unroll
+      for (int q = 0; q < 8; ++q) {
+        const double2* src = reinterpret_cast<const double2*>(pbase + (size_t)min(t0 + q, ntile - 1) * kTileDoubles);
+        v0[q] = __ldcg(src + e0);
+        v1[q] = __ldcg(src + (have1 ? e1 : e0));
+      }
+#pragma unroll
+      for (int q = 0; q < 8; ++q) {
+        if (t0 + q < ntile) { s0.x += v0[q].x; s0.y += v0[q].y; s1.x += v1[q].x; s1.y += v1[q].y; }
+      }
+    }
+    reinterpret_cast<double2*>(T)[e0] = s0;
+    if (have1) reinterpret_cast<double2*>(T)[e1] = s1;
+  }
+}
+
+// ---- float64 Cholesky factorisation by the eight epilogue warps --------------------------------
+// Same blocked right-looking scheme as cholesky_blocked, for `nthreads` threads (whole warps, thread
+// index tid) that synchronise through `sync()`.
+// 1 / sqrt(x) for x > 0 without a range test on the pivot chain: x = m 4^k with m in [1, 4) (integer
+// operations on the exponent field), float32 estimate of 1 / sqrt(m) refined in float32 and by one
+// Newton step in float64, then scaled by 2^-k.  Subnormal or non-finite x give a meaningless value;
+// the caller clamps pivots to a positive floor first.
+__device__ __forceinline__ double rsqrt_f64_scaled(double x) {
+  const int hi = __double2hiint(x), lo = __double2loint(x);
+  const int k = ((((hi >> 20) & 0x7ff) - 1023)) >> 1;
+  const double m = __hiloint2double(hi - (k << 21), lo);
+  const float xf = (float)m;
+  float yf = rsqrtf(xf);
+  yf = yf * (1.5f - 0.5f * xf * yf * yf);
+  double y = (double)yf;
+  const double e = fma(-0.5 * m * y, y, 0.5);
+  y = fma(y, e, y);
+  return __hiloint2double(__double2hiint(y) - (k << 20), __double2loint(y));
+}
+
+// Diagonal 8 x 8 tile, factored by one thread in registers: measured faster than a lane-per-row
+// version (64-bit shuffles cost more than the arithmetic they save).  The chain of eight dependent
+// reciprocal square roots is the critical path of the whole factorisation, which is why the caller
+// keeps the other warps of this thread's scheduler off the FP64 pipe meanwhile.
+__device__ __forceinline__ void factor_diag_thread(double* D, const double* d0, double* rd) {
+  double a[8][8];
+#pragma unroll
+  for (int l = 0; l < 8; ++l)
+#pragma unroll
+    for (int m = 0; m <= l; ++m) a[l][m] = D[l * 8 + m];
+#pragma unroll
+  for (int c = 0; c < 8; ++c) {
+    double piv = a[c][c];
+    const double floor_ = 1e-12 * d0[c];
+    if (!(piv > floor_)) piv = floor_ > 0.0 ? floor_ : 1.0;
+    const double rs = rsqrt_f64_scaled(piv);
+    a[c][c] = piv * rs;
+    rd[c] = rs;
+#pragma unroll
+    for (int l = c + 1; l < 8; ++l) a[l][c] *= rs;
+#pragma unroll
+    for (int l = c + 1; l < 8; ++l)
+#pragma unroll
+      for (int m = c + 1; m <= l; ++m) a[l][m] -= a[l][c] * a[m][c];
+  }
+#pragma unroll
+  for (int l = 0; l < 8; ++l)
+#pragma unroll
+    for (int m = 0; m <= l; ++m) D[l * 8 + m] = a[l][m];
+}
+
+// The matrix is already in T (tile layout, see tile_offset); entries beyond n inside the last row of
+// tiles are replaced by the identity here.
+//   store(I, J, tile, rd)   receives the factor tile (I, J) (64 doubles, row-major) and the array of
+//                           reciprocal diagonal entries; called by a whole warp
+template <typename Store, typename Sync>
+__device__ __forceinline__ void cholesky_blocked_team(int n, double* T, double* aux, int tid, int nthreads,
+                                                      Store store, Sync sync) {
+  const int lane = tid & 31, warp = tid >> 5, nw = nthreads >> 5;
+  const int nb = (n + 7) >> 3, ntile = nb * (nb + 1) / 2;
+  double* d0 = aux;                 // original diagonal
+  double* rd = aux + 8 * nb;        // 1 / L[j][j]
+  // identity padding of rows / columns n .. 8 nb - 1 (last row of tiles), then the diagonal
+  for (int e = tid; e < nb * 64; e += nthreads) {
+    const int J = e >> 6, i = 8 * (nb - 1) + ((e >> 3) & 7), j = 8 * J + (e & 7);
+    if (i >= n || j >= n) T[tri_index(nb - 1, J) * 64 + (e & 63)] = (i == j) ? 1.0 : 0.0;
+  }
+  sync();
+  for (int i = tid; i < 8 * nb; i += nthreads) d0[i] = T[tile_offset(i, i)];
+  sync();
+  const int fr = lane >> 2, fk = lane & 3;
+  auto update_tile = [&](int J, int I, int K) {
+    const double* XI = T + tri_index(I, J) * 64 + fr * 8 + fk;
+    const double* XK = T + tri_index(K, J) * 64 + fr * 8 + fk;
+    double* C = T + tri_index(I, K) * 64 + fr * 8 + 2 * fk;
+    double c0 = C[0], c1 = C[1];
+    dmma_8x8x4(c0, c1, -XI[0], XK[0]);
+    dmma_8x8x4(c0, c1, -XI[4], XK[4]);
+    C[0] = c0; C[1] = c1;
+  };
+  if (tid == 0) factor_diag_thread(T, d0, rd);
+  sync();
+  for (int J = 0; J < nb; ++J) {
+    const double* D = T + tri_index(J, J) * 64;
+    for (int i = 8 * (J + 1) + tid; i < 8 * nb; i += nthreads) {
+      double* row = T + tri_index(i >> 3, J) * 64 + (i & 7) * 8;
+      double x[8];
+#pragma unroll
+      for (int c = 0; c < 8; ++c) x[c] = row[c];
+#pragma unroll
+      for (int c = 0; c < 8; ++c) {
+        double v = x[c];
+#pragma unroll
+        for (int k = 0; k < c; ++k) v -= x[k] * D[c * 8 + k];
+        x[c] = v * rd[8 * J + c];
+      }
+#pragma unroll
+      for (int c = 0; c < 8; ++c) row[c] = x[c];
+    }
+    sync();
+    if (J + 1 == nb) break;
+    for (int I = J + 1 + warp; I < nb; I += nw) update_tile(J, I, J + 1);
+    sync();
+    // The next diagonal tile is factored by one thread while the trailing matrix is updated by the
+    // warps of the other three schedulers (warp w issues on scheduler w & 3; the FP64 pipe is per
+    // scheduler, and the pivot chain must not queue behind the updates).
+    if ((warp & 3) == 0) {
+      if (tid == 0) factor_diag_thread(T + tri_index(J + 1, J + 1) * 64, d0 + 8 * (J + 1), rd + 8 * (J + 1));
+      __syncwarp();
+    } else {
+      const int mrem = nb - J - 2, ntr = mrem * (mrem + 1) / 2;
+      const int nworkers = nw - (nw + 3) / 4, me = warp - (warp >> 2) - 1;   // warps with (w & 3) != 0, in order
+      for (int q = me; q < ntr; q += nworkers) {
+        int ii, kk;
+        tri_decode(q, ii, kk);
+        update_tile(J, J + 2 + ii, J + 2 + kk);
+      }
+    }
+    sync();
+  }
+  for (int t = warp; t < ntile; t += nw) {
+    int I, J;
+    tri_decode(t, I, J);
+    store(I, J, T + t * 64, rd);
+  }
+}
+
+constexpr int kEpiThreads = 256;         // warps 0-7
+
+// Writes the accumulated 8 x 8 tiles of one warp unit (see gram_unit_accumulate) to the tile layout;
+// t0 = index of the first tile row / column the unit's coordinates are relative to.
+__device__ __forceinline__ void gram_unit_store_tiles(const GramAcc& acc, int ta, int tz, int t0, int lane,
+                                                      double* __restrict__ out) {
+  const int fr = lane >> 2, fk = lane & 3;
+#pragma unroll
+  for (int u = 0; u <= kMaxTiles8; ++u) {
+    int strip = -1, tb = 0;
+    if (u < kMaxTiles8 && u <= ta) { strip = ta; tb = u; }
+    else if (u >= 1 && kMaxTiles8 - u <= tz && tz != ta) { strip = tz; tb = kMaxTiles8 - u; }
+    if (strip < 0) continue;
+    *reinterpret_cast<double2*>(out + tri_index(t0 + strip, t0 + tb) * 64 + fr * 8 + 2 * fk) =
+        make_double2(acc.a[u][0], acc.a[u][1]);
+  }
+}
+
+// 8 x 8 tiles of the partial Gram matrix that do not fit the eight warp units (see the kernel): the
+// strips ta = u and tz = nb8 - 1 - u of the units u = 8 .. units - 1, listed strip by strip.
+// nb8 <= 20 leaves at most 2 units = 42 tiles, six per warp.
+constexpr int kExtraTiles = 6;
+__device__ __forceinline__ bool extra_tile(int e, int nb8, int units, int& ta, int& tb) {
+  for (int u = 8; u < units; ++u) {
+    const int a = u, z = nb8 - 1 - u;
+    if (e <= a) { ta = a; tb = e; return true; }
+    e -= a + 1;
+    if (z != a) {
+      if (e <= z) { ta = z; tb = e; return true; }
+      e -= z + 1;
+    }
+  }
+  return false;
+}
+
+
+// ---- work of the tile that finishes a step last (all 256 epilogue threads) ----------------------
+// Kept out of line: the tile epilogue is register-bound, and these run once per request and step.
+
+// Cholesky factor of the summed Gram matrix, written in the layout the triangular solve reads
+// (see lt_row_offset) followed by the reciprocal diagonal.  Tm: cholesky_smem_bytes(p) of scratch.
+__device__ __noinline__ void team_cholesky(const double* pbase, int nt, int p, float* out, double* Tm) {
+  const int et = threadIdx.x, warp = et >> 5, lane = et & 31;
+  const int P = (p + 7) & ~7, nb = (p + 7) >> 3;
+  auto epi_sync = [&]() { named_barrier(1, kEpiThreads); };
+  // identity padding of the layout rows / columns p .. P-1 and the entries left of the diagonal
+  for (int i = warp; i < P; i += 8) {
+    int j0 = i & ~3;
+    float* row = out + lt_row_offset(i, P) - j0;
+    for (int j = j0 + lane; j < P; j += 32)
+      if (j < i || i >= p || j >= p) row[j] = (i == j) ? 1.f : 0.f;
+  }
+  for (int j = p + et; j < P; j += kEpiThreads) out[kLtFloats + j] = 1.f;
+  team_sum_partials(Tm, pbase, nt, nb * (nb + 1) / 2 * 64, et, kEpiThreads);
+  epi_sync();
+  // row j of the layout holds L[i][j] for i >= (j & ~3): lane -> (j, half of the tile's rows), so that
+  // a lane's four entries are consecutive floats
+  auto store = [&](int I, int J, const double* tile, const double* rd) {
+    const int jl = lane >> 2, i0 = (lane & 3) * 2;
+    const int j = 8 * J + jl;
+    if (j < p) {
+      float* dst = out + lt_row_offset(j, P) - (j & ~3);
+#pragma unroll
+      for (int q = 0; q < 2; ++q) {
+        const int i = 8 * I + i0 + q;
+        if (i < p && i >= j) dst[i] = (float)tile[(i0 + q) * 8 + jl];
+      }
+      if (I == J && (lane & 3) == 0) out[kLtFloats + j] = (float)rd[j];
+    }
+  };
+  cholesky_blocked_team(p, Tm, Tm + (size_t)nb * (nb + 1) / 2 * 64, et, kEpiThreads, store, epi_sync);
+}
+
+// Rayleigh-Ritz on the window next to the cut (see eig_kernels.cuh) and the convergence estimate.
+// C: ritz_smem_bytes(w) of scratch; dg: p floats of scratch.
+__device__ __noinline__ void team_ritz(const double* pbase, int nt, int p, int w, int r, int m, float* out_u,
+                                       float* C, float* dg, float* s_scale, int* s_flag, int max_sweeps,
+                                       float conv_tol, int steps, int* status) {
+  const int et = threadIdx.x, warp = et >> 5, lane = et & 31;
+  auto epi_sync = [&]() { named_barrier(1, kEpiThreads); };
+  const int w0 = p - w, nbot = p - r;
+  const int ldc = ritz_ldc(w);
+  float* sig = C + (size_t)w * ldc;
+  for (int e = et; e < w * ldc; e += kEpiThreads) C[e] = 0.f;
+  if (et == 0) *s_scale = 0.f;
+  epi_sync();
+  {
+    float mx = 0.f;
+    for (int i = et; i < p; i += kEpiThreads) {
+      float v = (float)gram_entry_cg(nt, pbase + tile_offset(i, i));
+      dg[i] = sqrtf(fmaxf(v, 0.f));                      // sqrt of the diagonal of B'
+      mx = fmaxf(mx, v);
+    }
+    mx = warp_max(mx);
+    if (lane == 0 && mx > 0.f) atomicMax(reinterpret_cast<int*>(s_scale), __float_as_int(mx));
+  }
+  {
+    // the window block of B' (rows / columns w0 .. p-1), gathered into a tile layout of its own
+    const int nbw = (w + 7) >> 3, cnt = nbw * (nbw + 1) / 2 * 64;
+    double* Tw = reinterpret_cast<double*>(C + (((size_t)w * ldc + w + 1) & ~(size_t)1));
+    for (int e = et; e < cnt; e += kEpiThreads) {
+      int I, J;
+      tri_decode(e >> 6, I, J);
+      int i = 8 * I + ((e >> 3) & 7), j = 8 * J + (e & 7);
+      double v = 0.0;
+      if (i < w && j < w) v = gram_entry_cg(nt, pbase + tile_offset(w0 + max(i, j), w0 + min(i, j)));
+      Tw[e] = v;
+    }
+    epi_sync();
+    auto store = [&](int I, int J, const double* tile, const double*) {
+      for (int q = lane; q < 64; q += 32) {
+        const int i = 8 * I + (q >> 3), j = 8 * J + (q & 7);
+        if (i < w && j <= i) C[j * ldc + i] = (float)tile[q];
+      }
+    };
+    cholesky_blocked_team(w, Tw, Tw + (size_t)cnt, et, kEpiThreads, store, epi_sync);
+  }
+  epi_sync();
+  const float s1 = sqrtf(*s_scale);
+  if (conv_tol > 0.f && p < m) {
+    // Has the iteration settled?  The basis vectors converge to eigenvectors in order, so
+    // theta_k ~ sqrt(B'_kk) estimates the k-th eigenvalue of G and theta_min the first one left
+    // out of the basis.  After q multiplications a kept direction k still carries about
+    // (theta_min / theta_k)^q of the directions outside the basis, which moves the energies by
+    // about 2 theta_k (theta_min / theta_k)^q; relative to the scale theta_1 of the energies, and
+    // only for directions that the cut can tell apart from the discarded ones (more than
+    // 1e-3 theta_1 above theta_min; closer ones may mix freely, Eq. 15 is not unique there).
+    float tmin = 3.0e38f;
+    for (int i = lane; i < p; i += 32) tmin = fminf(tmin, dg[i]);
+    tmin = warp_min(tmin);
+    float worst = 0.f;
+    for (int i = et; i < r; i += kEpiThreads) {
+      float th = dg[i];
+      if (th - tmin > 1e-3f * s1 && th > 0.f)
+        worst = fmaxf(worst, 2.f * (th / s1) * __powf(tmin / th, (float)steps));
+    }
+    worst = warp_max(worst);
+    if (lane == 0 && worst > conv_tol) atomicOr(status, kStatusNoConverge);
+  }
+  const int nact = min(kEpiThreads, ((((w + 1) >> 1) * 4) + 31) & ~31);
+  if (et == 0) *s_flag = 0;
+  epi_sync();
+  if (et < nact) {
+    bool converged;
+    if (w <= 32) converged = jacobi_sweeps<8>(C, ldc, w, s1, max_sweeps, nact, s_flag);
+    else if (w <= 64) converged = jacobi_sweeps<16>(C, ldc, w, s1, max_sweeps, nact, s_flag);
+    else if (w <= 96) converged = jacobi_sweeps<24>(C, ldc, w, s1, max_sweeps, nact, s_flag);
+    else converged = jacobi_sweeps<(kPMax + 3) / 4>(C, ldc, w, s1, max_sweeps, nact, s_flag);
+    if (!converged && et == 0) atomicOr(status, kStatusNoConverge);
+  }
+  named_barrier(3, kEpiThreads);
+  for (int k = warp; k < w; k += 8) {
+    float sm = 0.f;
+    for (int row = lane; row < w; row += 32) { float x = C[k * ldc + row]; sm += x * x; }
+    sm = warp_sum(sm);
+    if (lane == 0) sig[k] = sqrtf(sm);
+  }
+  epi_sync();
+  // rank the columns by singular value (ascending, ties by larger index first); the nbot smallest
+  // become unit vectors out_u[j * nbot + rank]
+  for (int k = warp; k < w; k += 8) {
+    float sk = sig[k];
+    int rank = 0;
+    for (int q = lane; q < w; q += 32) {
+      float sq = sig[q];
+      rank += (sq < sk) || (sq == sk && q > k);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) rank += __shfl_xor_sync(0xffffffffu, rank, o);
+    if (rank < nbot) {
+      float scale = sk > 0.f ? 1.f / sk : 0.f;
+      for (int j = lane; j < w; j += 32) out_u[j * nbot + rank] = C[k * ldc + j] * scale;
+    }
+  }
+}
+
+__global__ void __launch_bounds__(kPowThreads, 1)
+subspace_kernel(const __grid_constant__ CUtensorMap map_gh, const __grid_constant__ CUtensorMap map_gl,
+                const __grid_constant__ CUtensorMap map_y0h, const __grid_constant__ CUtensorMap map_y0l,
+                const __grid_constant__ CUtensorMap map_y1h, const __grid_constant__ CUtensorMap map_y1l,
+                const FusedParams prm) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  float* xs = reinterpret_cast<float*>(smem);                       // aliases the ring after the MMAs
+  float* xq = reinterpret_cast<float*>(smem + kXsBytes);            // previous block (last step)
+  float* lt = reinterpret_cast<float*>(smem + kPowRegion);
+  float* dinv = lt + kLtFloats;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(lt + kLbufStride);
+  uint64_t* full = bars;                 // [2]
+  uint64_t* empty = bars + 2;            // [2]
+  uint64_t* acc_full = bars + 4;
+  uint64_t* acc_empty = bars + 5;
+  uint64_t* epi_done = bars + 6;         // the region no longer belongs to the epilogue
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 8);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  volatile int* s_word = reinterpret_cast<volatile int*>(tmem_slot + 2);      // broadcast slot of the epilogue
+  int* s_flag = reinterpret_cast<int*>(tmem_slot + 3);                        // Jacobi rotation flag
+  float* s_scale = reinterpret_cast<float*>(tmem_slot + 4);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  unsigned* gabort = prm.sync + (size_t)prm.batch * kSyncStride;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kPowStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+    mbar_init(acc_full, 1);
+    mbar_init(acc_empty, 128);
+    mbar_init(epi_done, kEpiThreads);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 9) tmem_alloc(tmem_slot, kPowTmemCols);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  const int s_begin = prm.sched[blockIdx.x], s_end = prm.sched[blockIdx.x + 1];
+  const int* s_items = prm.sched + gridDim.x + 1;
+  const int last_step = prm.steps - 1;
+  auto decode = [&](int item, int& b, ReqPlan& rp, int& tile) {
+    b = find_request(item, prm.batch, [&](int q) { return prm.plan[q].ptile_off; });
+    rp = prm.plan[b];
+    tile = item - rp.ptile_off;
+  };
+
+  if (warp == 8) {
+    // ------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      uint32_t it = 0, n = 0;
+      bool ok = true;
+      for (int step = 0; step <= last_step && ok; ++step) {
+        const CUtensorMap* myh = (step & 1) ? &map_y1h : &map_y0h;
+        const CUtensorMap* myl = (step & 1) ? &map_y1l : &map_y0l;
+        for (int si = s_begin; si < s_end && ok; ++si, ++n) {
+          const int item = s_items[si];
+          int b, tile; ReqPlan rp;
+          decode(item, b, rp, tile);
+          // the previous item's staged block (and whatever its last tile factored) lives in the
+          // ring until its epilogue is done
+          if (n > 0 && !(ok = mbar_wait(epi_done, (n - 1) & 1u, abort_flag))) break;
+          if (step > 0) {
+            // every tile of the request has written its slab of the block this step multiplies
+            const unsigned nt = (unsigned)((rp.m + kTile - 1) / kTile);
+            if (!(ok = flag_wait_ge(prm.sync + (size_t)b * kSyncStride, nt * (unsigned)step, gabort, abort_flag))) break;
+            fence_proxy_async_all();
+          }
+          int k_chunks = (rp.m + kBK - 1) / kBK;
+          for (int kc = 0; kc < k_chunks; ++kc, ++it) {
+            int s = it % kPowStages;
+            if (!(ok = mbar_wait(&empty[s], ((it / kPowStages) & 1u) ^ 1u, abort_flag))) break;
+            mbar_expect_tx(&full[s], kPowStageBytes);
+            uint32_t dst = smem_u32(smem + s * kPowStageBytes);
+            int grow = rp.presel_off + tile * kTile;
+            tma_load_2d(dst, &map_gh, kc * kBK, grow, &full[s]);
+            tma_load_2d(dst + kPowBytesA, &map_gl, kc * kBK, grow, &full[s]);
+            tma_load_2d(dst + 2 * kPowBytesA, myh, kc * kBK, b * kPMax, &full[s]);
+            tma_load_2d(dst + 2 * kPowBytesA + kPowBytesB, myl, kc * kBK, b * kPMax, &full[s]);
+          }
+        }
+      }
+    }
+    __syncwarp();
+  } else if (warp == 9) {
+    // ------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      uint32_t it = 0, n = 0;
+      bool ok = true;
+      for (int step = 0; step <= last_step && ok; ++step) {
+        for (int si = s_begin; si < s_end && ok; ++si, ++n) {
+          const int item = s_items[si];
+          int b, tile; ReqPlan rp;
+          decode(item, b, rp, tile);
+          const uint32_t idesc = umma_idesc(kTile, (rp.p + 15) & ~15);
+          if (!(ok = mbar_wait(acc_empty, (n & 1u) ^ 1u, abort_flag))) break;
+          tc_fence_after();
+          int k_chunks = (rp.m + kBK - 1) / kBK;
+          for (int kc = 0; kc < k_chunks; ++kc, ++it) {
+            int s = it % kPowStages;
+            if (!(ok = mbar_wait(&full[s], (it / kPowStages) & 1u, abort_flag))) break;
+            tc_fence_after();
+            uint32_t base = smem_u32(smem + s * kPowStageBytes);
+            // T += G_hi Y_hi + G_lo Y_hi + G_hi Y_lo
+#pragma unroll
+            for (int term = 0; term < 3; ++term) {
+              uint64_t adesc = umma_desc(base + (term == 1 ? kPowBytesA : 0));
+              uint64_t bdesc = umma_desc(base + 2 * kPowBytesA + (term == 2 ? kPowBytesB : 0));
+#pragma unroll
+              for (int k = 0; k < kBK / 16; ++k)
+                umma_bf16(tmem_base, adesc + 2 * k, bdesc + 2 * k, idesc, (kc | term | k) != 0);
+            }
+            umma_commit(&empty[s]);
+          }
+          if (!ok) break;
+          umma_commit(acc_full);
+        }
+      }
+    }
+    __syncwarp();
+  } else {
+    // ------------------------------------------------------------ epilogue, warps 0-7
+    const int et = threadIdx.x;                    // 0 .. 255
+    const int r = (warp & 3) * 32 + lane;          // TMEM lane = row of the tile (warps 0-3 solve)
+    const uint32_t t_lane = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
+    auto epi_sync = [&]() { named_barrier(1, kEpiThreads); };
+    // thread 0 waits for a counter; everybody learns the outcome
+    auto team_wait = [&](const unsigned* ctr, unsigned target) -> bool {
+      epi_sync();
+      if (et == 0) *s_word = flag_wait_ge(ctr, target, gabort, abort_flag) ? 1 : 0;
+      epi_sync();
+      return *s_word != 0;
+    };
+    uint32_t n = 0;
+    int cached_b = -1, cached_step = -1;
+    bool ok = true;
+    for (int step = 0; step <= last_step; ++step) {
+      const bool identity = step == 0, is_last = step == last_step;
+      __nv_bfloat16* y_hi = prm.y_hi[(step & 1) ^ 1];
+      __nv_bfloat16* y_lo = prm.y_lo[(step & 1) ^ 1];
+      float* yf = is_last ? prm.yf[1] : (step == last_step - 1 ? prm.yf[0] : nullptr);
+      float* qprev = is_last ? prm.yf[0] : nullptr;
+      for (int si = s_begin; si < s_end; ++si, ++n) {
+        const int item = s_items[si];
+        int b, tile; ReqPlan rp;
+        decode(item, b, rp, tile);
+        const int p = rp.p, P = (p + 7) & ~7;
+        unsigned* sync_b = prm.sync + (size_t)b * kSyncStride;
+        if (!identity && (b != cached_b || step != cached_step)) {
+          // the factor of the previous block, published by whichever tile finished that step last
+          ok = team_wait(sync_b + 1, (unsigned)step) && ok;
+          if (ok) {
+            const float4* src = reinterpret_cast<const float4*>(prm.lbuf + (size_t)b * kLbufStride);
+            float4* dst = reinterpret_cast<float4*>(lt);
+            int n4 = (lt_row_offset(P, P) + 3) / 4;    // floats used by the P-wide layout
+            for (int e = et; e < n4; e += kEpiThreads) dst[e] = __ldcg(src + e);
+            const float* dsrc = prm.lbuf + (size_t)b * kLbufStride + kLtFloats;
+            for (int e = et; e < P; e += kEpiThreads) dinv[e] = __ldcg(dsrc + e);
+          }
+          epi_sync();
+          cached_b = b; cached_step = step;
+        }
+        const int nrows = min(kTile, rp.m - tile * kTile);
+        if (warp < 4) {
+          ok = ok && mbar_wait(acc_full, n & 1u, abort_flag);
+          tc_fence_after();
+          const bool row_ok = r < nrows;
+          // ---- Y_next row = T row * L^-T; staged as xs[c][r] ----
+#pragma unroll 1
+          for (int cb = 0; cb * 32 < P; ++cb) {
+            float v[32];
+            tmem_ld32(t_lane + cb * 32, v);
+#pragma unroll
+            for (int sb = 0; sb < 4; ++sb) {
+              const int jb = cb * 32 + sb * 8;
+              if (jb < P) {
+                float acc[8];
+#pragma unroll
+                for (int e = 0; e < 8; ++e) acc[e] = v[sb * 8 + e];
+                if (!identity) solve_block8(acc, jb, smem_u32(lt), smem_u32(dinv), smem_u32(xs), r, P);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) xs[(jb + e) * kXsLd + r] = (row_ok && ok) ? acc[e] : 0.f;
+              }
+            }
+          }
+          tc_fence_before();
+          mbar_arrive(acc_empty);
+        } else if (is_last) {
+          // ---- last step, warps 4-7: rows of Q = Y L^-T for the previous block Y, in place ----
+          ok = ok && mbar_wait(acc_full, n & 1u, abort_flag);      // the ring is no longer read
+          const int t4 = et - 128;
+          float* qrows = qprev + ((size_t)rp.presel_off + tile * kTile) * kPMax;
+          for (int c = t4; c < P; c += 128) {
+#pragma unroll 1
+            for (int r0 = 0; r0 < kTile; r0 += 8) {
+              float v[8];
+#pragma unroll
+              for (int u = 0; u < 8; ++u)
+                v[u] = (r0 + u < nrows && c < p) ? __ldcg(qrows + (size_t)(r0 + u) * kPMax + c) : 0.f;
+#pragma unroll
+              for (int u = 0; u < 8; ++u) xq[c * kXsLd + r0 + u] = v[u];
+            }
+          }
+          named_barrier(2, 128);
+          for (int jb = 0; jb < P; jb += 8) {
+            float acc[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) acc[e] = xq[(jb + e) * kXsLd + t4];
+            solve_block8(acc, jb, smem_u32(lt), smem_u32(dinv), smem_u32(xq), t4, P);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) xq[(jb + e) * kXsLd + t4] = acc[e];
+          }
+          named_barrier(2, 128);
+          for (int c = t4; c < p; c += 128)
+            for (int rr = 0; rr < nrows; ++rr) qrows[(size_t)rr * kPMax + c] = xq[c * kXsLd + rr];
+        }
+        epi_sync();                                  // the staged block is complete
+        if (is_last && et < nrows) {
+          // first half of Eq. 15 while both blocks are on chip: sum_j Y'_ij Q_ij, parked in the
+          // energy array until the Ritz vectors of the request are known
+          float total = 0.f;
+          for (int c = 0; c < p; ++c) total += xs[c * kXsLd + et] * xq[c * kXsLd + et];
+          prm.energy[(size_t)rp.presel_off + tile * kTile + et] = total;
+        }
+        // ---- bf16 planes of the new block (K-major operand of the next step): 8 positions per thread
+        if (!is_last) {
+          const int cols = (rp.m + kBK - 1) / kBK * kBK;
+          for (int wi = et; wi < p * 16; wi += kEpiThreads) {
+            int c = wi >> 4, ch = wi & 15;
+            int pos = tile * kTile + ch * 8;
+            if (pos >= cols) continue;
+            const float4* xp = reinterpret_cast<const float4*>(xs + c * kXsLd + ch * 8);
+            float4 a = xp[0], d = xp[1];
+            float f[8] = {a.x, a.y, a.z, a.w, d.x, d.y, d.z, d.w};
+            uint32_t ph[4], pl[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              __nv_bfloat162 hi = __floats2bfloat162_rn(f[2 * e], f[2 * e + 1]);
+              ph[e] = *reinterpret_cast<uint32_t*>(&hi);
+              pl[e] = pack_bf16(f[2 * e] - __low2float(hi), f[2 * e + 1] - __high2float(hi));
+            }
+            size_t o = ((size_t)b * kPMax + c) * prm.ld + pos;
+            *reinterpret_cast<uint4*>(y_hi + o) = make_uint4(ph[0], ph[1], ph[2], ph[3]);
+            *reinterpret_cast<uint4*>(y_lo + o) = make_uint4(pl[0], pl[1], pl[2], pl[3]);
+          }
+        }
+        if (yf != nullptr) {
+          // float32 block, one token per row; consecutive threads write consecutive columns
+          float* yrows = yf + ((size_t)rp.presel_off + tile * kTile) * kPMax;
+          for (int c = et & 127; c < p; c += 128)
+            for (int rr = et >> 7; rr < nrows; rr += 2) yrows[(size_t)rr * kPMax + c] = xs[c * kXsLd + rr];
+        }
+        // ---- float64 partial Gram of the tile on the FP64 tensor cores ----
+        const int coff = is_last ? ((p - rp.win) & ~7) : 0;
+        {
+          // The last step only feeds the Rayleigh-Ritz window: the trailing block of columns from
+          // coff on, plus the diagonal of the leading columns (the scale of the problem).
+          const int pw = p - coff;
+          const int nb8 = (pw + 7) >> 3, units = (nb8 + 1) / 2, nslab = (nrows + kSlabRows - 1) / kSlabRows;
+          double* slabs = reinterpret_cast<double*>(smem + kXsBytes);
+          double* out = prm.partial + (size_t)item * kTileDoubles;
+          for (int c = et; c < coff; c += kEpiThreads) {
+            double sq = 0.0;
+            for (int rr = 0; rr < nrows; ++rr) { double x = (double)xs[c * kXsLd + rr]; sq += x * x; }
+            out[tile_offset(c, c)] = sq;
+          }
+          // Units 0-7 go to the eight warps.  With more than 128 columns one or two units are left
+          // over: a second, short pass over the slabs deals their 8 x 8 tiles round-robin to the
+          // warps (at most kExtraTiles each) instead of leaving them to one or two warps.
+          const int fr = lane >> 2, fk = lane & 3;
+          auto fill_slab = [&](double* slab, int sl) {
+            for (int e = et; e < nb8 * 8 * kSlabRows; e += kEpiThreads) {
+              int c = e >> 4, rr = e & 15;
+              slab[c * kSlabLd + rr] = (double)xs[(coff + c) * kXsLd + sl * kSlabRows + rr];
+            }
+          };
+          {
+            const bool have = warp < units;
+            const int ta = have ? warp : 0, tz = have ? nb8 - 1 - warp : 0;
+            GramAcc acc;
+#pragma unroll
+            for (int u = 0; u <= kMaxTiles8; ++u) { acc.a[u][0] = 0.0; acc.a[u][1] = 0.0; }
+            for (int sl = 0; sl < nslab; ++sl) {
+              double* slab = slabs + (sl & 1) * (kPMax * kSlabLd);
+              fill_slab(slab, sl);
+              epi_sync();
+              if (have) gram_unit_accumulate(acc, slab, ta, tz, lane);
+              // the other buffer is refilled next; this one is reused two slabs later, after the
+              // barrier of the next slab
+            }
+            if (have) gram_unit_store_tiles(acc, ta, tz, coff >> 3, lane, out);
+            epi_sync();
+          }
+          if (units > 8) {
+            int xa_t[kExtraTiles], xb_t[kExtraTiles];
+            double xacc[kExtraTiles][2];
+            int n_extra = 0;
+#pragma unroll
+            for (int q = 0; q < kExtraTiles; ++q) {
+              xacc[q][0] = 0.0; xacc[q][1] = 0.0; xa_t[q] = 0; xb_t[q] = 0;
+              if (extra_tile(warp + 8 * q, nb8, units, xa_t[q], xb_t[q])) n_extra = q + 1;
+            }
+            for (int sl = 0; sl < nslab; ++sl) {
+              double* slab = slabs + (sl & 1) * (kPMax * kSlabLd);
+              fill_slab(slab, sl);
+              epi_sync();
+              const double* base = slab + fr * kSlabLd + fk;
+#pragma unroll 1
+              for (int ks = 0; ks < kSlabRows / 4; ++ks) {
+#pragma unroll
+                for (int q = 0; q < kExtraTiles; ++q)
+                  if (q < n_extra)
+                    dmma_8x8x4(xacc[q][0], xacc[q][1], base[xa_t[q] * 8 * kSlabLd + 4 * ks],
+                               base[xb_t[q] * 8 * kSlabLd + 4 * ks]);
+              }
+            }
+#pragma unroll
+            for (int q = 0; q < kExtraTiles; ++q) {
+              if (q < n_extra)
+                *reinterpret_cast<double2*>(out + tri_index((coff >> 3) + xa_t[q], (coff >> 3) + xb_t[q]) * 64 +
+                                            fr * 8 + 2 * fk) = make_double2(xacc[q][0], xacc[q][1]);
+            }
+            epi_sync();
+          }
+        }
+        // ---- arrival: this tile's slab and partial sums are published -------------------------
+        __threadfence();
+        fence_proxy_async_all();
+        epi_sync();
+        const unsigned nt = (unsigned)((rp.m + kTile - 1) / kTile);
+        if (et == 0) {
+          unsigned old = atomicAdd(sync_b, 1u);
+          // one decision for the whole team (a CTA that has given up factors nothing)
+          *s_word = (old + 1u == nt * (unsigned)(step + 1) && !*abort_flag) ? 1 : 0;
+        }
+        epi_sync();
+        if (*s_word) {
+          // ---- the last tile of the request to finish this step factors the summed Gram matrix ----
+          __threadfence();
+          const double* pbase = prm.partial + (size_t)rp.ptile_off * kTileDoubles;
+          double* Tm = reinterpret_cast<double*>(smem);        // the region is free: every thread passed the barrier
+          if (!is_last) {
+            team_cholesky(pbase, (int)nt, p, prm.lbuf + (size_t)b * kLbufStride, Tm);
+            __threadfence();
+            epi_sync();
+            if (et == 0) st_release_u32(sync_b + 1, (unsigned)(step + 1));
+          } else {
+            team_ritz(pbase, (int)nt, p, rp.win, rp.r, rp.m, prm.ub + (size_t)b * kPMax * kPMax, reinterpret_cast<float*>(smem), lt,
+                      s_scale, s_flag, prm.max_sweeps, prm.conv_tol, prm.steps, prm.status);
+            __threadfence();
+            epi_sync();
+            if (et == 0) st_release_u32(sync_b + 2, 1u);
+          }
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        mbar_arrive(epi_done);
+      }
+    }
+    // ------------------------------------------------------------ Eq. 15 for this CTA's tiles
+    // c_i = sum_j Y'_ij Q_ij - sum_k (Y'_{i,win} u_k)(Q_{i,win} u_k)  (see eig_kernels.cuh)
+    {
+      float* us = reinterpret_cast<float*>(smem);                      // [w][nbot]
+      int cached_u = -1;
+      for (int si = s_begin; si < s_end; ++si) {
+        const int item = s_items[si];
+        int b, tile; ReqPlan rp;
+        decode(item, b, rp, tile);
+        const int p = rp.p, w = rp.win, w0 = p - w, nbot = p - rp.r;
+        if (b != cached_u) {
+          ok = team_wait(prm.sync + (size_t)b * kSyncStride + 2, 1u) && ok;
+          const float* usrc = prm.ub + (size_t)b * kPMax * kPMax;
+          if (ok) for (int e = et; e < w * nbot; e += kEpiThreads) us[e] = __ldcg(usrc + e);
+          epi_sync();
+          cached_u = b;
+        }
+        const int nrows = min(kTile, rp.m - tile * kTile);
+        // the discarded Ritz pairs take only the window columns of the two blocks: one thread per
+        // row, window slices read straight from the float32 blocks
+        for (int rr = et; rr < nrows; rr += kEpiThreads) {
+          const size_t grow = (size_t)rp.presel_off + tile * kTile + rr;
+          const float* yrow = prm.yf[1] + grow * kPMax + w0;
+          const float* qrow = prm.yf[0] + grow * kPMax + w0;
+          // projections of the two window slices on every discarded Ritz vector, accumulated over
+          // chunks of 32 window columns (all loads of a chunk in flight together)
+          float sub_ = 0.f;
+          for (int k0 = 0; k0 < nbot; k0 += 8) {
+            float ya[8], qa[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) { ya[u] = 0.f; qa[u] = 0.f; }
+            for (int j0 = 0; j0 < w; j0 += 32) {
+              float yv[32], qv[32];
+#pragma unroll
+              for (int jj = 0; jj < 32; ++jj) {
+                const bool in = ok && j0 + jj < w;
+                yv[jj] = in ? __ldcg(yrow + j0 + jj) : 0.f;
+                qv[jj] = in ? __ldcg(qrow + j0 + jj) : 0.f;
+              }
+#pragma unroll
+              for (int jj = 0; jj < 32; ++jj) {
+                if (j0 + jj < w) {
+                  const float* ur = us + (j0 + jj) * nbot + k0;
+#pragma unroll
+                  for (int u = 0; u < 8; ++u) {
+                    const float uu = k0 + u < nbot ? ur[u] : 0.f;
+                    ya[u] += yv[jj] * uu; qa[u] += qv[jj] * uu;
+                  }
+                }
+              }
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u) sub_ += ya[u] * qa[u];
+          }
+          const float total = ok ? __ldcg(prm.energy + grow) : 0.f;
+          prm.energy[grow] = fmaxf(total - sub_, 0.f);
+        }
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 9) tmem_dealloc(tmem_base, kPowTmemCols);
+  if (threadIdx.x == 0 && *abort_flag) atomicOr(prm.status, kStatusTimeout);
+}
+
+}  // namespace sub
+}  // namespace covspec
