@@ -96,35 +96,40 @@ __device__ __forceinline__ double gram_entry_cg(int ntile, const double* src) {
   return s;
 }
 // T[0 .. count) = sum over the request's tiles (tile order: deterministic) of their partial
-// matrices; count a multiple of 64.  Coalesced 16-byte loads, 16 of them in flight per thread.
+// matrices; count a multiple of 64.  Coalesced 16-byte loads, 32 of them in flight per thread.
 __device__ __forceinline__ void team_sum_partials(double* T, const double* pbase, int ntile, int count,
                                                   int tid, int nthreads) {
   const int pairs = count >> 1;
-  for (int e0 = tid; e0 < pairs; e0 += 2 * nthreads) {
-    const int e1 = e0 + nthreads;
-    const bool have1 = e1 < pairs;
-    double2 s0 = make_double2(0.0, 0.0), s1 = s0;
+  for (int e0 = tid; e0 < pairs; e0 += 4 * nthreads) {
+    int e[4];
+    double2 s[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      e[u] = e0 + u * nthreads < pairs ? e0 + u * nthreads : e0;
+      s[u] = make_double2(0.0, 0.0);
+    }
     for (int t0 = 0; t0 < ntile; t0 += 8) {
-      double2 v0[8], v1[8];
+      double2 v[4][8];
 #pragma unroll
       for (int q = 0; q < 8; ++q) {
         const double2* src = reinterpret_cast<const double2*>(pbase + (size_t)min(t0 + q, ntile - 1) * kTileDoubles);
-        v0[q] = __ldcg(src + e0);
-        v1[q] = __ldcg(src + (have1 ? e1 : e0));
+#pragma unroll
+        for (int u = 0; u < 4; ++u) v[u][q] = __ldcg(src + e[u]);
       }
 #pragma unroll
       for (int q = 0; q < 8; ++q) {
-        if (t0 + q < ntile) { s0.x += v0[q].x; s0.y += v0[q].y; s1.x += v1[q].x; s1.y += v1[q].y; }
+        if (t0 + q < ntile) {
+#pragma unroll
+          for (int u = 0; u < 4; ++u) { s[u].x += v[u][q].x; s[u].y += v[u][q].y; }
+        }
       }
     }
-    reinterpret_cast<double2*>(T)[e0] = s0;
-    if (have1) reinterpret_cast<double2*>(T)[e1] = s1;
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+      if (e0 + u * nthreads < pairs) reinterpret_cast<double2*>(T)[e0 + u * nthreads] = s[u];
   }
 }
 
-// ---- float64 Cholesky factorisation by the eight epilogue warps --------------------------------
-// Same blocked right-looking scheme as cholesky_blocked, for `nthreads` threads (whole warps, thread
-// index tid) that synchronise through `sync()`.
 // 1 / sqrt(x) for x > 0 without a range test on the pivot chain: x = m 4^k with m in [1, 4) (integer
 // operations on the exponent field), float32 estimate of 1 / sqrt(m) refined in float32 and by one
 // Newton step in float64, then scaled by 2^-k.  Subnormal or non-finite x give a meaningless value;
@@ -143,9 +148,12 @@ __device__ __forceinline__ double rsqrt_f64_scaled(double x) {
 }
 
 // Diagonal 8 x 8 tile, factored by one thread in registers: measured faster than a lane-per-row
-// version (64-bit shuffles cost more than the arithmetic they save).  The chain of eight dependent
-// reciprocal square roots is the critical path of the whole factorisation, which is why the caller
-// keeps the other warps of this thread's scheduler off the FP64 pipe meanwhile.
+// version (64-bit shuffles cost more than the arithmetic they save).  Two columns at a time: for the
+// leading 2 x 2 block [[al, be], [be, ga]] the factor is l11 = sqrt(al), l21 = be / l11,
+// l22 = sqrt(de / al) with de = al ga - be^2, so the two reciprocal square roots (of al and de) run
+// side by side instead of one after the other.  The chain of dependent pivots is the critical path
+// of the whole factorisation.  A pivot below 1e-12 of its original diagonal entry (a numerically
+// dependent direction) is clamped there; the next multiplication by G restores the direction.
 __device__ __forceinline__ void factor_diag_thread(double* D, const double* d0, double* rd) {
   double a[8][8];
 #pragma unroll
@@ -153,19 +161,28 @@ __device__ __forceinline__ void factor_diag_thread(double* D, const double* d0, 
 #pragma unroll
     for (int m = 0; m <= l; ++m) a[l][m] = D[l * 8 + m];
 #pragma unroll
-  for (int c = 0; c < 8; ++c) {
-    double piv = a[c][c];
-    const double floor_ = 1e-12 * d0[c];
-    if (!(piv > floor_)) piv = floor_ > 0.0 ? floor_ : 1.0;
-    const double rs = rsqrt_f64_scaled(piv);
-    a[c][c] = piv * rs;
-    rd[c] = rs;
+  for (int c = 0; c < 8; c += 2) {
+    const double f0 = 1e-12 * d0[c], f1 = 1e-12 * d0[c + 1];
+    double al = a[c][c];
+    if (!(al > f0)) al = f0 > 0.0 ? f0 : 1.0;
+    const double be = a[c + 1][c], ga = a[c + 1][c + 1];
+    double de = fma(al, ga, -be * be);                  // al * (second pivot)
+    const double fd = f1 * al;
+    if (!(de > fd)) de = fd > 0.0 ? fd : al;
+    const double ra = rsqrt_f64_scaled(al), rq = rsqrt_f64_scaled(de);
+    const double l11 = al * ra, l21 = be * ra, inv22 = rq * l11, l22 = de * rq * ra;
+    a[c][c] = l11; a[c + 1][c] = l21; a[c + 1][c + 1] = l22;
+    rd[c] = ra; rd[c + 1] = inv22;
 #pragma unroll
-    for (int l = c + 1; l < 8; ++l) a[l][c] *= rs;
+    for (int l = c + 2; l < 8; ++l) {
+      const double x1 = a[l][c] * ra;
+      a[l][c + 1] = (a[l][c + 1] - x1 * l21) * inv22;
+      a[l][c] = x1;
+    }
 #pragma unroll
-    for (int l = c + 1; l < 8; ++l)
+    for (int l = c + 2; l < 8; ++l)
 #pragma unroll
-      for (int m = c + 1; m <= l; ++m) a[l][m] -= a[l][c] * a[m][c];
+      for (int m = c + 2; m <= l; ++m) a[l][m] -= a[l][c] * a[m][c] + a[l][c + 1] * a[m][c + 1];
   }
 #pragma unroll
   for (int l = 0; l < 8; ++l)
@@ -202,42 +219,76 @@ __device__ __forceinline__ void cholesky_blocked_team(int n, double* T, double* 
     dmma_8x8x4(c0, c1, -XI[4], XK[4]);
     C[0] = c0; C[1] = c1;
   };
+  // row `i` of the tile (I, J) <- row * L_JJ^-T (forward substitution over the 8 columns)
+  auto solve_row = [&](int J, int i) {
+    const double* D = T + tri_index(J, J) * 64;
+    double* row = T + tri_index(i >> 3, J) * 64 + (i & 7) * 8;
+    double x[8];
+#pragma unroll
+    for (int c = 0; c < 8; ++c) x[c] = row[c];
+#pragma unroll
+    for (int c = 0; c < 8; ++c) {
+      double v = x[c];
+#pragma unroll
+      for (int k = 0; k < c; ++k) v -= x[k] * D[c * 8 + k];
+      x[c] = v * rd[8 * J + c];
+    }
+#pragma unroll
+    for (int c = 0; c < 8; ++c) row[c] = x[c];
+  };
+  auto update_tile2 = [&](int J, int Ia, int Ka, int Ib, int Kb) {
+    const double* XIa = T + tri_index(Ia, J) * 64 + fr * 8 + fk;
+    const double* XKa = T + tri_index(Ka, J) * 64 + fr * 8 + fk;
+    const double* XIb = T + tri_index(Ib, J) * 64 + fr * 8 + fk;
+    const double* XKb = T + tri_index(Kb, J) * 64 + fr * 8 + fk;
+    double* Ca = T + tri_index(Ia, Ka) * 64 + fr * 8 + 2 * fk;
+    double* Cb = T + tri_index(Ib, Kb) * 64 + fr * 8 + 2 * fk;
+    double a0 = Ca[0], a1 = Ca[1], b0 = Cb[0], b1 = Cb[1];
+    const double xa0 = -XIa[0], xa4 = -XIa[4], xb0 = -XIb[0], xb4 = -XIb[4];
+    const double ka0 = XKa[0], ka4 = XKa[4], kb0 = XKb[0], kb4 = XKb[4];
+    dmma_8x8x4(a0, a1, xa0, ka0);
+    dmma_8x8x4(b0, b1, xb0, kb0);
+    dmma_8x8x4(a0, a1, xa4, ka4);
+    dmma_8x8x4(b0, b1, xb4, kb4);
+    Ca[0] = a0; Ca[1] = a1; Cb[0] = b0; Cb[1] = b1;
+  };
   if (tid == 0) factor_diag_thread(T, d0, rd);
   sync();
-  for (int J = 0; J < nb; ++J) {
-    const double* D = T + tri_index(J, J) * 64;
-    for (int i = 8 * (J + 1) + tid; i < 8 * nb; i += nthreads) {
-      double* row = T + tri_index(i >> 3, J) * 64 + (i & 7) * 8;
-      double x[8];
-#pragma unroll
-      for (int c = 0; c < 8; ++c) x[c] = row[c];
-#pragma unroll
-      for (int c = 0; c < 8; ++c) {
-        double v = x[c];
-#pragma unroll
-        for (int k = 0; k < c; ++k) v -= x[k] * D[c * 8 + k];
-        x[c] = v * rd[8 * J + c];
-      }
-#pragma unroll
-      for (int c = 0; c < 8; ++c) row[c] = x[c];
-    }
-    sync();
-    if (J + 1 == nb) break;
-    for (int I = J + 1 + warp; I < nb; I += nw) update_tile(J, I, J + 1);
-    sync();
-    // The next diagonal tile is factored by one thread while the trailing matrix is updated by the
-    // warps of the other three schedulers (warp w issues on scheduler w & 3; the FP64 pipe is per
-    // scheduler, and the pivot chain must not queue behind the updates).
-    if ((warp & 3) == 0) {
-      if (tid == 0) factor_diag_thread(T + tri_index(J + 1, J + 1) * 64, d0 + 8 * (J + 1), rd + 8 * (J + 1));
+  // One barrier of the whole team per 8-column panel.  The chain that bounds the factorisation -
+  // panel J's diagonal tile -> tile (J+1, J) -> its update of tile (J+1, J+1) -> that tile's eight
+  // dependent pivots - runs on warp 0 alone; the warps of the other three schedulers (the FP64 pipe
+  // is per scheduler: warp w issues on scheduler w & 3, so warp 4 stays idle) solve the rest of the
+  // panel and update the rest of the trailing matrix meanwhile.  They need tile (J+1, J) for the
+  // tiles of column J+1: warp 0 arrives on barrier 4 once it is solved.
+  const bool bulk = (warp & 3) != 0;
+  const int nbulk = nw - (nw + 3) / 4, me = warp - (warp >> 2) - 1;          // bulk warps, in order
+  const int bulk_threads = nbulk * 32, btid = me * 32 + lane;
+  for (int J = 0; J + 1 < nb; ++J) {
+    if (warp == 0) {
+      if (lane < 8) solve_row(J, 8 * (J + 1) + lane);
       __syncwarp();
-    } else {
-      const int mrem = nb - J - 2, ntr = mrem * (mrem + 1) / 2;
-      const int nworkers = nw - (nw + 3) / 4, me = warp - (warp >> 2) - 1;   // warps with (w & 3) != 0, in order
-      for (int q = me; q < ntr; q += nworkers) {
-        int ii, kk;
-        tri_decode(q, ii, kk);
-        update_tile(J, J + 2 + ii, J + 2 + kk);
+      asm volatile("bar.arrive 4, %0;" ::"r"(bulk_threads + 32) : "memory");
+      update_tile(J, J + 1, J + 1);
+      __syncwarp();
+      if (lane == 0) factor_diag_thread(T + tri_index(J + 1, J + 1) * 64, d0 + 8 * (J + 1), rd + 8 * (J + 1));
+      __syncwarp();
+    } else if (bulk) {
+      for (int i = 8 * (J + 2) + btid; i < 8 * nb; i += bulk_threads) solve_row(J, i);
+      asm volatile("bar.sync 4, %0;" ::"r"(bulk_threads + 32) : "memory");
+      // tiles (I, K), J+1 <= K <= I, I >= J+2, dealt one by one to the bulk warps (row-major
+      // order); two tiles at a time so that their tensor-core instructions overlap
+      int I = J + 2, K = J + 1 + me;
+      auto settle = [&]() { while (I < nb && K > I) { K -= I - J; ++I; } };
+      settle();
+      while (I < nb) {
+        const int I1 = I, K1 = K;
+        K += nbulk; settle();
+        if (I < nb) {
+          update_tile2(J, I1, K1, I, K);
+          K += nbulk; settle();
+        } else {
+          update_tile(J, I1, K1);
+        }
       }
     }
     sync();
@@ -589,28 +640,65 @@ subspace_kernel(const __grid_constant__ CUtensorMap map_gh, const __grid_constan
           cached_b = b; cached_step = step;
         }
         const int nrows = min(kTile, rp.m - tile * kTile);
+        // ---- Y_next row = T row * L^-T (forward substitution per row), staged as xs[c][r] ----
+        // Between the first and the last step two threads share a row: warps 0-3 own the 32-column
+        // super-block S being solved (contributions of the previous super-block and of its own
+        // columns), warps 4-7 run one super-block ahead and sum what the columns before that
+        // contribute to super-block S + 1 (hs, double-buffered behind the staged block).
+        const bool split = !identity && !is_last;
+        const int nS = (P + 31) >> 5;
+        float* hs = reinterpret_cast<float*>(smem + kXsBytes);          // [2][32][kXsLd]
         if (warp < 4) {
           ok = ok && mbar_wait(acc_full, n & 1u, abort_flag);
           tc_fence_after();
-          const bool row_ok = r < nrows;
-          // ---- Y_next row = T row * L^-T; staged as xs[c][r] ----
+        }
+        const bool row_ok = r < nrows;
 #pragma unroll 1
-          for (int cb = 0; cb * 32 < P; ++cb) {
+        for (int S = 0; S < nS; ++S) {
+          if (warp < 4) {
             float v[32];
-            tmem_ld32(t_lane + cb * 32, v);
+            tmem_ld32(t_lane + S * 32, v);
+            const float* hcur = hs + (S & 1) * 32 * kXsLd;
 #pragma unroll
             for (int sb = 0; sb < 4; ++sb) {
-              const int jb = cb * 32 + sb * 8;
+              const int jb = S * 32 + sb * 8;
               if (jb < P) {
                 float acc[8];
 #pragma unroll
                 for (int e = 0; e < 8; ++e) acc[e] = v[sb * 8 + e];
-                if (!identity) solve_block8(acc, jb, smem_u32(lt), smem_u32(dinv), smem_u32(xs), r, P);
+                if (!identity) {
+                  int g0 = 0;
+                  if (split && S >= 2) {
+                    g0 = 8 * (S - 1);
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) acc[e] += hcur[(sb * 8 + e) * kXsLd + r];
+                  }
+                  solve_apply_groups(acc, jb, g0, jb >> 2, smem_u32(lt), smem_u32(xs), r, P);
+                  solve_inblock8(acc, jb, smem_u32(lt), smem_u32(dinv), P);
+                }
 #pragma unroll
                 for (int e = 0; e < 8; ++e) xs[(jb + e) * kXsLd + r] = (row_ok && ok) ? acc[e] : 0.f;
               }
             }
+          } else if (split && S >= 1 && S + 1 < nS) {
+            // minus the contributions of the columns before 32 S to super-block S + 1
+            float* hnext = hs + ((S + 1) & 1) * 32 * kXsLd;
+#pragma unroll 1
+            for (int sb = 0; sb < 4; ++sb) {
+              const int jb = (S + 1) * 32 + sb * 8;
+              if (jb < P) {
+                float acc[8];
+#pragma unroll
+                for (int e = 0; e < 8; ++e) acc[e] = 0.f;
+                solve_apply_groups(acc, jb, 0, 8 * S, smem_u32(lt), smem_u32(xs), r, P);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) hnext[(sb * 8 + e) * kXsLd + r] = acc[e];
+              }
+            }
           }
+          if (split) epi_sync();
+        }
+        if (warp < 4) {
           tc_fence_before();
           mbar_arrive(acc_empty);
         } else if (is_last) {
@@ -634,7 +722,8 @@ subspace_kernel(const __grid_constant__ CUtensorMap map_gh, const __grid_constan
             float acc[8];
 #pragma unroll
             for (int e = 0; e < 8; ++e) acc[e] = xq[(jb + e) * kXsLd + t4];
-            solve_block8(acc, jb, smem_u32(lt), smem_u32(dinv), smem_u32(xq), t4, P);
+            solve_apply_groups(acc, jb, 0, jb >> 2, smem_u32(lt), smem_u32(xq), t4, P);
+            solve_inblock8(acc, jb, smem_u32(lt), smem_u32(dinv), P);
 #pragma unroll
             for (int e = 0; e < 8; ++e) xq[(jb + e) * kXsLd + t4] = acc[e];
           }

@@ -1,6 +1,7 @@
-// Tensor-core kernels of the low-rank redundancy step (Eq. 13-15): the Gram matrix of the stacked
-// preselected tokens and the block power step of the subspace iteration that reaches its top-r
-// eigenspace.
+// Tensor-core pieces of the low-rank redundancy step (Eq. 13-15): the Gram kernel of the stacked
+// preselected tokens, and the shared-memory plan, triangular solve and float64 partial-Gram
+// routines of the block power step (the step itself is part of the fused kernel in
+// subspace_fused.cuh) with which the subspace iteration reaches the top-r eigenspace.
 //
 // G = Z_M^T Z_M (Eq. 13-14; its eigenpairs are sigma_k^2 and the right singular vectors of Z_M) is
 // produced by tcgen05.mma kind::f16 from the gathered bf16 rows, accumulated in float32 in TMEM and
@@ -16,7 +17,7 @@
 //   G planes   [sum M_b (+pad), ld]  row presel_off(b) + i, column j          (ld = max M rounded to 64)
 //   Y planes   [batch * 160, ld]     row b*160 + basis vector, column = token position (K-major B operand)
 //   Yf         [sum M_b, 160]        float32 copy of the last block, one token per row
-//   partial    [tiles, 12880]        packed lower triangles (a*(a+1)/2 + b) in float64
+//   partial    [tiles, 13440]        8 x 8 tiles of the lower triangle in float64 (subspace_fused.cuh)
 // Columns of G and Y between M_b and the next multiple of 64 are kept finite / zero respectively so
 // that whole 64-wide k-chunks can be multiplied.
 #pragma once
@@ -274,7 +275,7 @@ basis_init_kernel(const ReqPlan* __restrict__ plan, __nv_bfloat16* __restrict__ 
 }
 
 // ================================================================================================
-// Power step
+// Power step: shared-memory plan and epilogue routines
 // ================================================================================================
 constexpr int kPowStages = 2;
 constexpr int kPowBytesA = kTile * kBK * 2;              // one plane of the G tile, 16 KB
@@ -289,24 +290,6 @@ constexpr int kPowSmem = kPowRegion + kLbufStride * 4 + 1024 + 1024;
 constexpr int kPowTmemCols = 256;
 constexpr int kPowThreads = 320;                         // 8 epilogue warps, TMA producer, MMA issuer
 static_assert(kPMax * kXsLd * 4 <= kPowStages * kPowStageBytes, "staged block must fit in the ring");
-
-struct PowerParams {
-  const ReqPlan* plan;
-  int batch;
-  int n_items;              // 128-row tiles over all stage-2 requests
-  const int* sched;         // [gridDim.x + 1] offsets, then the item lists of every CTA (longest
-                            // items first, balanced on the host)
-  int identity;             // first step: no triangular factor yet
-  const float* lbuf;        // [batch][kLbufStride] triangular factor + reciprocal diagonal
-  __nv_bfloat16* y_hi;      // output planes
-  __nv_bfloat16* y_lo;
-  int ld;
-  float* yf;                // [sum M_b, kPMax] float32 copy of the new block, or nullptr
-  float* qprev;             // last step: float32 copy of the previous block Y on entry, overwritten
-                            // with the orthonormal basis Q = Y L^-T it stands for; else nullptr
-  double* partial;          // [tiles][kTriMax]
-  int* status;
-};
 
 __device__ __forceinline__ float lds_f32(uint32_t addr) {
   float v;
@@ -343,30 +326,30 @@ __device__ __forceinline__ void solve_group_apply(const SolveGroup& g, float (&a
   }
 }
 
-// Columns jb .. jb+7 of one row of X = T L^-T (blocked forward substitution).  acc holds
-// t[jb..jb+7] on entry and x[jb..jb+7] on return; the x_i already solved are read from the staged
-// block xs[i * kXsLd + r].  lt / dinv: the factor in the layout of lt_row_offset for width P and
-// its reciprocal diagonal.  All three are shared-memory addresses (32-bit window offsets); the
-// loads of one group of four rows are in flight while the previous group is applied.
-__device__ __forceinline__ void solve_block8(float (&acc)[8], int jb, uint32_t lt, uint32_t dinv,
-                                             uint32_t xs, int r, int P) {
-  const int groups = jb >> 2;                      // even: jb is a multiple of 8
-  if (groups > 0) {
-    uint32_t xr = xs + r * 4;
-    uint32_t at = lt + jb * 4;                     // lt_row_offset(i, P) + jb - 4 * (i >> 2) at i = 0
-    int stride = P;                                // rows 4a .. 4a+3 have P - 4a entries
-    SolveGroup ga, gb;
-    solve_group_load(ga, xr, at, stride);
-    for (int g = 0; g < groups; g += 2) {
-      xr += 4 * kXsLd * 4; at += (4 * stride - 4) * 4; stride -= 4;
-      solve_group_load(gb, xr, at, stride);
-      solve_group_apply(ga, acc);
-      xr += 4 * kXsLd * 4; at += (4 * stride - 4) * 4; stride -= 4;
-      if (g + 2 < groups) solve_group_load(ga, xr, at, stride);
-      solve_group_apply(gb, acc);
-    }
+// acc[0..7] -= sum over the groups g0 .. g1-1 (four solved columns i each; g1 - g0 even) of
+// x_i * L[jb + e][i]: the part of the forward substitution for columns jb .. jb+7 that only needs
+// x_i already staged in xs[i * kXsLd + r].  The loads of one group are in flight while the previous
+// group is applied.
+__device__ __forceinline__ void solve_apply_groups(float (&acc)[8], int jb, int g0, int g1, uint32_t lt,
+                                                   uint32_t xs, int r, int P) {
+  if (g1 <= g0) return;
+  uint32_t xr = xs + (r + 4 * g0 * kXsLd) * 4;
+  uint32_t at = lt + (4 * g0 * P - 8 * g0 * (g0 - 1) + jb - 4 * g0) * 4;   // row 4 g0 of the layout, column jb
+  int stride = P - 4 * g0;                         // rows 4a .. 4a+3 have P - 4a entries
+  SolveGroup ga, gb;
+  solve_group_load(ga, xr, at, stride);
+  for (int g = g0; g < g1; g += 2) {
+    xr += 4 * kXsLd * 4; at += (4 * stride - 4) * 4; stride -= 4;
+    solve_group_load(gb, xr, at, stride);
+    solve_group_apply(ga, acc);
+    xr += 4 * kXsLd * 4; at += (4 * stride - 4) * 4; stride -= 4;
+    if (g + 2 < g1) solve_group_load(ga, xr, at, stride);
+    solve_group_apply(gb, acc);
   }
-  // triangular solve inside the block: row jb+jj of the layout starts at column jb + (jj & ~3)
+}
+// Triangular solve inside the block of columns jb .. jb+7: acc holds t - (contributions of the
+// columns before jb) on entry and x[jb..jb+7] on return.
+__device__ __forceinline__ void solve_inblock8(float (&acc)[8], int jb, uint32_t lt, uint32_t dinv, int P) {
 #pragma unroll
   for (int jj = 0; jj < 8; ++jj) {
     float x = acc[jj] * lds_f32(dinv + (jb + jj) * 4);
@@ -433,280 +416,6 @@ __device__ __forceinline__ void gram_unit_accumulate(GramAcc& acc, const double*
 }
 #undef COVSPEC_GRAM_A
 #undef COVSPEC_GRAM_Z
-
-// Writes the accumulated tiles of one warp to the packed lower triangle.
-__device__ __forceinline__ void gram_unit_store(const GramAcc& acc, int ta, int tz, int p, int coff,
-                                                int lane, double* __restrict__ out) {
-  const int fr = lane >> 2, fk = lane & 3;
-#pragma unroll
-  for (int u = 0; u <= kMaxTiles8; ++u) {
-    int strip = -1, tb = 0;
-    if (u < kMaxTiles8 && u <= ta) { strip = ta; tb = u; }
-    else if (u >= 1 && kMaxTiles8 - u <= tz && tz != ta) { strip = tz; tb = kMaxTiles8 - u; }
-    if (strip < 0) continue;
-    int row = 8 * strip + fr, col = 8 * tb + 2 * fk;
-    if (row < p) {
-      if (col <= row) out[tri_index(coff + row, coff + col)] = acc.a[u][0];
-      if (col + 1 <= row) out[tri_index(coff + row, coff + col + 1)] = acc.a[u][1];
-    }
-  }
-}
-
-__global__ void __launch_bounds__(kPowThreads, 1)
-power_tc_kernel(const __grid_constant__ CUtensorMap map_gh, const __grid_constant__ CUtensorMap map_gl,
-                const __grid_constant__ CUtensorMap map_yh, const __grid_constant__ CUtensorMap map_yl,
-                const PowerParams prm) {
-  extern __shared__ uint8_t smem_raw[];
-  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  float* xs = reinterpret_cast<float*>(smem);                       // aliases the ring after the MMAs
-  float* xq = reinterpret_cast<float*>(smem + kXsBytes);            // previous block (last step)
-  float* lt = reinterpret_cast<float*>(smem + kPowRegion);
-  float* dinv = lt + kLtFloats;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(lt + kLbufStride);
-  uint64_t* full = bars;                 // [2]
-  uint64_t* empty = bars + 2;            // [2]
-  uint64_t* acc_full = bars + 4;
-  uint64_t* acc_empty = bars + 5;
-  uint64_t* epi_done = bars + 6;         // the staged block no longer occupies the ring
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 8);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-
-  if (threadIdx.x == 0) {
-    for (int s = 0; s < kPowStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
-    mbar_init(acc_full, 1);
-    mbar_init(acc_empty, 128);
-    mbar_init(epi_done, 256);
-    *abort_flag = 0;
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-  }
-  if (warp == 9) tmem_alloc(tmem_slot, kPowTmemCols);
-  tc_fence_before();
-  __syncthreads();
-  tc_fence_after();
-  const uint32_t tmem_base = *tmem_slot;
-
-  const int s_begin = prm.sched[blockIdx.x], s_end = prm.sched[blockIdx.x + 1];
-  const int* s_items = prm.sched + gridDim.x + 1;
-  auto decode = [&](int item, int& b, ReqPlan& rp, int& tile) {
-    b = find_request(item, prm.batch, [&](int q) { return prm.plan[q].ptile_off; });
-    rp = prm.plan[b];
-    tile = item - rp.ptile_off;
-  };
-
-  if (warp == 8) {
-    if (lane == 0) {
-      uint32_t it = 0, n = 0;
-      bool ok = true;
-      for (int si = s_begin; si < s_end && ok; ++si, ++n) {
-        const int item = s_items[si];
-        int b, tile; ReqPlan rp;
-        decode(item, b, rp, tile);
-        // the previous item's staged block lives in the ring until its epilogue is done
-        if (n > 0 && !(ok = mbar_wait(epi_done, (n - 1) & 1u, abort_flag))) break;
-        int k_chunks = (rp.m + kBK - 1) / kBK;
-        for (int kc = 0; kc < k_chunks; ++kc, ++it) {
-          int s = it % kPowStages;
-          if (!(ok = mbar_wait(&empty[s], ((it / kPowStages) & 1u) ^ 1u, abort_flag))) break;
-          mbar_expect_tx(&full[s], kPowStageBytes);
-          uint32_t dst = smem_u32(smem + s * kPowStageBytes);
-          int grow = rp.presel_off + tile * kTile;
-          tma_load_2d(dst, &map_gh, kc * kBK, grow, &full[s]);
-          tma_load_2d(dst + kPowBytesA, &map_gl, kc * kBK, grow, &full[s]);
-          tma_load_2d(dst + 2 * kPowBytesA, &map_yh, kc * kBK, b * kPMax, &full[s]);
-          tma_load_2d(dst + 2 * kPowBytesA + kPowBytesB, &map_yl, kc * kBK, b * kPMax, &full[s]);
-        }
-      }
-    }
-    __syncwarp();
-  } else if (warp == 9) {
-    if (lane == 0) {
-      uint32_t it = 0, n = 0;
-      bool ok = true;
-      for (int si = s_begin; si < s_end && ok; ++si, ++n) {
-        const int item = s_items[si];
-        int b, tile; ReqPlan rp;
-        decode(item, b, rp, tile);
-        const uint32_t idesc = umma_idesc(kTile, (rp.p + 15) & ~15);
-        if (!(ok = mbar_wait(acc_empty, (n & 1u) ^ 1u, abort_flag))) break;
-        tc_fence_after();
-        int k_chunks = (rp.m + kBK - 1) / kBK;
-        for (int kc = 0; kc < k_chunks; ++kc, ++it) {
-          int s = it % kPowStages;
-          if (!(ok = mbar_wait(&full[s], (it / kPowStages) & 1u, abort_flag))) break;
-          tc_fence_after();
-          uint32_t base = smem_u32(smem + s * kPowStageBytes);
-          // T += G_hi Y_hi + G_lo Y_hi + G_hi Y_lo
-#pragma unroll
-          for (int term = 0; term < 3; ++term) {
-            uint64_t adesc = umma_desc(base + (term == 1 ? kPowBytesA : 0));
-            uint64_t bdesc = umma_desc(base + 2 * kPowBytesA + (term == 2 ? kPowBytesB : 0));
-#pragma unroll
-            for (int k = 0; k < kBK / 16; ++k)
-              umma_bf16(tmem_base, adesc + 2 * k, bdesc + 2 * k, idesc, (kc | term | k) != 0);
-          }
-          umma_commit(&empty[s]);
-        }
-        if (!ok) break;
-        umma_commit(acc_full);
-      }
-    }
-    __syncwarp();
-  } else {
-    // ------------------------------------------------------------ epilogue, warps 0-7
-    const int et = threadIdx.x;                    // 0 .. 255
-    const int r = (warp & 3) * 32 + lane;          // TMEM lane = row of the tile (warps 0-3 solve)
-    const uint32_t t_lane = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
-    uint32_t n = 0;
-    int cached_b = -1;
-    bool ok = true;
-    for (int si = s_begin; si < s_end; ++si, ++n) {
-      const int item = s_items[si];
-      int b, tile; ReqPlan rp;
-      decode(item, b, rp, tile);
-      const int p = rp.p, P = (p + 7) & ~7;
-      if (!prm.identity && b != cached_b) {
-        named_barrier(1, 256);                     // nobody still reads the previous factor
-        const float4* src = reinterpret_cast<const float4*>(prm.lbuf + (size_t)b * kLbufStride);
-        float4* dst = reinterpret_cast<float4*>(lt);
-        int n4 = (lt_row_offset(P, P) + 3) / 4;    // floats used by the P-wide layout
-        for (int e = et; e < n4; e += 256) dst[e] = src[e];
-        const float* dsrc = prm.lbuf + (size_t)b * kLbufStride + kLtFloats;
-        for (int e = et; e < P; e += 256) dinv[e] = dsrc[e];
-        named_barrier(1, 256);
-        cached_b = b;
-      }
-      const int nrows = min(kTile, rp.m - tile * kTile);
-      if (warp < 4) {
-        ok = ok && mbar_wait(acc_full, n & 1u, abort_flag);
-        tc_fence_after();
-        const bool row_ok = r < nrows;
-        // ---- Y_next row = T row * L^-T; staged as xs[c][r] ----
-#pragma unroll 1
-        for (int cb = 0; cb * 32 < P; ++cb) {
-          float v[32];
-          tmem_ld32(t_lane + cb * 32, v);
-#pragma unroll
-          for (int sb = 0; sb < 4; ++sb) {
-            const int jb = cb * 32 + sb * 8;
-            if (jb < P) {
-              float acc[8];
-#pragma unroll
-              for (int e = 0; e < 8; ++e) acc[e] = v[sb * 8 + e];
-              if (!prm.identity) solve_block8(acc, jb, smem_u32(lt), smem_u32(dinv), smem_u32(xs), r, P);
-#pragma unroll
-              for (int e = 0; e < 8; ++e) xs[(jb + e) * kXsLd + r] = (row_ok && ok) ? acc[e] : 0.f;
-            }
-          }
-        }
-        tc_fence_before();
-        mbar_arrive(acc_empty);
-      } else if (prm.qprev != nullptr) {
-        // ---- last step, warps 4-7: rows of Q = Y L^-T for the previous block Y, in place ----
-        ok = ok && mbar_wait(acc_full, n & 1u, abort_flag);      // the ring is no longer read
-        const int t4 = et - 128;
-        float* qrows = prm.qprev + ((size_t)rp.presel_off + tile * kTile) * kPMax;
-        // thread = column (two columns when P > 128), eight rows per trip so that the loads overlap
-        for (int c = t4; c < P; c += 128) {
-#pragma unroll 1
-          for (int r0 = 0; r0 < kTile; r0 += 8) {
-            float v[8];
-#pragma unroll
-            for (int u = 0; u < 8; ++u)
-              v[u] = (r0 + u < nrows && c < p) ? qrows[(size_t)(r0 + u) * kPMax + c] : 0.f;
-#pragma unroll
-            for (int u = 0; u < 8; ++u) xq[c * kXsLd + r0 + u] = v[u];
-          }
-        }
-        named_barrier(2, 128);
-        for (int jb = 0; jb < P; jb += 8) {
-          float acc[8];
-#pragma unroll
-          for (int e = 0; e < 8; ++e) acc[e] = xq[(jb + e) * kXsLd + t4];
-          solve_block8(acc, jb, smem_u32(lt), smem_u32(dinv), smem_u32(xq), t4, P);
-#pragma unroll
-          for (int e = 0; e < 8; ++e) xq[(jb + e) * kXsLd + t4] = acc[e];
-        }
-        named_barrier(2, 128);
-        for (int c = t4; c < p; c += 128)
-          for (int rr = 0; rr < nrows; ++rr) qrows[(size_t)rr * kPMax + c] = xq[c * kXsLd + rr];
-      }
-      named_barrier(1, 256);                       // the staged block is complete
-      // ---- bf16 planes of the new block (K-major operand of the next step): 8 positions per thread
-      if (prm.qprev == nullptr) {
-        const int cols = (rp.m + kBK - 1) / kBK * kBK;
-        for (int wi = et; wi < p * 16; wi += 256) {
-          int c = wi >> 4, ch = wi & 15;
-          int pos = tile * kTile + ch * 8;
-          if (pos >= cols) continue;
-          const float4* xp = reinterpret_cast<const float4*>(xs + c * kXsLd + ch * 8);
-          float4 a = xp[0], d = xp[1];
-          float f[8] = {a.x, a.y, a.z, a.w, d.x, d.y, d.z, d.w};
-          uint32_t ph[4], pl[4];
-#pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            __nv_bfloat162 hi = __floats2bfloat162_rn(f[2 * e], f[2 * e + 1]);
-            ph[e] = *reinterpret_cast<uint32_t*>(&hi);
-            pl[e] = pack_bf16(f[2 * e] - __low2float(hi), f[2 * e + 1] - __high2float(hi));
-          }
-          size_t o = ((size_t)b * kPMax + c) * prm.ld + pos;
-          *reinterpret_cast<uint4*>(prm.y_hi + o) = make_uint4(ph[0], ph[1], ph[2], ph[3]);
-          *reinterpret_cast<uint4*>(prm.y_lo + o) = make_uint4(pl[0], pl[1], pl[2], pl[3]);
-        }
-      }
-      if (prm.yf != nullptr) {
-        // float32 block, one token per row; consecutive threads write consecutive columns
-        float* yrows = prm.yf + ((size_t)rp.presel_off + tile * kTile) * kPMax;
-        for (int c = et & 127; c < p; c += 128)
-          for (int rr = et >> 7; rr < nrows; rr += 2) yrows[(size_t)rr * kPMax + c] = xs[c * kXsLd + rr];
-      }
-      // ---- float64 partial Gram of the tile on the FP64 tensor cores ----
-      {
-        // The last step only feeds the Rayleigh-Ritz window: the trailing block of columns from
-        // coff on, plus the diagonal of the leading columns (the scale of the problem).
-        const int coff = prm.qprev != nullptr ? ((p - rp.win) & ~7) : 0;
-        const int pw = p - coff;
-        const int nb8 = (pw + 7) >> 3, units = (nb8 + 1) / 2, nslab = (nrows + kSlabRows - 1) / kSlabRows;
-        double* slabs = reinterpret_cast<double*>(smem + kXsBytes);
-        double* out = prm.partial + (size_t)item * kTriMax;
-        for (int c = et; c < coff; c += 256) {
-          double sq = 0.0;
-          for (int rr = 0; rr < nrows; ++rr) { double x = (double)xs[c * kXsLd + rr]; sq += x * x; }
-          out[tri_index(c, c)] = sq;
-        }
-        for (int u0 = 0; u0 < units; u0 += 8) {
-          const int unit = u0 + warp;
-          const bool have = unit < units;
-          const int ta = have ? unit : 0, tz = have ? nb8 - 1 - unit : 0;
-          GramAcc acc;
-#pragma unroll
-          for (int u = 0; u <= kMaxTiles8; ++u) { acc.a[u][0] = 0.0; acc.a[u][1] = 0.0; }
-          for (int sl = 0; sl < nslab; ++sl) {
-            double* slab = slabs + (sl & 1) * (kPMax * kSlabLd);
-            // float32 -> float64, rows 16 sl .. 16 sl + 15 of every column (zero beyond the tile)
-            for (int e = et; e < nb8 * 8 * kSlabRows; e += 256) {
-              int c = e >> 4, rr = e & 15;
-              slab[c * kSlabLd + rr] = (double)xs[(coff + c) * kXsLd + sl * kSlabRows + rr];
-            }
-            named_barrier(1, 256);
-            if (have) gram_unit_accumulate(acc, slab, ta, tz, lane);
-            // the other buffer is refilled next; this one is reused two slabs later, after the
-            // barrier of the next slab
-          }
-          if (have) gram_unit_store(acc, ta, tz, pw, coff, lane, out);
-          named_barrier(1, 256);
-        }
-      }
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-      mbar_arrive(epi_done);
-    }
-  }
-
-  tc_fence_before();
-  __syncthreads();
-  if (warp == 9) tmem_dealloc(tmem_base, kPowTmemCols);
-  if (threadIdx.x == 0 && *abort_flag) atomicOr(prm.status, kStatusTimeout);
-}
 
 }  // namespace sub
 }  // namespace covspec
