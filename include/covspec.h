@@ -77,7 +77,9 @@ typedef struct {
   long long max_total_presel;    /* sum of M_b (0: derive from max_total_vis)  */
   int relevance_path;  /* 0: Eq. 10 on the tensor cores (tcgen05) whenever the configuration allows
                           (bf16, 128-wide heads, max over heads, d >= 64), else the CUDA-core path;
-                          1: always the CUDA-core path                                            */
+                          1: always the CUDA-core path; 2: the two-SM form of the tensor-core kernel
+                          (tcgen05.mma.cta_group::2 on pairs of token tiles; measured no faster than
+                          the one-SM form, kept selectable)                                        */
   int lowrank_mode;    /* 0: energy in the top-r singular subspace (Eq. 14-15, the paper's criterion);
                           1: greedy pivoted selection (not in the paper): pick B_vis times the token with
                              the largest residual energy after projecting out the picked ones; needs
@@ -94,6 +96,9 @@ typedef struct {
                           energy) and raises COVSPEC_ERR_NOCONVERGE in the device status word when the
                           estimate exceeds conv_tol (default 2e-3; 0 disables the check).  More steps
                           (eig_iters) or more extra vectors (eig_oversample) settle such inputs      */
+  int eig_early_stop;  /* 1 (default): a request whose estimate, predicted two steps ahead from the Ritz
+                          value estimates of the running iteration, is below conv_tol / 8 stops there
+                          instead of running all eig_iters steps; 0: always eig_iters steps           */
 } covspec_config;
 
 /* One batch of requests (Sec. III-A notation in brackets). */

@@ -44,6 +44,7 @@ class Config(C.Structure):
         ("max_vis_per_req", C.c_int), ("max_presel_per_req", C.c_int),
         ("max_total_presel", C.c_longlong), ("relevance_path", C.c_int), ("lowrank_mode", C.c_int),
         ("ritz_window", C.c_int), ("activity_overlap", C.c_int), ("conv_tol", C.c_float),
+        ("eig_early_stop", C.c_int),
     ]
 
 

@@ -22,6 +22,7 @@ struct ReqPlan {
   int ldm;                 // m rounded up to a multiple of 4 (row stride of the float32 Gram matrix)
   int stage2;              // 1 when b_vis < m (Eq. 13-15 are evaluated)
   int tile_off;            // first 128-token tile of the request in the tensor-core relevance kernel
+  int pair_off;            // first pair of 128-token tiles of the request (two-SM relevance kernel)
   int gram_tile_off;       // first lower-triangle 128 x 128 tile of the request's Gram matrix
   int ptile_off;           // first 128-row tile of the request's subspace-iteration block
   int win;                 // basis vectors in the Rayleigh-Ritz window next to the cut at r

@@ -17,6 +17,7 @@
 #include "gemm_simt.cuh"
 #include "greedy_kernels.cuh"
 #include "relevance_tc.cuh"
+#include "relevance_pair.cuh"
 #include "subspace_tc.cuh"
 #include "subspace_fused.cuh"
 #include "score_kernels.cuh"
@@ -62,6 +63,7 @@ struct Plan {
   int tiles[T_COUNT] = {0};
   int t_max = 0, p_max = 0, m_max = 0, win_max = 0, nbot_max = 0;
   int n_tiles = 0;                            // 128-token tiles over all requests
+  int n_pairs = 0;                            // pairs of neighbouring tiles of one request
   int n_gram_tiles = 0, n_ptiles = 0;         // lower-triangle Gram tiles / 128-row block tiles (stage 2)
   int pow_grid = 0;                           // CTAs of the power step
   std::vector<int> sched;                     // [pow_grid + 1] offsets + item lists (longest first)
@@ -200,7 +202,7 @@ int get_plan(covspec_ctx* ctx, const covspec_problem* p, cudaStream_t stream) {
   pl.req.assign(B, ReqPlan{});
   pl.keep_offsets.assign(B + 1, 0);
   pl.presel_offsets.assign(B + 1, 0);
-  pl.n_stage2 = 0; pl.t_max = 0; pl.p_max = 0; pl.m_max = 0; pl.n_tiles = 0;
+  pl.n_stage2 = 0; pl.t_max = 0; pl.p_max = 0; pl.m_max = 0; pl.n_tiles = 0; pl.n_pairs = 0;
   pl.n_gram_tiles = 0; pl.n_ptiles = 0;
   pl.win_max = 0; pl.nbot_max = 0;
   long long g_off = 0, c_off = 0;
@@ -217,6 +219,8 @@ int get_plan(covspec_ctx* ctx, const covspec_problem* p, cudaStream_t stream) {
     r.ldm = (int)round_up(r.m, 4);
     r.tile_off = pl.n_tiles;
     pl.n_tiles += (r.n + tc::kTileM - 1) / tc::kTileM;
+    r.pair_off = pl.n_pairs;
+    pl.n_pairs += ((r.n + tc::kTileM - 1) / tc::kTileM + 1) / 2;
     r.gram_tile_off = pl.n_gram_tiles;
     r.ptile_off = pl.n_ptiles;
     r.g_off = g_off;
@@ -420,8 +424,53 @@ int make_map_bf16(CUtensorMap* map, const void* base, long long rows, long long 
 
 bool tc_supported(const covspec_ctx* ctx) {
   const covspec_config& c = ctx->cfg;
-  return ctx->tc_ready && c.relevance_path == 0 && c.dtype == COVSPEC_BF16 && c.n_heads > 0 &&
+  return ctx->tc_ready && c.relevance_path != 1 && c.dtype == COVSPEC_BF16 && c.n_heads > 0 &&
          c.head_dim == tc::kHeadDim && c.head_reduce == 0 && c.d >= tc::kBK;
+}
+
+// Eq. 10 on the tensor cores, two-SM form (relevance_pair.cuh): query embedding (MODE 1), -inf fill,
+// fused projection + cosine max over pairs of token tiles.
+int relevance_pair(covspec_ctx* ctx, const covspec_problem* p, float* s_query, cudaStream_t s) {
+  const covspec_config& cfg = ctx->cfg;
+  const Plan& pl = ctx->plan;
+  int P = ctx->P, d = cfg.d;
+  __nv_bfloat16* qn = reinterpret_cast<__nv_bfloat16*>(ctx->Qn);
+  CUtensorMap map_x, map_wk, map_q, map_wq, map_qn, map_qnl;
+  long long lo_off = (long long)cfg.max_total_txt * P;   // lo parts follow the hi parts
+  int st;
+  if ((st = make_map_bf16(&map_x, p->X, pl.total_vis, d, tc::kTileM))) return st;
+  if ((st = make_map_bf16(&map_wk, p->Wk, P, d, tc::kTileN / 2))) return st;
+  if ((st = make_map_bf16(&map_q, p->Q, pl.total_txt, d, tc::kTileM))) return st;
+  if ((st = make_map_bf16(&map_wq, p->Wq, P, d, tc::kTileN / 2))) return st;
+  if ((st = make_map_bf16(&map_qn, qn, pl.total_txt, P, tc::kTT / 2))) return st;
+  if ((st = make_map_bf16(&map_qnl, qn + lo_off, pl.total_txt, P, tc::kTT / 2))) return st;
+  int n_hp = (cfg.n_heads + 1) / 2;
+  tc2::PairParams prm{};
+  prm.plan = ctx->d_plan; prm.batch = p->batch;
+  prm.n_groups = n_hp; prm.hp_per_group = 1;
+  prm.n_heads = cfg.n_heads; prm.k_chunks = (d + tc::kBK - 1) / tc::kBK; prm.P = P;
+  prm.status = ctx->status;
+  const int max_clusters = ctx->num_sms / 2;
+  // query side
+  prof_mark(ctx, ST_QEMBED, 0, s);
+  prm.rows_total = pl.total_txt;
+  prm.n_items = (int)((pl.total_txt + 2 * tc::kTileM - 1) / (2 * tc::kTileM)) * prm.n_groups;
+  prm.qn_out = qn; prm.qn_lo_off = lo_off; prm.s_query = nullptr;
+  int grid = 2 * std::min(prm.n_items, max_clusters);
+  tc2::relevance_pair_kernel<1><<<grid, tc2::kPairThreads, tc2::kSmemBytes2, s>>>(map_q, map_wq, map_qn, map_qnl, prm);
+  LAUNCH_CHECK(ctx);
+  prof_mark(ctx, ST_QEMBED, 1, s);
+  // visual side
+  prof_mark(ctx, ST_RELEVANCE, 0, s);
+  tc::fill_neg_inf_kernel<<<(unsigned)((pl.total_vis + 255) / 256), 256, 0, s>>>(s_query, pl.total_vis);
+  LAUNCH_CHECK(ctx);
+  prm.n_items = pl.n_pairs * prm.n_groups;
+  prm.qn_out = nullptr; prm.s_query = s_query;
+  grid = 2 * std::min(prm.n_items, max_clusters);
+  tc2::relevance_pair_kernel<0><<<grid, tc2::kPairThreads, tc2::kSmemBytes2, s>>>(map_x, map_wk, map_qn, map_qnl, prm);
+  LAUNCH_CHECK(ctx);
+  prof_mark(ctx, ST_RELEVANCE, 1, s);
+  return COVSPEC_OK;
 }
 
 // Eq. 10 on the tensor cores: query embedding (MODE 1), -inf fill, fused projection + cosine max.
@@ -478,7 +527,9 @@ int launch_activity(covspec_ctx* ctx, const covspec_problem* p, float* s_act, bo
   LayerPtrs lp{};
   for (int l = 0; l <= cfg.act_layers; ++l) lp.h[l] = p->Hs[l];
   if (background) {
-    unsigned grid = (unsigned)std::min<long long>((rowsX + 15) / 16, (long long)ctx->num_sms * cfg.activity_overlap);
+    // beside the two-SM relevance kernel only one block per SM fits (shared-memory reserve)
+    int per_sm = cfg.relevance_path == 2 ? 1 : cfg.activity_overlap;
+    unsigned grid = (unsigned)std::min<long long>((rowsX + 15) / 16, (long long)ctx->num_sms * per_sm);
     if (cfg.act_layers <= 4)
       activity_stream_kernel<T, 4><<<grid, 512, 0, s>>>(lp, cfg.act_layers, rowsX, cfg.d, s_act);
     else if (cfg.act_layers <= 8)
@@ -526,7 +577,7 @@ int score_impl(covspec_ctx* ctx, const covspec_problem* p, float* s_query, float
     CUDA_TRY(cudaEventRecord(ctx->ev_join, ctx->side));
   }
   if (use_tc) {
-    int st = relevance_tc(ctx, p, s_query, s);
+    int st = cfg.relevance_path == 2 ? relevance_pair(ctx, p, s_query, s) : relevance_tc(ctx, p, s_query, s);
     if (st) return st;
   } else {
   prof_mark(ctx, ST_QEMBED, 0, s);
@@ -633,7 +684,7 @@ int select_impl(covspec_ctx* ctx, const covspec_problem* p, const float* s_fused
       return COVSPEC_OK;
     }
     sub::basis_init_kernel<<<gb, 256, 0, s>>>(ctx->d_plan, ctx->Yp[0][0], ctx->Yp[0][1], ctx->Yp[1][0],
-                                              ctx->Yp[1][1], ctx->ld, energy, ctx->sync, B);
+                                              ctx->Yp[1][1], ctx->ld, energy, ctx->sync, B, cfg.eig_iters);
     LAUNCH_CHECK(ctx);
     // every multiplication by G, the factorisations between them, the Rayleigh-Ritz solve and the
     // energies: one cooperative launch (its CTAs wait on one another through global counters)
@@ -645,6 +696,7 @@ int select_impl(covspec_ctx* ctx, const covspec_problem* p, const float* s_fused
     fp.ld = ctx->ld;
     fp.partial = ctx->partial; fp.ub = ctx->Ub; fp.energy = energy; fp.sync = ctx->sync;
     fp.max_sweeps = 30; fp.conv_tol = cfg.conv_tol; fp.status = ctx->status;
+    fp.early_stop = cfg.eig_early_stop && cfg.conv_tol > 0.f;
     void* args[] = {&ctx->map_gh, &ctx->map_gl, &ctx->map_y[0][0], &ctx->map_y[0][1], &ctx->map_y[1][0],
                     &ctx->map_y[1][1], &fp};
     CUDA_TRY(cudaLaunchCooperativeKernel(reinterpret_cast<void*>(sub::subspace_kernel), dim3(pl.pow_grid),
@@ -654,7 +706,7 @@ int select_impl(covspec_ctx* ctx, const covspec_problem* p, const float* s_fused
     // no request reaches stage 2: the final selection keeps the preselected sets; energies are zero
     dim3 gz(1, B);
     sub::basis_init_kernel<<<gz, 256, 0, s>>>(ctx->d_plan, ctx->Yp[0][0], ctx->Yp[0][1], ctx->Yp[1][0],
-                                              ctx->Yp[1][1], ctx->ld, energy, ctx->sync, B);
+                                              ctx->Yp[1][1], ctx->ld, energy, ctx->sync, B, cfg.eig_iters);
     LAUNCH_CHECK(ctx);
   }
   if (pl.n_stage2 > 0) prof_mark(ctx, ST_EIG, 1, s);
@@ -714,6 +766,7 @@ void covspec_default_config(covspec_config* c) {
   c->ritz_window = 16;
   c->activity_overlap = 1;
   c->conv_tol = 2e-3f;
+  c->eig_early_stop = 1;
 }
 
 int covspec_budgets(const covspec_config* cfg, int n, int keep, int* b_vis, int* m, int* r) {
@@ -851,6 +904,10 @@ int covspec_prune_init(const covspec_config* cfg, covspec_ctx** out) {
                              tc::kSmemBytes) == cudaSuccess &&
         cudaFuncSetAttribute(tc::relevance_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              tc::kSmemBytes) == cudaSuccess &&
+        cudaFuncSetAttribute(tc2::relevance_pair_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             tc2::kSmemBytes2) == cudaSuccess &&
+        cudaFuncSetAttribute(tc2::relevance_pair_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             tc2::kSmemBytes2) == cudaSuccess &&
         cudaFuncSetAttribute(sub::gram_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              sub::kGramSmem) == cudaSuccess &&
         cudaFuncSetAttribute(sub::subspace_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,

@@ -9,6 +9,11 @@
 //   factor[b]   number of triangular factors published for request b; the epilogue of step k needs
 //               factor[b] >= k
 //   ritz[b]     1 once the Rayleigh-Ritz vectors of the last block are published
+//   last[b]     index of the request's last step: eig_iters on entry; the tile that factors step k
+//               lowers it to k + 2 when the Ritz value estimates say that the energies will have
+//               settled by then (see team_cholesky).  It only ever decreases, and a change made after
+//               step k first matters two steps later, so every role of every CTA reads the same
+//               answer to "is step s skipped?" and "is step s the last?"
 // The tile that makes arrive[b] reach tiles(b) * (k + 1) (an atomic ticket; nobody waits for it to be
 // a particular CTA) sums the partial Gram matrices in tile order and factors the sum right there: a
 // Cholesky factorisation after the first steps, the Rayleigh-Ritz solve of the window next to the cut
@@ -24,7 +29,7 @@
 namespace covspec {
 namespace sub {
 
-constexpr int kSyncStride = 4;           // unsigned words per request: arrive, factor, ritz, unused
+constexpr int kSyncStride = 4;           // unsigned words per request: arrive, factor, ritz, last
 
 struct FusedParams {
   const ReqPlan* plan;
@@ -44,6 +49,7 @@ struct FusedParams {
   unsigned* sync;           // [batch][kSyncStride] counters (zero on entry), then the abort word
   int max_sweeps;
   float conv_tol;           // bound on the estimated energy error before NOCONVERGE is raised
+  int early_stop;           // 1: requests whose estimate is far below conv_tol stop before `steps`
   int* status;
 };
 
@@ -73,6 +79,26 @@ __device__ __forceinline__ bool flag_wait_ge(const unsigned* ctr, unsigned targe
   *abort_flag = 1;
   atomicExch(gabort, 1u);
   return false;
+}
+
+// One thread decides whether step `step` (>= 1) of a request runs, and waits until it can: returns
+// 1 when every tile has finished step - 1 (run; *last_out = the request's last step as known now),
+// 0 when the request's last step is before `step` (skip), -1 when the wait was given up.  `last` is
+// examined before `arrive`: after the request's final step arrive reaches the count the skipped
+// next step would wait for.
+__device__ __forceinline__ int step_decide(const unsigned* sync_b, unsigned nt, int step, unsigned* gabort,
+                                           volatile int* abort_flag, int* last_out) {
+  for (uint32_t i = 0; i < kFlagSpinLimit; ++i) {
+    const unsigned arrived = ld_acquire_u32(sync_b);
+    const int last = (int)ld_acquire_u32(sync_b + 3);
+    if (last < step) return 0;
+    if (arrived >= nt * (unsigned)step) { *last_out = last; return 1; }
+    if ((i & 15u) == 15u && (ld_acquire_u32(gabort) != 0u || *abort_flag)) { *abort_flag = 1; return -1; }
+    __nanosleep(64);
+  }
+  *abort_flag = 1;
+  atomicExch(gabort, 1u);
+  return -1;
 }
 
 // Layout of a partial Gram matrix in global memory: the 8 x 8 tiles of the lower triangle, tile
@@ -341,7 +367,14 @@ __device__ __forceinline__ bool extra_tile(int e, int nb8, int units, int& ta, i
 
 // Cholesky factor of the summed Gram matrix, written in the layout the triangular solve reads
 // (see lt_row_offset) followed by the reciprocal diagonal.  Tm: cholesky_smem_bytes(p) of scratch.
-__device__ __noinline__ void team_cholesky(const double* pbase, int nt, int p, float* out, double* Tm) {
+// Returns (to every thread) whether the iteration may stop two steps from now: from the diagonal of
+// the summed Gram matrix B = Y'^T Y' (theta_i = sqrt(B_ii) estimates the i-th eigenvalue of G once the
+// basis has started to order itself) the energy error after q_final multiplications is predicted as
+// max_i 2 (theta_i / theta_1) (theta_min / theta_i)^q_final over the kept directions i < r that the
+// cut can tell apart from the discarded ones (theta_i - theta_min > 1e-3 theta_1), the estimate
+// team_ritz reports at the end; stop_below is the bound it has to stay under (0: never stop early).
+__device__ __noinline__ bool team_cholesky(const double* pbase, int nt, int p, int r, float* out, double* Tm,
+                                           float* dg, volatile int* s_word, int q_final, float stop_below) {
   const int et = threadIdx.x, warp = et >> 5, lane = et & 31;
   const int P = (p + 7) & ~7, nb = (p + 7) >> 3;
   auto epi_sync = [&]() { named_barrier(1, kEpiThreads); };
@@ -355,6 +388,25 @@ __device__ __noinline__ void team_cholesky(const double* pbase, int nt, int p, f
   for (int j = p + et; j < P; j += kEpiThreads) out[kLtFloats + j] = 1.f;
   team_sum_partials(Tm, pbase, nt, nb * (nb + 1) / 2 * 64, et, kEpiThreads);
   epi_sync();
+  if (stop_below > 0.f) {
+    for (int i = et; i < p; i += kEpiThreads) dg[i] = sqrtf(fmaxf((float)Tm[tile_offset(i, i)], 0.f));
+    if (et == 0) *s_word = 0;
+    epi_sync();
+    if (warp == 0) {
+      float tmin = 3.0e38f, tmax = 0.f;
+      for (int i = lane; i < p; i += 32) { tmin = fminf(tmin, dg[i]); tmax = fmaxf(tmax, dg[i]); }
+      tmin = warp_min(tmin); tmax = warp_max(tmax);
+      float worst = 0.f;
+      for (int i = lane; i < r; i += 32) {
+        float th = dg[i];
+        if (th - tmin > 1e-3f * tmax && th > 0.f) worst = fmaxf(worst, 2.f * (th / tmax) * __powf(tmin / th, (float)q_final));
+      }
+      worst = warp_max(worst);
+      if (lane == 0 && tmax > 0.f && worst < stop_below) *s_word = 1;
+    }
+    epi_sync();
+  }
+  const bool stop = stop_below > 0.f && *s_word != 0;
   // row j of the layout holds L[i][j] for i >= (j & ~3): lane -> (j, half of the tile's rows), so that
   // a lane's four entries are consecutive floats
   auto store = [&](int I, int J, const double* tile, const double* rd) {
@@ -371,6 +423,7 @@ __device__ __noinline__ void team_cholesky(const double* pbase, int nt, int p, f
     }
   };
   cholesky_blocked_team(p, Tm, Tm + (size_t)nb * (nb + 1) / 2 * 64, et, kEpiThreads, store, epi_sync);
+  return stop;
 }
 
 // Rayleigh-Ritz on the window next to the cut (see eig_kernels.cuh) and the convergence estimate.
@@ -495,9 +548,9 @@ subspace_kernel(const __grid_constant__ CUtensorMap map_gh, const __grid_constan
   uint64_t* epi_done = bars + 6;         // the region no longer belongs to the epilogue
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 8);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-  volatile int* s_word = reinterpret_cast<volatile int*>(tmem_slot + 2);      // broadcast slot of the epilogue
-  int* s_flag = reinterpret_cast<int*>(tmem_slot + 3);                        // Jacobi rotation flag
-  float* s_scale = reinterpret_cast<float*>(tmem_slot + 4);
+  volatile int* s_word = reinterpret_cast<volatile int*>(tmem_slot + 2);      // [2] broadcast slots of the epilogue
+  int* s_flag = reinterpret_cast<int*>(tmem_slot + 4);                        // Jacobi rotation flag
+  float* s_scale = reinterpret_cast<float*>(tmem_slot + 5);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   unsigned* gabort = prm.sync + (size_t)prm.batch * kSyncStride;
 
@@ -536,15 +589,19 @@ subspace_kernel(const __grid_constant__ CUtensorMap map_gh, const __grid_constan
           const int item = s_items[si];
           int b, tile; ReqPlan rp;
           decode(item, b, rp, tile);
+          if (step > 0) {
+            // every tile of the request has written its slab of the block this step multiplies,
+            // unless the request has already had its last step
+            const unsigned nt = (unsigned)((rp.m + kTile - 1) / kTile);
+            int last_b;
+            const int go = step_decide(prm.sync + (size_t)b * kSyncStride, nt, step, gabort, abort_flag, &last_b);
+            if (go < 0) { ok = false; break; }
+            if (go == 0) { --n; continue; }
+            fence_proxy_async_all();
+          }
           // the previous item's staged block (and whatever its last tile factored) lives in the
           // ring until its epilogue is done
           if (n > 0 && !(ok = mbar_wait(epi_done, (n - 1) & 1u, abort_flag))) break;
-          if (step > 0) {
-            // every tile of the request has written its slab of the block this step multiplies
-            const unsigned nt = (unsigned)((rp.m + kTile - 1) / kTile);
-            if (!(ok = flag_wait_ge(prm.sync + (size_t)b * kSyncStride, nt * (unsigned)step, gabort, abort_flag))) break;
-            fence_proxy_async_all();
-          }
           int k_chunks = (rp.m + kBK - 1) / kBK;
           for (int kc = 0; kc < k_chunks; ++kc, ++it) {
             int s = it % kPowStages;
@@ -572,6 +629,13 @@ subspace_kernel(const __grid_constant__ CUtensorMap map_gh, const __grid_constan
           int b, tile; ReqPlan rp;
           decode(item, b, rp, tile);
           const uint32_t idesc = umma_idesc(kTile, (rp.p + 15) & ~15);
+          if (step > 0) {
+            const unsigned nt = (unsigned)((rp.m + kTile - 1) / kTile);
+            int last_b;
+            const int go = step_decide(prm.sync + (size_t)b * kSyncStride, nt, step, gabort, abort_flag, &last_b);
+            if (go < 0) { ok = false; break; }
+            if (go == 0) { --n; continue; }
+          }
           if (!(ok = mbar_wait(acc_empty, (n & 1u) ^ 1u, abort_flag))) break;
           tc_fence_after();
           int k_chunks = (rp.m + kBK - 1) / kBK;
@@ -614,17 +678,32 @@ subspace_kernel(const __grid_constant__ CUtensorMap map_gh, const __grid_constan
     int cached_b = -1, cached_step = -1;
     bool ok = true;
     for (int step = 0; step <= last_step; ++step) {
-      const bool identity = step == 0, is_last = step == last_step;
+      const bool identity = step == 0;
       __nv_bfloat16* y_hi = prm.y_hi[(step & 1) ^ 1];
       __nv_bfloat16* y_lo = prm.y_lo[(step & 1) ^ 1];
-      float* yf = is_last ? prm.yf[1] : (step == last_step - 1 ? prm.yf[0] : nullptr);
-      float* qprev = is_last ? prm.yf[0] : nullptr;
       for (int si = s_begin; si < s_end; ++si, ++n) {
         const int item = s_items[si];
         int b, tile; ReqPlan rp;
         decode(item, b, rp, tile);
         const int p = rp.p, P = (p + 7) & ~7;
         unsigned* sync_b = prm.sync + (size_t)b * kSyncStride;
+        const unsigned nt = (unsigned)((rp.m + kTile - 1) / kTile);
+        // does the request still run this step, and is it its last one?  (one answer for the team)
+        int last_b = last_step;
+        if (!identity) {
+          epi_sync();
+          if (et == 0) {
+            int lb = last_step;
+            const int go = step_decide(sync_b, nt, step, gabort, abort_flag, &lb);
+            s_word[0] = go; s_word[1] = lb;
+          }
+          epi_sync();
+          const int go = s_word[0];
+          last_b = s_word[1];
+          if (go == 0) { --n; continue; }
+          if (go < 0) ok = false;
+        }
+        const bool is_last = step == last_b;
         if (!identity && (b != cached_b || step != cached_step)) {
           // the factor of the previous block, published by whichever tile finished that step last
           ok = team_wait(sync_b + 1, (unsigned)step) && ok;
@@ -639,6 +718,16 @@ subspace_kernel(const __grid_constant__ CUtensorMap map_gh, const __grid_constan
           epi_sync();
           cached_b = b; cached_step = step;
         }
+        // the block before the last multiplication is kept in float32 as well: whether this is that
+        // step is known once the previous step's factor (and its decision) has been published
+        if (!identity && !is_last) {
+          if (et == 0) s_word[1] = (int)ld_acquire_u32(sync_b + 3);
+          epi_sync();
+          last_b = s_word[1];
+          epi_sync();
+        }
+        float* yf = is_last ? prm.yf[1] : (step == last_b - 1 ? prm.yf[0] : nullptr);
+        float* qprev = is_last ? prm.yf[0] : nullptr;
         const int nrows = min(kTile, rp.m - tile * kTile);
         // ---- Y_next row = T row * L^-T (forward substitution per row), staged as xs[c][r] ----
         // Between the first and the last step two threads share a row: warps 0-3 own the 32-column
@@ -844,7 +933,6 @@ subspace_kernel(const __grid_constant__ CUtensorMap map_gh, const __grid_constan
         __threadfence();
         fence_proxy_async_all();
         epi_sync();
-        const unsigned nt = (unsigned)((rp.m + kTile - 1) / kTile);
         if (et == 0) {
           unsigned old = atomicAdd(sync_b, 1u);
           // one decision for the whole team (a CTA that has given up factors nothing)
@@ -857,13 +945,20 @@ subspace_kernel(const __grid_constant__ CUtensorMap map_gh, const __grid_constan
           const double* pbase = prm.partial + (size_t)rp.ptile_off * kTileDoubles;
           double* Tm = reinterpret_cast<double*>(smem);        // the region is free: every thread passed the barrier
           if (!is_last) {
-            team_cholesky(pbase, (int)nt, p, prm.lbuf + (size_t)b * kLbufStride, Tm);
+            // after the second multiplication and later: may step + 2 be the last one?  (asked with a
+            // margin of 8 under the tolerance; the estimate is rough while the basis is still mixing)
+            const bool may_stop = prm.early_stop && step >= 1 && step + 2 < last_b && p < rp.m;
+            const bool stop = team_cholesky(pbase, (int)nt, p, rp.r, prm.lbuf + (size_t)b * kLbufStride, Tm, dinv,
+                                            s_word, step + 3, may_stop ? 0.125f * prm.conv_tol : 0.f);
             __threadfence();
             epi_sync();
-            if (et == 0) st_release_u32(sync_b + 1, (unsigned)(step + 1));
+            if (et == 0) {
+              if (stop) st_release_u32(sync_b + 3, (unsigned)(step + 2));
+              st_release_u32(sync_b + 1, (unsigned)(step + 1));
+            }
           } else {
             team_ritz(pbase, (int)nt, p, rp.win, rp.r, rp.m, prm.ub + (size_t)b * kPMax * kPMax, reinterpret_cast<float*>(smem), lt,
-                      s_scale, s_flag, prm.max_sweeps, prm.conv_tol, prm.steps, prm.status);
+                      s_scale, s_flag, prm.max_sweeps, prm.conv_tol, step + 1, prm.status);
             __threadfence();
             epi_sync();
             if (et == 0) st_release_u32(sync_b + 2, 1u);

@@ -240,16 +240,16 @@ split_planes_kernel(const ReqPlan* __restrict__ plan, const float* __restrict__ 
 // Start block of the subspace iteration: entries uniform in [-1, 1) from a counter hash of
 // (request, basis vector, position); zero in the padding columns and in the unused basis rows
 // p .. round_up(p, 16) - 1 of both plane buffers (the MMA reads them, nothing else writes them).
-// The same launch clears the per-request counters of the fused subspace kernel (4 words per request,
-// then the abort word) and writes zero energies for the requests that skip stage 2.
+// The same launch resets the per-request words of the fused subspace kernel (three counters and the
+// index of the last step per request, then the abort word) and writes zero energies for the requests that skip stage 2.
 __global__ void __launch_bounds__(256)
 basis_init_kernel(const ReqPlan* __restrict__ plan, __nv_bfloat16* __restrict__ y_hi,
                   __nv_bfloat16* __restrict__ y_lo, __nv_bfloat16* __restrict__ y2_hi,
                   __nv_bfloat16* __restrict__ y2_lo, int ld, float* __restrict__ energy,
-                  unsigned* __restrict__ sync, int batch) {
+                  unsigned* __restrict__ sync, int batch, int last_step) {
   ReqPlan rp = plan[blockIdx.y];
   if (blockIdx.x == 0) {
-    if (threadIdx.x < 4) sync[blockIdx.y * 4 + threadIdx.x] = 0u;
+    if (threadIdx.x < 4) sync[blockIdx.y * 4 + threadIdx.x] = threadIdx.x == 3 ? (unsigned)last_step : 0u;
     if (blockIdx.y == 0 && threadIdx.x >= 32 && threadIdx.x < 36) sync[batch * 4 + threadIdx.x - 32] = 0u;
     if (!rp.stage2)
       for (int i = threadIdx.x; i < rp.m; i += blockDim.x) energy[rp.presel_off + i] = 0.f;

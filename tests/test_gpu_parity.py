@@ -65,6 +65,14 @@ def test_zero_token_on_the_tensor_core_path():
     _report(wl.name, parity.run_gpu(wl))
 
 
+@pytest.mark.parametrize("kw", [SMALL[2], SMALL[7]], ids=lambda kw: f"seed{kw['seed']}")
+def test_two_sm_relevance_kernel(kw):
+    # relevance_path = 2: the cta_group::2 form of the relevance kernel (pairs of token tiles on pairs
+    # of SMs) gives the same scores; ragged sizes, an odd number of tiles, more than 256 query elements
+    wl = workloads.make_workload(f"pair{kw['seed']}", **kw)
+    _report(wl.name, parity.run_gpu(wl, pruner_kw=dict(relevance_path=2)))
+
+
 def test_degenerate_requests():
     # N = 1; B_vis >= N (keep everything); B_vis = N - 1; B_vis = 1; T = 1
     wl = workloads.make_workload("degenerate", seed=21, dtype=torch.bfloat16, batch=6,
