@@ -330,9 +330,10 @@ def run_correction(args):
 class Runner:
     """One configuration on one device: input sets, context, output buffers."""
 
-    def __init__(self, api, name, dev, seed, copies=0):
+    def __init__(self, api, name, dev, seed, copies=0, batch=0):
         self.name, self.dev = name, dev
-        wl0 = workloads.make_config(name, device=dev, seed=seed)
+        over = dict(batch=batch) if batch else {}
+        wl0 = workloads.make_config(name, device=dev, seed=seed, **over)
         self.wl0 = wl0
         self.n_vis = np.diff(wl0.vis_offsets).tolist()
         self.n_txt = np.diff(wl0.txt_offsets).tolist()
@@ -342,7 +343,7 @@ class Runner:
         copies = copies or max(2, int(math.ceil(4 * L2_BYTES / in_bytes)))
         self.copies = min(copies, 8)
         sizes = (self.n_vis, self.n_txt)
-        self.sets = [wl0] + [workloads.make_config(name, device=dev, seed=seed + 17 * (i + 1), sizes=sizes)
+        self.sets = [wl0] + [workloads.make_config(name, device=dev, seed=seed + 17 * (i + 1), sizes=sizes, **over)
                              for i in range(self.copies - 1)]
         self.pr = api.Pruner.for_workload(wl0)
         self.ms = [self.pr.marshal(w) for w in self.sets]
@@ -429,6 +430,9 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-others", action="store_true", help="skip the other named configurations")
     ap.add_argument("--no-e2e", action="store_true", help="skip the end-to-end leg (profiling runs)")
+    ap.add_argument("--batch", type=int, default=0,
+                    help="cut the configuration to this many requests (small cases for profiler captures; "
+                         "the line then says so in config.workload)")
     ap.add_argument("--ref-budget", type=float, default=20.0)
     ap.add_argument("--kernel", default="prune", choices=["prune", "correct"],
                     help="prune: the headline path (default); correct: the gating / correction kernel")
@@ -461,7 +465,7 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
-    run = Runner(api, args.config, dev, rank_seed(args.config, rank), args.copies)
+    run = Runner(api, args.config, dev, rank_seed(args.config, rank), args.copies, args.batch)
     wl0, pr, work = run.wl0, run.pr, run.work
     tokens = run.tokens
 
