@@ -37,10 +37,12 @@ import torch
 
 from paper_2605_02218_b200 import workloads
 
-# dram__bytes_read.sum + dram__bytes_write.sum of the visual-side relevance kernel per visual token
-# (one ncu capture on a c5-shaped batch cut to two requests, scaled by the tokens one launch
-# processes; see the summary named here).  None while no capture of the current kernel exists.
-NCU_RELEVANCE_TRAFFIC = {"bytes_per_token": None, "config": "c5", "source": None}
+# dram__bytes_read.sum + dram__bytes_write.sum of the visual-side relevance kernel from one ncu
+# capture on c5 cut to one request (16384 tokens: 148.6 MB, of which the 25.7 MB of projection
+# weights are read once per launch and the rest grows with the tokens), scaled to the tokens one
+# launch of the full workload processes; see the summary named here.
+NCU_RELEVANCE_TRAFFIC = {"bytes_per_token": (148.589e6 - 25.69e6) / 16384, "fixed_bytes": 25.69e6, "config": "c5",
+                         "source": "profiles/relevance_tc_kernel_c5_one_request.md"}
 NCU_CORRECT_BYTES_PER_ROW = 343.9e6 / 512          # profiles/correct_kernel_vocab152k.md
 
 METRIC = "visual_tokens_pruned_per_s"
@@ -562,7 +564,7 @@ def main():
         rel_tf = work["relevance_flops"] / (rel_ms * 1e-3) / 1e12 if rel_ms > 0 else 0.0
         traffic = None
         if NCU_RELEVANCE_TRAFFIC["bytes_per_token"] and NCU_RELEVANCE_TRAFFIC["config"] == args.config:
-            traffic = NCU_RELEVANCE_TRAFFIC["bytes_per_token"] * tokens
+            traffic = NCU_RELEVANCE_TRAFFIC["bytes_per_token"] * tokens + NCU_RELEVANCE_TRAFFIC["fixed_bytes"]
         roofline = dict(bound=roof["bound"], achieved=roof["achieved"], peak=roof["peak"], unit=roof["unit"],
                         frac=roof["frac"], traffic=traffic,
                         kernel="covspec_prune (fused call, all stages); dominant stage: %s" % dom,
@@ -575,6 +577,8 @@ def main():
                                               frac=rel_tf / burst if burst else None, ms_per_launch=rel_ms,
                                               flops_per_launch=work["relevance_flops"], traffic=traffic,
                                               traffic_source=NCU_RELEVANCE_TRAFFIC["source"],
+                                              note="stage time by events; the activity stream (Eq. 11) runs "
+                                                   "beside this kernel on a second stream and slows it",
                                               peak_source="burst bf16, " + peaks["source"]))
         line = dict(
             metric=METRIC, value=world * tokens / (ms_step * 1e-3), unit=UNIT, n_gpus=world,
