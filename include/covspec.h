@@ -177,6 +177,12 @@ int covspec_prune(covspec_ctx* ctx, const covspec_problem* p, void* out_hidden, 
  * COVSPEC_ERR_NOCONVERGE) and clears it. */
 int covspec_get_device_status(covspec_ctx* ctx, void* stream);
 
+/* Diagnostics of the subspace iteration behind Eq. 14 for the last covspec_select / covspec_prune call
+ * on this context: multiplications[b] (host, [batch]) receives the number of multiplications by the
+ * Gram matrix that request b ran (eig_iters + 1 unless it stopped early, see eig_early_stop; 0 for a
+ * request that skipped stage 2).  Synchronises `stream`. */
+int covspec_get_iteration_counts(covspec_ctx* ctx, int batch, int* multiplications, void* stream);
+
 /* Device-side gating and correction over the vocabulary (Sec. III-B.1 and III-C.2), one call for
  * `rows` decoding positions; needs no context and no workspace.
  *  logit_dtype   COVSPEC_F32, COVSPEC_BF16 or COVSPEC_F16 (the paper sends logits as float16)

@@ -28,7 +28,7 @@ EXPORTS = [
     "covspec_profile_stage_name", "covspec_query_score_static", "covspec_selftest_wait_timeout",
     "covspec_correct", "covspec_fanout", "covspec_branch_candidates",
     "covspec_uplink_bits", "covspec_downlink_bits", "covspec_comm_latency", "covspec_ema_update",
-    "covspec_draft_length",
+    "covspec_draft_length", "covspec_get_iteration_counts",
 ]
 STATIC_MAX_BATCH = 256
 STATIC_MAX_QUERY_ELEMS = 1 << 20
@@ -96,6 +96,7 @@ def load_library():
     lib.covspec_compact_rows.argtypes = [vp, C.POINTER(Problem), vp, ip, vp, C.c_longlong, vp, vp]
     lib.covspec_get_device_status.argtypes = [vp, vp]
     lib.covspec_selftest_wait_timeout.argtypes = [vp, vp]
+    lib.covspec_get_iteration_counts.argtypes = [vp, C.c_int, ip, vp]
     lib.covspec_fanout.argtypes = [C.c_int, C.c_double, C.c_int]
     lib.covspec_uplink_bits.argtypes = [C.c_longlong, C.c_int, C.c_longlong, C.c_int]
     lib.covspec_uplink_bits.restype = C.c_double
@@ -349,6 +350,15 @@ class Pruner:
         st = self.lib.covspec_selftest_wait_timeout(self._ctx, _stream())
         if st:
             raise CovspecError(st, "covspec_selftest_wait_timeout")
+
+    def iteration_counts(self, batch: int):
+        """covspec_get_iteration_counts: multiplications by the Gram matrix per request of the last call."""
+        out = np.zeros(batch, dtype=np.int32)
+        st = self.lib.covspec_get_iteration_counts(self._ctx, int(batch), out.ctypes.data_as(C.POINTER(C.c_int)),
+                                                   _stream())
+        if st:
+            raise CovspecError(st, "covspec_get_iteration_counts")
+        return out
 
     def device_status(self) -> int:
         return int(self.lib.covspec_get_device_status(self._ctx, _stream()))

@@ -1101,6 +1101,18 @@ int covspec_get_device_status(covspec_ctx* ctx, void* stream) {
   return COVSPEC_OK;
 }
 
+int covspec_get_iteration_counts(covspec_ctx* ctx, int batch, int* multiplications, void* stream) {
+  if (!ctx || !multiplications || batch < 1 || batch > ctx->cfg.max_batch) return COVSPEC_ERR_ARG;
+  if (!ctx->plan.valid || (int)ctx->plan.req.size() != batch) return COVSPEC_ERR_SHAPE;
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  std::vector<unsigned> words((size_t)batch * sub::kSyncStride);
+  CUDA_TRY(cudaMemcpyAsync(words.data(), ctx->sync, sizeof(unsigned) * words.size(), cudaMemcpyDeviceToHost, s));
+  CUDA_TRY(cudaStreamSynchronize(s));
+  for (int b = 0; b < batch; ++b)
+    multiplications[b] = ctx->plan.req[b].stage2 ? (int)words[(size_t)b * sub::kSyncStride + 3] + 1 : 0;
+  return COVSPEC_OK;
+}
+
 int covspec_correct(int logit_dtype, int rows, int vocab, long long ld, const void* z_draft,
                     const void* z_target, const int* drafted, const float* uniforms, float gamma,
                     float* margin, int* gate, float* accept, float* resid_mass, int* token,

@@ -703,7 +703,6 @@ subspace_kernel(const __grid_constant__ CUtensorMap map_gh, const __grid_constan
           if (go == 0) { --n; continue; }
           if (go < 0) ok = false;
         }
-        const bool is_last = step == last_b;
         if (!identity && (b != cached_b || step != cached_step)) {
           // the factor of the previous block, published by whichever tile finished that step last
           ok = team_wait(sync_b + 1, (unsigned)step) && ok;
@@ -718,15 +717,16 @@ subspace_kernel(const __grid_constant__ CUtensorMap map_gh, const __grid_constan
           epi_sync();
           cached_b = b; cached_step = step;
         }
-        // the block before the last multiplication is kept in float32 as well: whether this is that
-        // step is known once the previous step's factor (and its decision) has been published
-        if (!identity && !is_last) {
+        // whether this is the request's last step is known once the previous step's factor has been
+        // published: the tile that computed it may have declared this step the last one
+        if (!identity) {
           if (et == 0) s_word[1] = (int)ld_acquire_u32(sync_b + 3);
           epi_sync();
           last_b = s_word[1];
           epi_sync();
         }
-        float* yf = is_last ? prm.yf[1] : (step == last_b - 1 ? prm.yf[0] : nullptr);
+        const bool is_last = step == last_b;
+        float* yf = is_last ? prm.yf[1] : nullptr;
         float* qprev = is_last ? prm.yf[0] : nullptr;
         const int nrows = min(kTile, rp.m - tile * kTile);
         // ---- Y_next row = T row * L^-T (forward substitution per row), staged as xs[c][r] ----
@@ -795,15 +795,25 @@ subspace_kernel(const __grid_constant__ CUtensorMap map_gh, const __grid_constan
           ok = ok && mbar_wait(acc_full, n & 1u, abort_flag);      // the ring is no longer read
           const int t4 = et - 128;
           float* qrows = qprev + ((size_t)rp.presel_off + tile * kTile) * kPMax;
-          for (int c = t4; c < P; c += 128) {
+          {
+            // the block this step multiplied, row t4 of the tile, from its two bf16 planes
+            const __nv_bfloat16* ph = prm.y_hi[step & 1] + (size_t)b * kPMax * prm.ld + tile * kTile + t4;
+            const __nv_bfloat16* pl = prm.y_lo[step & 1] + (size_t)b * kPMax * prm.ld + tile * kTile + t4;
+            const unsigned short* uh = reinterpret_cast<const unsigned short*>(ph);
+            const unsigned short* ul = reinterpret_cast<const unsigned short*>(pl);
+            const bool have_row = t4 < nrows;
 #pragma unroll 1
-            for (int r0 = 0; r0 < kTile; r0 += 8) {
-              float v[8];
+            for (int c0 = 0; c0 < P; c0 += 8) {
+              unsigned short vh[8], vl[8];
+#pragma unroll
+              for (int u = 0; u < 8; ++u) {
+                const bool in = have_row && c0 + u < p;
+                vh[u] = in ? __ldcg(uh + (size_t)(c0 + u) * prm.ld) : (unsigned short)0;
+                vl[u] = in ? __ldcg(ul + (size_t)(c0 + u) * prm.ld) : (unsigned short)0;
+              }
 #pragma unroll
               for (int u = 0; u < 8; ++u)
-                v[u] = (r0 + u < nrows && c < p) ? __ldcg(qrows + (size_t)(r0 + u) * kPMax + c) : 0.f;
-#pragma unroll
-              for (int u = 0; u < 8; ++u) xq[c * kXsLd + r0 + u] = v[u];
+                xq[(c0 + u) * kXsLd + t4] = __uint_as_float((uint32_t)vh[u] << 16) + __uint_as_float((uint32_t)vl[u] << 16);
             }
           }
           named_barrier(2, 128);
@@ -817,8 +827,9 @@ subspace_kernel(const __grid_constant__ CUtensorMap map_gh, const __grid_constan
             for (int e = 0; e < 8; ++e) xq[(jb + e) * kXsLd + t4] = acc[e];
           }
           named_barrier(2, 128);
-          for (int c = t4; c < p; c += 128)
-            for (int rr = 0; rr < nrows; ++rr) qrows[(size_t)rr * kPMax + c] = xq[c * kXsLd + rr];
+          // only the window columns are read again (second half of Eq. 15)
+          for (int c = (p - rp.win) + (t4 & 31); c < p; c += 32)
+            for (int rr = t4 >> 5; rr < nrows; rr += 4) qrows[(size_t)rr * kPMax + c] = xq[c * kXsLd + rr];
         }
         epi_sync();                                  // the staged block is complete
         if (is_last && et < nrows) {
@@ -851,10 +862,10 @@ subspace_kernel(const __grid_constant__ CUtensorMap map_gh, const __grid_constan
           }
         }
         if (yf != nullptr) {
-          // float32 block, one token per row; consecutive threads write consecutive columns
+          // float32 window columns of the final block, one token per row (second half of Eq. 15)
           float* yrows = yf + ((size_t)rp.presel_off + tile * kTile) * kPMax;
-          for (int c = et & 127; c < p; c += 128)
-            for (int rr = et >> 7; rr < nrows; rr += 2) yrows[(size_t)rr * kPMax + c] = xs[c * kXsLd + rr];
+          for (int c = (p - rp.win) + (et & 31); c < p; c += 32)
+            for (int rr = et >> 5; rr < nrows; rr += 8) yrows[(size_t)rr * kPMax + c] = xs[c * kXsLd + rr];
         }
         // ---- float64 partial Gram of the tile on the FP64 tensor cores ----
         const int coff = is_last ? ((p - rp.win) & ~7) : 0;
@@ -945,15 +956,17 @@ subspace_kernel(const __grid_constant__ CUtensorMap map_gh, const __grid_constan
           const double* pbase = prm.partial + (size_t)rp.ptile_off * kTileDoubles;
           double* Tm = reinterpret_cast<double*>(smem);        // the region is free: every thread passed the barrier
           if (!is_last) {
-            // after the second multiplication and later: may step + 2 be the last one?  (asked with a
-            // margin of 8 under the tolerance; the estimate is rough while the basis is still mixing)
-            const bool may_stop = prm.early_stop && step >= 1 && step + 2 < last_b && p < rp.m;
+            // after the second multiplication and later: may the next step be the last one?  (asked with a
+            // margin of 8 under the tolerance, 64 at the first opportunity: the estimate is rough while
+            // the basis is still mixing)
+            const bool may_stop = prm.early_stop && step >= 1 && step + 1 < last_b && p < rp.m;
+            const float margin = step == 1 ? 0.015625f : 0.125f;
             const bool stop = team_cholesky(pbase, (int)nt, p, rp.r, prm.lbuf + (size_t)b * kLbufStride, Tm, dinv,
-                                            s_word, step + 3, may_stop ? 0.125f * prm.conv_tol : 0.f);
+                                            s_word, step + 2, may_stop ? margin * prm.conv_tol : 0.f);
             __threadfence();
             epi_sync();
             if (et == 0) {
-              if (stop) st_release_u32(sync_b + 3, (unsigned)(step + 2));
+              if (stop) st_release_u32(sync_b + 3, (unsigned)(step + 1));
               st_release_u32(sync_b + 1, (unsigned)(step + 1));
             }
           } else {

@@ -361,3 +361,25 @@ def test_capacity_and_argument_errors():
     with pytest.raises(api.CovspecError) as e:
         pr.prune(m)
     assert e.value.status == -1
+
+
+def test_iteration_counts_reflect_the_adaptive_stop():
+    # Requests that skip the spectral stage report 0 multiplications; the others report a count
+    # between the minimum the stop rule can reach and eig_iters + 1, and exactly eig_iters + 1 when
+    # the adaptive stop is switched off.
+    from paper_2605_02218_b200 import api
+    wl = workloads.make_workload("counts", seed=41, dtype=torch.bfloat16, batch=4, n_vis=(300, 900),
+                                 n_txt=(4, 12), d=256, n_heads=4, rank=16, keep_ratio=0.25).to("cuda:0")
+    for stop in (1, 0):
+        pr = api.Pruner.for_workload(wl, eig_early_stop=stop)
+        pr.prune(pr.marshal(wl))
+        counts = pr.iteration_counts(wl.batch)
+        iters = pr.cfg.eig_iters
+        assert pr.device_status() == 0
+        pr.close()
+        assert len(counts) == wl.batch
+        for c in counts:
+            assert c == 0 or 3 <= c <= iters + 1
+        assert any(c > 0 for c in counts)
+        if not stop:
+            assert all(c in (0, iters + 1) for c in counts)
