@@ -30,29 +30,66 @@ template <> struct Vec<float> { static constexpr int N = 4; };
 template <> struct Vec<__half> { static constexpr int N = 8; };
 template <> struct Vec<__nv_bfloat16> { static constexpr int N = 8; };
 
-// Loads the N consecutive logits that start at element `i` (a multiple of N) of `row`; elements at
-// or beyond `w` read as -inf (probability zero).  The row base is 16-byte aligned.
+constexpr float kLog2e = 1.4426950408889634f;
+
+// 2^x on the special-function unit, results below the normal range flushed to zero (a probability
+// under 1e-38): one instruction, where the denormal-preserving form takes four.
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+// 16 bytes of logits: the largest element and the N values as floats.  Elements at or beyond `w`
+// read as -inf (probability zero).  The row base is 16-byte aligned.
+__device__ __forceinline__ void unpack(const uint4& raw, float (&v)[4], const float*) {
+  v[0] = __uint_as_float(raw.x); v[1] = __uint_as_float(raw.y);
+  v[2] = __uint_as_float(raw.z); v[3] = __uint_as_float(raw.w);
+}
+__device__ __forceinline__ void unpack(const uint4& raw, float (&v)[8], const __half*) {
+  const __half2* h = reinterpret_cast<const __half2*>(&raw);
+#pragma unroll
+  for (int k = 0; k < 4; ++k) { float2 f = __half22float2(h[k]); v[2 * k] = f.x; v[2 * k + 1] = f.y; }
+}
+__device__ __forceinline__ void unpack(const uint4& raw, float (&v)[8], const __nv_bfloat16*) {
+  const uint32_t u[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+  for (int k = 0; k < 4; ++k) { v[2 * k] = __uint_as_float(u[k] << 16); v[2 * k + 1] = __uint_as_float(u[k] & 0xffff0000u); }
+}
+__device__ __forceinline__ float vec_max(const uint4& raw, const float*) {
+  return fmaxf(fmaxf(__uint_as_float(raw.x), __uint_as_float(raw.y)),
+               fmaxf(__uint_as_float(raw.z), __uint_as_float(raw.w)));
+}
+__device__ __forceinline__ float vec_max(const uint4& raw, const __half*) {
+  const __half2* h = reinterpret_cast<const __half2*>(&raw);
+  __half2 m = __hmax2(__hmax2(h[0], h[1]), __hmax2(h[2], h[3]));       // exact: a maximum rounds nothing
+  return __half2float(__hmax(__low2half(m), __high2half(m)));
+}
+__device__ __forceinline__ float vec_max(const uint4& raw, const __nv_bfloat16*) {
+  const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&raw);
+  __nv_bfloat162 m = __hmax2(__hmax2(h[0], h[1]), __hmax2(h[2], h[3]));
+  return __bfloat162float(__hmax(__low2bfloat16(m), __high2bfloat16(m)));
+}
+
+// The N consecutive logits that start at element `i` (a multiple of N) of `row`, as raw bits; the
+// tail vector of a row whose length is not a multiple of N is completed with -inf.
+template <typename T>
+__device__ __forceinline__ uint4 load_raw(const T* __restrict__ row, int i, int w) {
+  constexpr int N = Vec<T>::N;
+  if (i + N <= w) return *reinterpret_cast<const uint4*>(row + i);
+  T e[N];
+#pragma unroll
+  for (int k = 0; k < N; ++k) e[k] = i + k < w ? row[i + k] : (T)(-INFINITY);
+  return *reinterpret_cast<const uint4*>(e);
+}
 template <typename T>
 __device__ __forceinline__ void load_vec(const T* __restrict__ row, int i, int w, float (&v)[Vec<T>::N]) {
-  constexpr int N = Vec<T>::N;
-  if (i + N <= w) {
-    uint4 raw = *reinterpret_cast<const uint4*>(row + i);
-    const T* e = reinterpret_cast<const T*>(&raw);
-#pragma unroll
-    for (int k = 0; k < N; ++k) v[k] = cvt(e[k]);
-  } else {
-#pragma unroll
-    for (int k = 0; k < N; ++k) v[k] = i + k < w ? cvt(row[i + k]) : -INFINITY;
-  }
+  unpack(load_raw(row, i, w), v, (const T*)nullptr);
 }
 
 // Running (max, sum of exp(z - max)) pair of a softmax denominator.
 struct MaxSum {
   float m, s;
-  __device__ __forceinline__ void add(float z) {
-    if (z > m) { s = s * __expf(m - z) + 1.f; m = z; }
-    else s += __expf(z - m);
-  }
   __device__ __forceinline__ void merge(const MaxSum& o) {
     if (o.m > m) { s = s * __expf(m - o.m) + o.s; m = o.m; }
     else if (o.m > -INFINITY) s += o.s * __expf(o.m - m);
@@ -65,12 +102,10 @@ __device__ __forceinline__ MaxSum shfl_xor(const MaxSum& a, int o) {
   return r;
 }
 
-// Probability of one logit given the row maximum and the reciprocal denominator.  The product is
-// rounded on its own (no fused multiply-add with the subtraction that follows), so that identical
-// draft and target rows give a residual of exactly zero.
-__device__ __forceinline__ float prob(float z, float zmax, float inv_sum) {
-  return __fmul_rn(__expf(z - zmax), inv_sum);
-}
+// Probability of one logit: 2^(z log2(e) - c) with c = log2(e) max + log2(sum of exp(z - max)), one
+// fused multiply-add and one special-function instruction.  Draft and target rows go through the
+// same instructions, so identical rows give a residual of exactly zero.
+__device__ __forceinline__ float prob(float z, float neg_c) { return ex2(fmaf(z, kLog2e, neg_c)); }
 
 // Two largest values of a multiset.
 struct Top2 {
@@ -97,31 +132,40 @@ correct_kernel(const T* __restrict__ zd, const T* __restrict__ zt, long long ldz
   const int row = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const T* rd = zd + (size_t)row * ldz;
   const T* rt = zt + (size_t)row * ldz;
+  const T* const tag = nullptr;
   // contiguous segment of this warp, in whole vectors
   const int nvec = (w + N - 1) / N;
   const int vec_per_warp = (nvec + kWarps - 1) / kWarps;
   const int v0 = warp * vec_per_warp, v1 = min(nvec, v0 + vec_per_warp);
 
   // ---- sweep 1: softmax denominators of both rows (Eq. 2, 4), two largest draft logits (Eq. 16) ----
+  // The sums run relative to the largest logit seen so far by this thread, in the base-2 domain:
+  // exp(z - m) = 2^(z log2(e) - m log2(e)).
   MaxSum md{-INFINITY, 0.f}, mt{-INFINITY, 0.f};
+  float nd = 0.f, nt = 0.f;                     // -m log2(e) of the two running maxima
   Top2 top{-INFINITY, -INFINITY};
 #pragma unroll 2
   for (int v = v0 + lane; v < v1; v += 32) {
-    float a[N], b[N];
-    load_vec(rd, v * N, w, a);
-    load_vec(rt, v * N, w, b);
+    const uint4 ra = load_raw(rd, v * N, w), rb = load_raw(rt, v * N, w);
     // one rescale per vector: every vector holds at least one element of the vocabulary, so its
-    // maximum is finite and exp(-inf - max) = 0 takes care of the padding
-    float va = a[0], vb = b[0];
-#pragma unroll
-    for (int k = 1; k < N; ++k) { va = fmaxf(va, a[k]); vb = fmaxf(vb, b[k]); }
-    if (va > md.m) { md.s *= __expf(md.m - va); md.m = va; }
-    if (vb > mt.m) { mt.s *= __expf(mt.m - vb); mt.m = vb; }
+    // maximum is finite and 2^(-inf) = 0 takes care of the padding
+    const float va = vec_max(ra, tag), vb = vec_max(rb, tag);
+    if (va > md.m) { md.s *= __expf(md.m - va); md.m = va; nd = -va * kLog2e; }
+    if (vb > mt.m) { mt.s *= __expf(mt.m - vb); mt.m = vb; nt = -vb * kLog2e; }
+    float a[N], b[N];
+    unpack(ra, a, tag);
+    unpack(rb, b, tag);
+    float sa = 0.f, sb = 0.f;
 #pragma unroll
     for (int k = 0; k < N; ++k) {
-      md.s += __expf(a[k] - md.m);
-      mt.s += __expf(b[k] - mt.m);
-      top.add(a[k]);
+      sa += ex2(fmaf(a[k], kLog2e, nd));
+      sb += ex2(fmaf(b[k], kLog2e, nt));
+    }
+    md.s += sa;
+    mt.s += sb;
+    if (va > top.b) {                           // rare once a few vectors have been seen
+#pragma unroll
+      for (int k = 0; k < N; ++k) top.add(a[k]);
     }
   }
 #pragma unroll
@@ -144,7 +188,9 @@ correct_kernel(const T* __restrict__ zd, const T* __restrict__ zt, long long ldz
       top.merge(other);
     }
     if (lane == 0) {
-      bc[0] = md.m; bc[1] = 1.f / md.s; bc[2] = mt.m; bc[3] = 1.f / mt.s;
+      // exponent offsets of the two distributions: p = 2^(z log2(e) + bc)
+      bc[0] = -(md.m * kLog2e + log2f(md.s));
+      bc[1] = -(mt.m * kLog2e + log2f(mt.s));
       float m = (1.f - (top.b > -INFINITY ? __expf(top.b - top.a) : 0.f)) * __expf(top.a - md.m) / md.s;
       margin[row] = m;
       gate[row] = m < gamma ? 1 : 0;                                       // Eq. 17
@@ -160,21 +206,30 @@ correct_kernel(const T* __restrict__ zd, const T* __restrict__ zt, long long ldz
     }
   }
   __syncthreads();
-  const float max_d = bc[0], inv_d = bc[1], max_t = bc[2], inv_t = bc[3];
+  const float cd = bc[0], ct = bc[1];
 
   // ---- sweep 2: residual mass per warp segment (Eq. 6 denominator) ----
   // use_pt: the residual is identically zero (the two distributions coincide): draw from p_t.
   for (int use_pt = 0; use_pt < 2; ++use_pt) {
     float part = 0.f;
+    if (!use_pt) {
 #pragma unroll 2
-    for (int v = v0 + lane; v < v1; v += 32) {
-      float a[N], b[N];
-      load_vec(rd, v * N, w, a);
-      load_vec(rt, v * N, w, b);
+      for (int v = v0 + lane; v < v1; v += 32) {
+        float a[N], b[N];
+        const uint4 ra = load_raw(rd, v * N, w), rb = load_raw(rt, v * N, w);
+        unpack(ra, a, tag);
+        unpack(rb, b, tag);
+        float acc = 0.f;
 #pragma unroll
-      for (int k = 0; k < N; ++k) {
-        float pt = prob(b[k], max_t, inv_t), pd = prob(a[k], max_d, inv_d);
-        part += use_pt ? pt : fmaxf(pt - pd, 0.f);
+        for (int k = 0; k < N; ++k) acc += fmaxf(prob(b[k], ct) - prob(a[k], cd), 0.f);
+        part += acc;
+      }
+    } else {
+      for (int v = v0 + lane; v < v1; v += 32) {
+        float b[N];
+        load_vec(rt, v * N, w, b);
+#pragma unroll
+        for (int k = 0; k < N; ++k) part += prob(b[k], ct);
       }
     }
     part = warp_sum(part);
@@ -215,7 +270,7 @@ correct_kernel(const T* __restrict__ zd, const T* __restrict__ zt, long long ldz
             load_vec(rt, v * N, w, b);
 #pragma unroll
             for (int k = 0; k < N; ++k) {
-              float pt = prob(b[k], max_t, inv_t), pd = prob(a[k], max_d, inv_d);
+              float pt = prob(b[k], ct), pd = prob(a[k], cd);
               r[k] = use_pt ? pt : fmaxf(pt - pd, 0.f);
               lsum += r[k];
             }
@@ -254,7 +309,7 @@ correct_kernel(const T* __restrict__ zd, const T* __restrict__ zt, long long ldz
           // the chosen segment held no positive entry at all (possible only through rounding):
           // scan back for the last positive probability in the whole row
           for (int i = w - 1; i >= 0 && tk < 0; --i) {
-            float pt = prob(cvt(rt[i]), max_t, inv_t), pd = prob(cvt(rd[i]), max_d, inv_d);
+            float pt = prob(cvt(rt[i]), ct), pd = prob(cvt(rd[i]), cd);
             if ((use_pt ? pt : pt - pd) > 0.f) tk = i;
           }
         }

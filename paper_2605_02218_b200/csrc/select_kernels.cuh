@@ -49,6 +49,46 @@ __device__ __forceinline__ unsigned block_exclusive_scan(unsigned v, unsigned* w
 // are taken.  out[0..k) receives the selected positions in ascending order, mapped through `remap`
 // when given.  `all_equal` treats every key as equal (selects the first k positions).
 constexpr int kRankSelectMax = 1024;   // up to this many keys the selection ranks every key directly
+constexpr int kRegKeys = 16;           // keys per thread the radix select keeps in registers
+
+// One digit of the radix select, by the first warp: with `kk` keys still to take among those that
+// match the digits fixed so far, the largest digit value d such that the keys with a larger digit
+// number fewer than kk (digit 0 when none does); *sel_k = kk minus those keys.  Lane l sums the
+// eight histogram bins 8 l .. 8 l + 7; a suffix scan over the lanes finds the lane that holds d.
+__device__ __forceinline__ void select_digit(const unsigned* hist, unsigned kk, unsigned prefix, int shift,
+                                             unsigned* sel_prefix, unsigned* sel_k) {
+  const int lane = threadIdx.x & 31;
+  if (kk == 0u) {                             // nothing left to take: no key is above the top digit
+    if (lane == 0) { *sel_prefix = prefix | (255u << shift); *sel_k = 0u; }
+    return;
+  }
+  unsigned h[8], mine = 0u;
+#pragma unroll
+  for (int e = 0; e < 8; ++e) { h[e] = hist[8 * lane + e]; mine += h[e]; }
+  unsigned above = mine;                      // inclusive suffix sum over lanes >= this one
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    unsigned t = __shfl_down_sync(0xffffffffu, above, o);
+    if (lane + o < 32) above += t;
+  }
+  above -= mine;                              // keys in the bins of higher lanes
+  const unsigned holds = __ballot_sync(0xffffffffu, above < kk && above + mine >= kk);
+  const int owner = holds ? 31 - __clz(holds) : 0;
+  if (lane == owner) {
+    unsigned c = above;
+    int e = 7;
+    for (; e > 0; --e) {
+      if (c + h[e] >= kk) break;
+      c += h[e];
+    }
+    if (!holds) {                             // fewer matching keys than kk: digit 0 takes the rest
+      e = 0;
+      c = above + mine - h[0];
+    }
+    *sel_prefix = prefix | ((unsigned)(8 * lane + e) << shift);
+    *sel_k = kk - c;
+  }
+}
 
 // `load(i)` returns key i as a float; `status` may be nullptr (non-finite keys are then not reported).
 template <typename LoadF>
@@ -90,6 +130,57 @@ __device__ void block_topk_by(LoadF load, int n, int k, bool all_equal,
     return;
   }
   unsigned prefix = 0u, mask = 0u, kk = (unsigned)k;
+  const int per = (n + (int)blockDim.x - 1) / (int)blockDim.x;
+  if (per <= kRegKeys) {
+    // Medium segments: every thread keeps a contiguous run of `per` keys in registers, so the four
+    // digit passes read nothing from memory and the ordered emission needs one block scan.
+    unsigned kreg[kRegKeys];
+    const int i0 = (int)threadIdx.x * per;
+    const int cnt = max(0, min(per, n - i0));
+    bool bad = false;
+#pragma unroll
+    for (int j = 0; j < kRegKeys; ++j) {
+      kreg[j] = 0u;
+      if (j < cnt && !all_equal) {
+        float v = load(i0 + j);
+        bad |= !(fabsf(v) <= 3.402823466e38f);
+        kreg[j] = order_key(v);
+      }
+    }
+    if (bad && status != nullptr) atomicOr(status, kStatusNonFinite);
+    if (!all_equal) {
+      for (int shift = 24; shift >= 0; shift -= 8) {
+        for (int i = threadIdx.x; i < 256; i += blockDim.x) hist[i] = 0u;
+        __syncthreads();
+#pragma unroll
+        for (int j = 0; j < kRegKeys; ++j)
+          if (j < cnt && (kreg[j] & mask) == prefix) atomicAdd(&hist[(kreg[j] >> shift) & 255u], 1u);
+        __syncthreads();
+        if (threadIdx.x < 32) select_digit(hist, kk, prefix, shift, &sel_prefix, &sel_k);
+        __syncthreads();
+        prefix = sel_prefix;
+        kk = sel_k;
+        mask |= 255u << shift;
+      }
+    }
+    unsigned gt = 0u, eq = 0u;
+#pragma unroll
+    for (int j = 0; j < kRegKeys; ++j)
+      if (j < cnt) { gt += kreg[j] > prefix; eq += kreg[j] == prefix; }
+    unsigned tot;
+    unsigned ex = block_exclusive_scan(gt | (eq << 16), warp_tot, &tot);
+    unsigned gt_before = ex & 0xffffu, eq_before = ex >> 16;
+#pragma unroll
+    for (int j = 0; j < kRegKeys; ++j) {
+      if (j < cnt) {
+        const bool g = kreg[j] > prefix, e = kreg[j] == prefix;
+        if (g || (e && eq_before < kk)) out[gt_before + min(eq_before, kk)] = remap ? remap[i0 + j] : i0 + j;
+        gt_before += g;
+        eq_before += e;
+      }
+    }
+    return;
+  }
   if (!all_equal) {
     bool bad = false;
     for (int shift = 24; shift >= 0; shift -= 8) {
@@ -102,16 +193,7 @@ __device__ void block_topk_by(LoadF load, int n, int k, bool all_equal,
         if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
       }
       __syncthreads();
-      if (threadIdx.x == 0) {
-        unsigned c = 0u;
-        int bin = 255;
-        for (; bin > 0; --bin) {
-          if (c + hist[bin] >= kk) break;
-          c += hist[bin];
-        }
-        sel_prefix = prefix | ((unsigned)bin << shift);
-        sel_k = kk - c;
-      }
+      if (threadIdx.x < 32) select_digit(hist, kk, prefix, shift, &sel_prefix, &sel_k);
       __syncthreads();
       prefix = sel_prefix;
       kk = sel_k;
