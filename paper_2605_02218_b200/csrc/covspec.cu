@@ -651,8 +651,8 @@ int select_impl(covspec_ctx* ctx, const covspec_problem* p, const float* s_fused
   if (pl.n_stage2 > 0) {
     prof_mark(ctx, ST_GRAM, 0, s);
     int vec16 = cfg.d * ctx->esize / 16;
-    gather_rows_kernel<<<(unsigned)pl.total_presel, 256, 0, s>>>(
-        reinterpret_cast<const uint4*>(p->X), presel, ctx->d_plan, B, 1, vec16,
+    gather_rows_kernel<<<gather_grid(pl.total_presel), kGatherWarps * 32, 0, s>>>(
+        reinterpret_cast<const uint4*>(p->X), presel, ctx->d_plan, B, 1, vec16, (int)pl.total_presel,
         reinterpret_cast<uint4*>(ctx->Zg), nullptr);
     LAUNCH_CHECK(ctx);
     int st;
@@ -720,8 +720,8 @@ int compact_impl(covspec_ctx* ctx, const covspec_problem* p, const int* keep_idx
                  int* out_pos, cudaStream_t s) {
   const Plan& pl = ctx->plan;
   int vec16 = ctx->cfg.d * ctx->esize / 16;
-  gather_rows_kernel<<<(unsigned)pl.total_keep, 256, 0, s>>>(
-      reinterpret_cast<const uint4*>(p->X), keep_idx, ctx->d_plan, p->batch, 0, vec16,
+  gather_rows_kernel<<<gather_grid(pl.total_keep), kGatherWarps * 32, 0, s>>>(
+      reinterpret_cast<const uint4*>(p->X), keep_idx, ctx->d_plan, p->batch, 0, vec16, (int)pl.total_keep,
       reinterpret_cast<uint4*>(out), out_pos);
   LAUNCH_CHECK(ctx);
   prof_mark(ctx, ST_FINAL, 1, s);
@@ -1011,9 +1011,9 @@ int covspec_compact_rows(covspec_ctx* ctx, const covspec_problem* p, const int* 
   if (st) return st;
   if (memcmp(keep_offsets, ctx->plan.keep_offsets.data(), sizeof(int) * (p->batch + 1)))
     return COVSPEC_ERR_SHAPE;
-  gather_rows_kernel<<<(unsigned)ctx->plan.total_keep, 256, 0, s>>>(
+  gather_rows_kernel<<<gather_grid(ctx->plan.total_keep), kGatherWarps * 32, 0, s>>>(
       reinterpret_cast<const uint4*>(src), keep_idx, ctx->d_plan, p->batch, 0, (int)(row_bytes / 16),
-      reinterpret_cast<uint4*>(out), nullptr);
+      (int)ctx->plan.total_keep, reinterpret_cast<uint4*>(out), nullptr);
   LAUNCH_CHECK(ctx);
   return COVSPEC_OK;
 }

@@ -95,6 +95,7 @@ template <typename LoadF>
 __device__ void block_topk_by(LoadF load, int n, int k, bool all_equal,
                               const int* __restrict__ remap, int* __restrict__ out, int* status) {
   __shared__ unsigned hist[256];
+  __shared__ unsigned whist[8][256];
   __shared__ unsigned sel_prefix, sel_k;
   __shared__ unsigned warp_tot[33];
   __shared__ unsigned skeys[kRankSelectMax];
@@ -150,11 +151,21 @@ __device__ void block_topk_by(LoadF load, int n, int k, bool all_equal,
     if (bad && status != nullptr) atomicOr(status, kStatusNonFinite);
     if (!all_equal) {
       for (int shift = 24; shift >= 0; shift -= 8) {
-        for (int i = threadIdx.x; i < 256; i += blockDim.x) hist[i] = 0u;
+        // scores of one request crowd into a few digit values: eight copies of the histogram
+        // (one per warp modulo 8) spread the same-address updates
+        for (int i = threadIdx.x; i < 8 * 256; i += blockDim.x) (&whist[0][0])[i] = 0u;
         __syncthreads();
+        unsigned* myhist = whist[(threadIdx.x >> 5) & 7];
 #pragma unroll
         for (int j = 0; j < kRegKeys; ++j)
-          if (j < cnt && (kreg[j] & mask) == prefix) atomicAdd(&hist[(kreg[j] >> shift) & 255u], 1u);
+          if (j < cnt && (kreg[j] & mask) == prefix) atomicAdd(&myhist[(kreg[j] >> shift) & 255u], 1u);
+        __syncthreads();
+        for (int i = threadIdx.x; i < 256; i += blockDim.x) {
+          unsigned c = 0u;
+#pragma unroll
+          for (int q = 0; q < 8; ++q) c += whist[q][i];
+          hist[i] = c;
+        }
         __syncthreads();
         if (threadIdx.x < 32) select_digit(hist, kk, prefix, shift, &sel_prefix, &sel_k);
         __syncthreads();
@@ -262,21 +273,38 @@ final_select_kernel(const float* __restrict__ energy, const int* __restrict__ pr
              keep_idx + rp.keep_off, status);
 }
 
-// out[row, :] = src[vis_off(b) + idx[row], :] as 16-byte vectors; one block per output row.
+// out[row, :] = src[vis_off(b) + idx[row], :] as 16-byte vectors; one warp per output row (its
+// first lane looks the request up), four vectors per lane in flight.
 // `use_presel` selects which plan offsets delimit the rows of a request (presel_off / keep_off).
-__global__ void __launch_bounds__(256)
+constexpr int kGatherWarps = 8;
+__global__ void __launch_bounds__(kGatherWarps * 32)
 gather_rows_kernel(const uint4* __restrict__ src, const int* __restrict__ idx,
-                   const ReqPlan* __restrict__ plan, int batch, int use_presel, int row_vec16,
+                   const ReqPlan* __restrict__ plan, int batch, int use_presel, int row_vec16, int rows,
                    uint4* __restrict__ dst, int* __restrict__ out_pos) {
-  int row = blockIdx.x;
-  int b = find_request(row, batch, [&](int q) {
-    return use_presel ? plan[q].presel_off : plan[q].keep_off;
-  });
-  int tok = idx[row];
-  const uint4* s = src + ((size_t)plan[b].vis_off + tok) * row_vec16;
+  const int lane = threadIdx.x & 31;
+  const int row = blockIdx.x * kGatherWarps + (threadIdx.x >> 5);
+  if (row >= rows) return;
+  long long first = 0;
+  int tok = 0;
+  if (lane == 0) {
+    int b = find_request(row, batch, [&](int q) {
+      return use_presel ? plan[q].presel_off : plan[q].keep_off;
+    });
+    tok = idx[row];
+    first = (long long)plan[b].vis_off + tok;
+    if (out_pos != nullptr) out_pos[row] = tok;
+  }
+  first = __shfl_sync(0xffffffffu, first, 0);
+  const uint4* s = src + (size_t)first * row_vec16;
   uint4* d = dst + (size_t)row * row_vec16;
-  for (int v = threadIdx.x; v < row_vec16; v += blockDim.x) d[v] = s[v];
-  if (out_pos != nullptr && threadIdx.x == 0) out_pos[row] = tok;
+  int v = lane;
+  for (; v + 96 < row_vec16; v += 128) {
+    uint4 a = __ldg(s + v), b2 = __ldg(s + v + 32), c = __ldg(s + v + 64), e = __ldg(s + v + 96);
+    d[v] = a; d[v + 32] = b2; d[v + 64] = c; d[v + 96] = e;
+  }
+  for (; v < row_vec16; v += 32) d[v] = __ldg(s + v);
 }
+
+inline unsigned gather_grid(long long rows) { return (unsigned)((rows + kGatherWarps - 1) / kGatherWarps); }
 
 }  // namespace covspec
