@@ -690,6 +690,7 @@ int select_impl(covspec_ctx* ctx, const covspec_problem* p, const float* s_fused
     // energies: one cooperative launch (its CTAs wait on one another through global counters)
     sub::FusedParams fp{};
     fp.plan = ctx->d_plan; fp.batch = B; fp.n_items = pl.n_ptiles; fp.sched = ctx->d_sched;
+    fp.spread_sum = pl.n_ptiles <= pl.pow_grid ? 1 : 0;      // one tile per CTA (see the schedule above)
     fp.steps = cfg.eig_iters + 1;
     fp.lbuf = ctx->Lbuf;
     for (int i = 0; i < 2; ++i) { fp.y_hi[i] = ctx->Yp[i][0]; fp.y_lo[i] = ctx->Yp[i][1]; fp.yf[i] = ctx->Yf[i]; }

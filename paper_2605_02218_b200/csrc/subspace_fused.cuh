@@ -29,7 +29,7 @@
 namespace covspec {
 namespace sub {
 
-constexpr int kSyncStride = 4;           // unsigned words per request: arrive, factor, ritz, last
+constexpr int kSyncStride = 8;           // unsigned words per request: arrive, factor, ritz, last, summed
 
 struct FusedParams {
   const ReqPlan* plan;
@@ -47,6 +47,7 @@ struct FusedParams {
   float* ub;                // [batch][kPMax * kPMax] Ritz vectors of the discarded pairs
   float* energy;            // [sum M_b] (out)
   unsigned* sync;           // [batch][kSyncStride] counters (zero on entry), then the abort word
+  int spread_sum;           // every CTA holds exactly one tile: the tiles of a request sum the partial matrices together
   int max_sweeps;
   float conv_tol;           // bound on the estimated energy error before NOCONVERGE is raised
   int early_stop;           // 1: requests whose estimate is far below conv_tol stop before `steps`
@@ -944,7 +945,41 @@ subspace_kernel(const __grid_constant__ CUtensorMap map_gh, const __grid_constan
         __threadfence();
         fence_proxy_async_all();
         epi_sync();
-        if (et == 0) {
+        int nt_sum = (int)nt;                        // partial matrices the factoring tile has to add up
+        if (prm.spread_sum && nt >= 4) {             // with fewer tiles the extra round trip costs more than it saves
+          // Every CTA holds one tile, so all tiles of the request are being worked on at the same
+          // time: instead of leaving the sum of the partial matrices to the last tile alone, every
+          // tile waits for the others and adds up its own slice of the matrix (in tile order, into
+          // the slot of tile 0); the last one to finish its slice factors the summed matrix.
+          if (et == 0) atomicAdd(sync_b, 1u);
+          ok = team_wait(sync_b, nt * (unsigned)(step + 1)) && ok;
+          double* sum0 = prm.partial + (size_t)rp.ptile_off * kTileDoubles;
+          const int used = (P >> 3) * ((P >> 3) + 1) / 2 * 64;
+          const int chunk = ((used + (int)nt - 1) / (int)nt + 1) & ~1;
+          const int e1 = min(used, (tile + 1) * chunk);
+          if (ok) {
+            for (int e = tile * chunk + 2 * et; e < e1; e += 2 * kEpiThreads) {
+              double2 acc = make_double2(0.0, 0.0);
+              for (int t0 = 0; t0 < (int)nt; t0 += 8) {
+                double2 v[8];
+#pragma unroll
+                for (int q = 0; q < 8; ++q)
+                  v[q] = __ldcg(reinterpret_cast<const double2*>(sum0 + (size_t)min(t0 + q, (int)nt - 1) * kTileDoubles + e));
+#pragma unroll
+                for (int q = 0; q < 8; ++q)
+                  if (t0 + q < (int)nt) { acc.x += v[q].x; acc.y += v[q].y; }
+              }
+              *reinterpret_cast<double2*>(sum0 + e) = acc;
+            }
+          }
+          __threadfence();
+          epi_sync();
+          if (et == 0) {
+            unsigned old = atomicAdd(sync_b + 4, 1u);
+            *s_word = (old + 1u == nt * (unsigned)(step + 1) && !*abort_flag) ? 1 : 0;
+          }
+          nt_sum = 1;
+        } else if (et == 0) {
           unsigned old = atomicAdd(sync_b, 1u);
           // one decision for the whole team (a CTA that has given up factors nothing)
           *s_word = (old + 1u == nt * (unsigned)(step + 1) && !*abort_flag) ? 1 : 0;
@@ -961,7 +996,7 @@ subspace_kernel(const __grid_constant__ CUtensorMap map_gh, const __grid_constan
             // the basis is still mixing)
             const bool may_stop = prm.early_stop && step >= 1 && step + 1 < last_b && p < rp.m;
             const float margin = step == 1 ? 0.015625f : 0.125f;
-            const bool stop = team_cholesky(pbase, (int)nt, p, rp.r, prm.lbuf + (size_t)b * kLbufStride, Tm, dinv,
+            const bool stop = team_cholesky(pbase, nt_sum, p, rp.r, prm.lbuf + (size_t)b * kLbufStride, Tm, dinv,
                                             s_word, step + 2, may_stop ? margin * prm.conv_tol : 0.f);
             __threadfence();
             epi_sync();
@@ -970,7 +1005,7 @@ subspace_kernel(const __grid_constant__ CUtensorMap map_gh, const __grid_constan
               st_release_u32(sync_b + 1, (unsigned)(step + 1));
             }
           } else {
-            team_ritz(pbase, (int)nt, p, rp.win, rp.r, rp.m, prm.ub + (size_t)b * kPMax * kPMax, reinterpret_cast<float*>(smem), lt,
+            team_ritz(pbase, nt_sum, p, rp.win, rp.r, rp.m, prm.ub + (size_t)b * kPMax * kPMax, reinterpret_cast<float*>(smem), lt,
                       s_scale, s_flag, prm.max_sweeps, prm.conv_tol, step + 1, prm.status);
             __threadfence();
             epi_sync();

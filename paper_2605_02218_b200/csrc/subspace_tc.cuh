@@ -249,8 +249,8 @@ basis_init_kernel(const ReqPlan* __restrict__ plan, __nv_bfloat16* __restrict__ 
                   unsigned* __restrict__ sync, int batch, int last_step) {
   ReqPlan rp = plan[blockIdx.y];
   if (blockIdx.x == 0) {
-    if (threadIdx.x < 4) sync[blockIdx.y * 4 + threadIdx.x] = threadIdx.x == 3 ? (unsigned)last_step : 0u;
-    if (blockIdx.y == 0 && threadIdx.x >= 32 && threadIdx.x < 36) sync[batch * 4 + threadIdx.x - 32] = 0u;
+    if (threadIdx.x < 8) sync[blockIdx.y * 8 + threadIdx.x] = threadIdx.x == 3 ? (unsigned)last_step : 0u;
+    if (blockIdx.y == 0 && threadIdx.x >= 32 && threadIdx.x < 36) sync[batch * 8 + threadIdx.x - 32] = 0u;
     if (!rp.stage2)
       for (int i = threadIdx.x; i < rp.m; i += blockDim.x) energy[rp.presel_off + i] = 0.f;
   }
