@@ -1126,15 +1126,15 @@ int covspec_correct(int logit_dtype, int rows, int vocab, long long ld, const vo
   if ((reinterpret_cast<uintptr_t>(z_draft) | reinterpret_cast<uintptr_t>(z_target)) & 15) return COVSPEC_ERR_ARG;
   cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
   if (logit_dtype == COVSPEC_F32)
-    corr::correct_kernel<float><<<rows, corr::kThreads, 0, s>>>(
+    corr::correct_kernel<float><<<rows * corr::kClusterCtas, corr::kThreads, 0, s>>>(
         static_cast<const float*>(z_draft), static_cast<const float*>(z_target), ld, vocab, drafted,
         uniforms, gamma, margin, gate, accept, resid_mass, token);
   else if (logit_dtype == COVSPEC_BF16)
-    corr::correct_kernel<__nv_bfloat16><<<rows, corr::kThreads, 0, s>>>(
+    corr::correct_kernel<__nv_bfloat16><<<rows * corr::kClusterCtas, corr::kThreads, 0, s>>>(
         static_cast<const __nv_bfloat16*>(z_draft), static_cast<const __nv_bfloat16*>(z_target), ld,
         vocab, drafted, uniforms, gamma, margin, gate, accept, resid_mass, token);
   else
-    corr::correct_kernel<__half><<<rows, corr::kThreads, 0, s>>>(
+    corr::correct_kernel<__half><<<rows * corr::kClusterCtas, corr::kThreads, 0, s>>>(
         static_cast<const __half*>(z_draft), static_cast<const __half*>(z_target), ld, vocab, drafted,
         uniforms, gamma, margin, gate, accept, resid_mass, token);
   CUDA_TRY(cudaGetLastError());
