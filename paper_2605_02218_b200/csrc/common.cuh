@@ -23,7 +23,7 @@ struct ReqPlan {
   int stage2;              // 1 when b_vis < m (Eq. 13-15 are evaluated)
   int tile_off;            // first 128-token tile of the request in the tensor-core relevance kernel
   int pair_off;            // first pair of 128-token tiles of the request (two-SM relevance kernel)
-  int gram_tile_off;       // first lower-triangle 128 x 128 tile of the request's Gram matrix
+  int gram_tile_off;       // first lower-triangle 128 x 256 item of the request's Gram matrix
   int ptile_off;           // first 128-row tile of the request's subspace-iteration block
   int win;                 // basis vectors in the Rayleigh-Ritz window next to the cut at r
   long long g_off;         // float offset of the request's float32 Gram matrix (float32 inputs only)

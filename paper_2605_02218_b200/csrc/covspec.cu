@@ -104,7 +104,7 @@ struct covspec_ctx {
   unsigned* sync = nullptr;              // per-request counters of the fused subspace kernel + abort word
   float* Cg = nullptr;                   // factor columns of the greedy low-rank mode
   long long cg_cap = 0;
-  CUtensorMap map_zg, map_gh, map_gl, map_y[2][2];
+  CUtensorMap map_zg, map_zgw, map_gh, map_gl, map_y[2][2];
   // pinned staging for the plan upload
   char* h_stage = nullptr;
   long long stage_bytes = 0, stage_sched_off = 0;
@@ -230,7 +230,7 @@ int get_plan(covspec_ctx* ctx, const covspec_problem* p, cudaStream_t stream) {
       if (r.p > r.m) r.p = r.m;
       ++pl.n_stage2;
       int nt = (r.m + sub::kTile - 1) / sub::kTile;
-      pl.n_gram_tiles += nt * (nt + 1) / 2;
+      pl.n_gram_tiles += sub::gram_items(nt);
       pl.n_ptiles += nt;
       if (f32) g_off += (long long)r.m * r.ldm;
       if (cfg.lowrank_mode == 1) {
@@ -663,7 +663,7 @@ int select_impl(covspec_ctx* ctx, const covspec_problem* p, const float* s_fused
       gp.k_chunks = (cfg.d + sub::kBK - 1) / sub::kBK;
       gp.g_hi = ctx->Ghi; gp.g_lo = ctx->Glo; gp.ld = ctx->ld; gp.status = ctx->status;
       int grid = std::min(pl.n_gram_tiles, ctx->num_sms);
-      sub::gram_tc_kernel<<<grid, 192, sub::kGramSmem, s>>>(ctx->map_zg, gp);
+      sub::gram_tc_kernel<<<grid, 192, sub::kGramSmem, s>>>(ctx->map_zg, ctx->map_zgw, gp);
       LAUNCH_CHECK(ctx);
     } else {
       if ((st = launch_table<T, T, float, float, false>(ctx, T_GRAM_G, 1, s))) return st;
@@ -931,6 +931,7 @@ int covspec_prune_init(const covspec_config* cfg, covspec_ctx** out) {
     // tensor maps over the workspace arrays of the subspace iteration (fixed for the context)
     int st = COVSPEC_OK;
     if (!f32) st = make_map_bf16(&ctx->map_zg, ctx->Zg, c.max_total_presel, c.d, sub::kTile);
+    if (!f32 && !st) st = make_map_bf16(&ctx->map_zgw, ctx->Zg, c.max_total_presel, c.d, sub::kGramN);
     if (!st) st = make_map_bf16(&ctx->map_gh, ctx->Ghi, ctx->cap_rows, ctx->ld, sub::kTile);
     if (!st) st = make_map_bf16(&ctx->map_gl, ctx->Glo, ctx->cap_rows, ctx->ld, sub::kTile);
     for (int i = 0; i < 2 && !st; ++i)

@@ -60,10 +60,27 @@ __device__ __forceinline__ void tri_decode(int t, int& ti, int& tj) {
 // ================================================================================================
 // Gram kernel
 // ================================================================================================
-constexpr int kGramStages = 6;
-constexpr int kGramStageBytes = 2 * kTile * kBK * 2;     // A and B tile, 16 KB each
+// Items are 128 x 256 blocks of the lower triangle (row tile ti, pair of column tiles 2 tjp and
+// 2 tjp + 1, tjp <= ti / 2): per 64-element k-chunk a 16 KB row tile and a 32 KB column tile feed
+// 128 x 256 x 64 products, two thirds of the operand bytes per product a square 128 x 128 item
+// needs (the feed from L2 bounds this kernel).  The half of a block that lies above the diagonal
+// (ti even, last pair) is computed and dropped.
+constexpr int kGramStages = 4;
+constexpr int kGramN = 2 * kTile;                         // columns of an item
+constexpr int kGramBytesA = kTile * kBK * 2;              // 16 KB
+constexpr int kGramStageBytes = kGramBytesA + kGramN * kBK * 2;   // 48 KB
 constexpr int kGramSmem = kGramStages * kGramStageBytes + 1024 + 1024;
-constexpr int kGramTmemCols = 256;                        // two 128-column accumulators
+constexpr int kGramTmemCols = 512;                        // two 256-column accumulators
+// Items of a request with nt row tiles, and the decoding of an item index.
+__host__ __device__ __forceinline__ int gram_items(int nt) {
+  int a = nt >> 1;
+  return (nt & 1) ? (a + 1) * (a + 1) : a * (a + 1);
+}
+__device__ __forceinline__ void gram_decode(int t, int& ti, int& tjp) {
+  ti = 0;
+  for (int cnt = 1; t >= cnt; cnt = (ti >> 1) + 1) { t -= cnt; ++ti; }
+  tjp = t;
+}
 
 struct GramParams {
   const ReqPlan* plan;
@@ -77,7 +94,8 @@ struct GramParams {
 };
 
 __global__ void __launch_bounds__(192, 1)
-gram_tc_kernel(const __grid_constant__ CUtensorMap map_z,   // gathered rows [sum M_b, d] bf16
+gram_tc_kernel(const __grid_constant__ CUtensorMap map_z,   // gathered rows [sum M_b, d] bf16, 128-row boxes
+               const __grid_constant__ CUtensorMap map_zw,  // the same tensor, 256-row boxes
                const GramParams prm) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -102,10 +120,10 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap map_z,   // gathered rows [su
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
-  auto decode = [&](int item, ReqPlan& rp, int& ti, int& tj) {
+  auto decode = [&](int item, ReqPlan& rp, int& ti, int& tjp) {
     int b = find_request(item, prm.batch, [&](int q) { return prm.plan[q].gram_tile_off; });
     rp = prm.plan[b];
-    tri_decode(item - rp.gram_tile_off, ti, tj);
+    gram_decode(item - rp.gram_tile_off, ti, tjp);
   };
 
   if (warp == 4) {
@@ -121,14 +139,14 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap map_z,   // gathered rows [su
           mbar_expect_tx(&full[s], kGramStageBytes);
           uint32_t dst = smem_u32(smem + s * kGramStageBytes);
           tma_load_2d(dst, &map_z, kc * kBK, rp.presel_off + ti * kTile, &full[s]);
-          tma_load_2d(dst + kGramStageBytes / 2, &map_z, kc * kBK, rp.presel_off + tj * kTile, &full[s]);
+          tma_load_2d(dst + kGramBytesA, &map_zw, kc * kBK, rp.presel_off + tj * kGramN, &full[s]);
         }
       }
     }
     __syncwarp();
   } else if (warp == 5) {
     if (lane == 0) {
-      const uint32_t idesc = umma_idesc(kTile, kTile);
+      const uint32_t idesc = umma_idesc(kTile, kGramN);
       uint32_t it = 0, n = 0;
       bool ok = true;
       for (int item = blockIdx.x; item < prm.n_items && ok; item += gridDim.x, ++n) {
@@ -140,10 +158,10 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap map_z,   // gathered rows [su
           if (!(ok = mbar_wait(&full[s], (it / kGramStages) & 1u, abort_flag))) break;
           tc_fence_after();
           uint32_t a_addr = smem_u32(smem + s * kGramStageBytes);
-          uint64_t adesc = umma_desc(a_addr), bdesc = umma_desc(a_addr + kGramStageBytes / 2);
+          uint64_t adesc = umma_desc(a_addr), bdesc = umma_desc(a_addr + kGramBytesA);
 #pragma unroll
           for (int k = 0; k < kBK / 16; ++k)
-            umma_bf16(tmem_base + buf * kTile, adesc + 2 * k, bdesc + 2 * k, idesc, (kc | k) != 0);
+            umma_bf16(tmem_base + buf * kGramN, adesc + 2 * k, bdesc + 2 * k, idesc, (kc | k) != 0);
           umma_commit(&empty[s]);
         }
         if (!ok) break;
@@ -166,10 +184,12 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap map_z,   // gathered rows [su
       const bool row_ok = row < rp.m;
       const size_t ld = (size_t)prm.ld;
 #pragma unroll 1
-      for (int c4 = 0; c4 < 4; ++c4) {
+      for (int c4 = 0; c4 < 8; ++c4) {
+        const int tc = 2 * tj + (c4 >> 2);            // column tile of this group of 32 columns
+        if (tc > ti) break;                           // above the diagonal: dropped
         float v[32];
-        tmem_ld32(t_lane + buf * kTile + c4 * 32, v);
-        const int col0 = tj * kTile + c4 * 32;
+        tmem_ld32(t_lane + buf * kGramN + c4 * 32, v);
+        const int col0 = tj * kGramN + c4 * 32;
         // entries outside the request's M x M block are stored as zeros: the power step multiplies
         // whole 64-wide k-chunks and must not meet stale non-finite values in the padding
 #pragma unroll
@@ -192,7 +212,7 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap map_z,   // gathered rows [su
             dl[q] = make_uint4(pl[4 * q], pl[4 * q + 1], pl[4 * q + 2], pl[4 * q + 3]);
           }
         }
-        if (ti != tj && row < prm.ld) {
+        if (ti != tc && row < prm.ld) {
           // mirrored tile: G[col, row] = G[row, col]; consecutive threads write consecutive columns
           unsigned short* mh = reinterpret_cast<unsigned short*>(prm.g_hi);
           unsigned short* ml = reinterpret_cast<unsigned short*>(prm.g_lo);
