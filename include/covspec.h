@@ -96,9 +96,10 @@ typedef struct {
                           energy) and raises COVSPEC_ERR_NOCONVERGE in the device status word when the
                           estimate exceeds conv_tol (default 2e-3; 0 disables the check).  More steps
                           (eig_iters) or more extra vectors (eig_oversample) settle such inputs      */
-  int eig_early_stop;  /* 1 (default): a request whose estimate, predicted two steps ahead from the Ritz
-                          value estimates of the running iteration, is below conv_tol / 8 stops there
-                          instead of running all eig_iters steps; 0: always eig_iters steps           */
+  int eig_early_stop;  /* 1 (default): a request whose estimate, predicted for the next step from the Ritz
+                          value estimates of the running iteration, is below conv_tol / 8 (conv_tol / 64
+                          after the second multiplication) makes that step its last instead of running
+                          all eig_iters steps; 0: always eig_iters steps                              */
 } covspec_config;
 
 /* One batch of requests (Sec. III-A notation in brackets). */
