@@ -145,7 +145,7 @@ class ClockSampler:
     """Samples SM clock and throttle reasons through NVML (read-only) while the timed region runs."""
 
     def __init__(self, index):
-        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self.samples, self.reasons, self.max_mhz, self.mask = [], set(), None, 0
         self._stop = threading.Event()
         self._thread = None
         try:
@@ -164,11 +164,15 @@ class ClockSampler:
             "hw_thermal_slowdown": getattr(nv, "nvmlClocksThrottleReasonHwThermalSlowdown", 0x40),
             "sw_thermal_slowdown": getattr(nv, "nvmlClocksThrottleReasonSwThermalSlowdown", 0x20),
             "sw_power_cap": getattr(nv, "nvmlClocksThrottleReasonSwPowerCap", 0x4),
+            "applications_clocks_setting": getattr(nv, "nvmlClocksThrottleReasonApplicationsClocksSetting", 0x2),
+            "sync_boost": getattr(nv, "nvmlClocksThrottleReasonSyncBoost", 0x10),
+            "display_clock_setting": getattr(nv, "nvmlClocksThrottleReasonDisplayClockSetting", 0x100),
         }
         while not self._stop.is_set():
             try:
                 self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
                 mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                self.mask |= int(mask)
                 for k, bit in names.items():
                     if mask & bit:
                         self.reasons.add(k)
@@ -190,8 +194,9 @@ class ClockSampler:
     def summary(self):
         if not self.samples:
             return dict(sm_mhz=None, sm_max_mhz=self.max_mhz, reasons=sorted(self.reasons), samples=0)
-        return dict(sm_mhz=float(np.median(self.samples)), sm_max_mhz=self.max_mhz,
-                    reasons=sorted(self.reasons), samples=len(self.samples))
+        return dict(sm_mhz=float(np.median(self.samples)), sm_min_mhz=float(min(self.samples)),
+                    sm_max_mhz=self.max_mhz, reasons=sorted(self.reasons), reason_mask=hex(self.mask),
+                    samples=len(self.samples))
 
 
 def oracle_sample(name, wl_cpu=None):
