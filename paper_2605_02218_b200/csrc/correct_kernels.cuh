@@ -213,6 +213,15 @@ correct_kernel(const T* __restrict__ zd, const T* __restrict__ zt, long long ldz
   const T* rd = zd + (size_t)row * ldz;
   const T* rt = zt + (size_t)row * ldz;
   const T* const tag = nullptr;
+  // scalars of the position, requested now so that their latency hides behind the first sweep
+  const float x_uniform = __ldg(uniforms + row);
+  float zd_y = 0.f, zt_y = 0.f;
+  const bool has_y = accept != nullptr && drafted != nullptr;
+  if (has_y && tid == 0 && crank == 0) {
+    const int y = __ldg(drafted + row);
+    zd_y = cvt(rd[y]);
+    zt_y = cvt(rt[y]);
+  }
   // contiguous segment of this warp, in whole vectors
   const int nvec = (w + N - 1) / N;
   const int vec_per_seg = (nvec + kSegs - 1) / kSegs;
@@ -284,10 +293,13 @@ correct_kernel(const T* __restrict__ zd, const T* __restrict__ zt, long long ldz
   if (warp == 0) {
     // the same merge, in rank order, in every CTA of the cluster
     md = MaxSum{-INFINITY, 0.f}; mt = md; top = Top2{-INFINITY, -INFINITY};
-    for (unsigned c = 0; c < (unsigned)kClusterCtas; ++c) {
-      MaxSum od{peer_float(&sh_part[0], c), peer_float(&sh_part[1], c)};
-      MaxSum ot{peer_float(&sh_part[2], c), peer_float(&sh_part[3], c)};
-      Top2 otop{peer_float(&sh_part[4], c), peer_float(&sh_part[5], c)};
+    // lane 6 c + k fetches value k of CTA c; the values are then handed round by shuffles
+    float mine = 0.f;
+    if (lane < 6 * kClusterCtas) mine = peer_float(&sh_part[lane % 6], (unsigned)(lane / 6));
+    for (int c = 0; c < kClusterCtas; ++c) {
+      MaxSum od{__shfl_sync(0xffffffffu, mine, 6 * c), __shfl_sync(0xffffffffu, mine, 6 * c + 1)};
+      MaxSum ot{__shfl_sync(0xffffffffu, mine, 6 * c + 2), __shfl_sync(0xffffffffu, mine, 6 * c + 3)};
+      Top2 otop{__shfl_sync(0xffffffffu, mine, 6 * c + 4), __shfl_sync(0xffffffffu, mine, 6 * c + 5)};
       md.merge(od); mt.merge(ot); top.merge(otop);
     }
     if (lane == 0) {
@@ -300,9 +312,8 @@ correct_kernel(const T* __restrict__ zd, const T* __restrict__ zt, long long ldz
         gate[row] = m < gamma ? 1 : 0;                                       // Eq. 17
         if (accept != nullptr) {
           float al = 1.f;
-          if (drafted != nullptr) {
-            int y = drafted[row];
-            float pd = __expf(cvt(rd[y]) - md.m) / md.s, pt = __expf(cvt(rt[y]) - mt.m) / mt.s;
+          if (has_y) {
+            float pd = __expf(zd_y - md.m) / md.s, pt = __expf(zt_y - mt.m) / mt.s;
             al = pd > 0.f ? fminf(1.f, pt / pd) : 1.f;                       // Eq. 5
           }
           accept[row] = al;
@@ -350,7 +361,7 @@ correct_kernel(const T* __restrict__ zd, const T* __restrict__ zt, long long ldz
     if (!use_pt && crank == 0 && tid == 0 && resid_mass != nullptr) resid_mass[row] = mass;
     if (mass > 0.f || use_pt) {
       // ---- sweep 3: the warp whose segment contains x * mass walks it in order ----
-      const float target = uniforms[row] * mass;
+      const float target = x_uniform * mass;
       float before = 0.f;
       int seg = -1;
       for (int q = 0; q < kSegs; ++q) {
