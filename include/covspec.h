@@ -50,7 +50,8 @@ typedef enum {
                                    settled within the tolerance after its last step, or the small
                                    eigen-solve hit its sweep limit                             */
   COVSPEC_ERR_TIMEOUT = -8,     /* device status: a bounded wait inside a kernel expired      */
-  COVSPEC_ERR_STATIC_CAPACITY = -9 /* covspec_query_score_static: beyond its fixed scratch size */
+  COVSPEC_ERR_STATIC_CAPACITY = -9, /* covspec_query_score_static: beyond its fixed scratch size */
+  COVSPEC_ERR_BOUNDS = -10      /* device status, checked build only: an index was out of range  */
 } covspec_status;
 
 /* Static configuration.  Fill with covspec_default_config() and override. */
@@ -174,8 +175,8 @@ int covspec_compact_rows(covspec_ctx* ctx, const covspec_problem* p, const int* 
 int covspec_prune(covspec_ctx* ctx, const covspec_problem* p, void* out_hidden, int* keep_idx,
                   int* keep_offsets, void* stream);
 
-/* Synchronises `stream`, returns the device status word (COVSPEC_OK, COVSPEC_ERR_TIMEOUT, COVSPEC_ERR_NONFINITE or
- * COVSPEC_ERR_NOCONVERGE) and clears it. */
+/* Synchronises `stream`, returns the device status word (COVSPEC_OK, COVSPEC_ERR_BOUNDS, COVSPEC_ERR_TIMEOUT,
+ * COVSPEC_ERR_NONFINITE or COVSPEC_ERR_NOCONVERGE) and clears it. */
 int covspec_get_device_status(covspec_ctx* ctx, void* stream);
 
 /* Diagnostics of the subspace iteration behind Eq. 14 for the last covspec_select / covspec_prune call
@@ -289,6 +290,13 @@ int covspec_query_score_static(int dtype, int d, int batch, const void* X, const
 
 /* Number of kernels the last call on this context launched. */
 int covspec_last_launch_count(const covspec_ctx* ctx);
+
+/* 1 when the library was built with -DCOVSPEC_DEBUG_BOUNDS (libcovspec_debug.so): the kernels whose
+ * global accesses are driven by computed indices (row gathers of Eq. 13 and of the compaction, the
+ * ordered emission of the top-k selections) test every such index, raise COVSPEC_ERR_BOUNDS in the
+ * device status word and skip the access instead of making it.  0 for the ordinary build, whose
+ * kernels carry no such tests.  Host-only, no arguments, cannot fail. */
+int covspec_build_has_bounds_checks(void);
 
 /* Text of a covspec_status; for COVSPEC_ERR_CUDA, covspec_last_cuda_error gives the runtime's. */
 const char* covspec_strerror(int status);

@@ -13,7 +13,9 @@ from typing import Optional
 import numpy as np
 import torch
 
-_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libcovspec.so")
+# COVSPEC_LIBRARY selects another build of the same library (the checked one, libcovspec_debug.so)
+_LIB_PATH = os.environ.get("COVSPEC_LIBRARY") or \
+    os.path.join(os.path.dirname(os.path.abspath(__file__)), "libcovspec.so")
 
 COVSPEC_F32, COVSPEC_BF16, COVSPEC_F16 = 0, 1, 2
 NORM_MODES = {"minmax": 0, "zscore": 1, "none": 2}
@@ -28,7 +30,7 @@ EXPORTS = [
     "covspec_profile_stage_name", "covspec_query_score_static", "covspec_selftest_wait_timeout",
     "covspec_correct", "covspec_fanout", "covspec_branch_candidates",
     "covspec_uplink_bits", "covspec_downlink_bits", "covspec_comm_latency", "covspec_ema_update",
-    "covspec_draft_length", "covspec_get_iteration_counts",
+    "covspec_draft_length", "covspec_get_iteration_counts", "covspec_build_has_bounds_checks",
 ]
 STATIC_MAX_BATCH = 256
 STATIC_MAX_QUERY_ELEMS = 1 << 20

@@ -12,6 +12,20 @@ constexpr int kMaxLayers = 17;    // act_layers + 1 snapshots at most
 // Device status bits (OR-ed into the context's status word).
 constexpr int kStatusNonFinite = 1;
 constexpr int kStatusNoConverge = 2;
+constexpr int kStatusBounds = 8;      // checked build only (4 is the wait time-out of the tensor-core kernels)
+
+// Checked build (-DCOVSPEC_DEBUG_BOUNDS, libcovspec_debug.so): index-driven global accesses test
+// their index first; a bad one raises kStatusBounds in the status word and the access is skipped, so
+// the context stays usable and the host reads COVSPEC_ERR_BOUNDS.  The ordinary build compiles the
+// test away.
+#ifdef COVSPEC_DEBUG_BOUNDS
+#define COVSPEC_IN_BOUNDS(idx, limit, status)                                              \
+  (((long long)(idx) >= 0 && (long long)(idx) < (long long)(limit))                        \
+       ? true                                                                              \
+       : ((status) != nullptr ? (atomicOr((status), ::covspec::kStatusBounds), false) : false))
+#else
+#define COVSPEC_IN_BOUNDS(idx, limit, status) true
+#endif
 
 // Per-request launch plan, built on the host from the offset arrays and uploaded once per shape.
 struct ReqPlan {

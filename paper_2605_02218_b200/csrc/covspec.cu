@@ -653,7 +653,7 @@ int select_impl(covspec_ctx* ctx, const covspec_problem* p, const float* s_fused
     int vec16 = cfg.d * ctx->esize / 16;
     gather_rows_kernel<<<gather_grid(pl.total_presel), kGatherWarps * 32, 0, s>>>(
         reinterpret_cast<const uint4*>(p->X), presel, ctx->d_plan, B, 1, vec16, (int)pl.total_presel,
-        reinterpret_cast<uint4*>(ctx->Zg), nullptr);
+        reinterpret_cast<uint4*>(ctx->Zg), nullptr, ctx->status);
     LAUNCH_CHECK(ctx);
     int st;
     dim3 gb(std::min(64, (pl.p_max * pl.m_max + 255) / 256 + 1), B);
@@ -723,7 +723,7 @@ int compact_impl(covspec_ctx* ctx, const covspec_problem* p, const int* keep_idx
   int vec16 = ctx->cfg.d * ctx->esize / 16;
   gather_rows_kernel<<<gather_grid(pl.total_keep), kGatherWarps * 32, 0, s>>>(
       reinterpret_cast<const uint4*>(p->X), keep_idx, ctx->d_plan, p->batch, 0, vec16, (int)pl.total_keep,
-      reinterpret_cast<uint4*>(out), out_pos);
+      reinterpret_cast<uint4*>(out), out_pos, ctx->status);
   LAUNCH_CHECK(ctx);
   prof_mark(ctx, ST_FINAL, 1, s);
   return COVSPEC_OK;
@@ -1015,7 +1015,7 @@ int covspec_compact_rows(covspec_ctx* ctx, const covspec_problem* p, const int* 
     return COVSPEC_ERR_SHAPE;
   gather_rows_kernel<<<gather_grid(ctx->plan.total_keep), kGatherWarps * 32, 0, s>>>(
       reinterpret_cast<const uint4*>(src), keep_idx, ctx->d_plan, p->batch, 0, (int)(row_bytes / 16),
-      (int)ctx->plan.total_keep, reinterpret_cast<uint4*>(out), nullptr);
+      (int)ctx->plan.total_keep, reinterpret_cast<uint4*>(out), nullptr, ctx->status);
   LAUNCH_CHECK(ctx);
   return COVSPEC_OK;
 }
@@ -1097,6 +1097,7 @@ int covspec_get_device_status(covspec_ctx* ctx, void* stream) {
   CUDA_TRY(cudaMemcpyAsync(&h, ctx->status, sizeof(int), cudaMemcpyDeviceToHost, s));
   CUDA_TRY(cudaMemsetAsync(ctx->status, 0, sizeof(int), s));
   CUDA_TRY(cudaStreamSynchronize(s));
+  if (h & kStatusBounds) return COVSPEC_ERR_BOUNDS;
   if (h & kStatusTimeout) return COVSPEC_ERR_TIMEOUT;
   if (h & kStatusNonFinite) return COVSPEC_ERR_NONFINITE;
   if (h & kStatusNoConverge) return COVSPEC_ERR_NOCONVERGE;
@@ -1227,11 +1228,20 @@ const char* covspec_strerror(int status) {
     case COVSPEC_ERR_TIMEOUT: return "a bounded wait inside a kernel expired";
     case COVSPEC_ERR_STATIC_CAPACITY:
       return "problem exceeds the fixed scratch capacity of the allocation-free entry point";
+    case COVSPEC_ERR_BOUNDS: return "checked build: an index-driven access was out of range and skipped";
     default: return "unknown status";
   }
 }
 
 const char* covspec_last_cuda_error(void) { return g_cuda_error.c_str(); }
+
+int covspec_build_has_bounds_checks(void) {
+#ifdef COVSPEC_DEBUG_BOUNDS
+  return 1;
+#else
+  return 0;
+#endif
+}
 
 }  // extern "C"
 

@@ -125,7 +125,7 @@ __device__ void block_topk_by(LoadF load, int n, int k, bool all_equal,
       }
       unsigned tot;
       unsigned ex = block_exclusive_scan(sel, warp_tot, &tot);
-      if (sel) out[run + ex] = remap ? remap[i] : i;
+      if (sel && COVSPEC_IN_BOUNDS(run + ex, k, status)) out[run + ex] = remap ? remap[i] : i;
       run += tot;
     }
     return;
@@ -185,7 +185,8 @@ __device__ void block_topk_by(LoadF load, int n, int k, bool all_equal,
     for (int j = 0; j < kRegKeys; ++j) {
       if (j < cnt) {
         const bool g = kreg[j] > prefix, e = kreg[j] == prefix;
-        if (g || (e && eq_before < kk)) out[gt_before + min(eq_before, kk)] = remap ? remap[i0 + j] : i0 + j;
+        if ((g || (e && eq_before < kk)) && COVSPEC_IN_BOUNDS(gt_before + min(eq_before, kk), k, status))
+          out[gt_before + min(eq_before, kk)] = remap ? remap[i0 + j] : i0 + j;
         gt_before += g;
         eq_before += e;
       }
@@ -229,7 +230,7 @@ __device__ void block_topk_by(LoadF load, int n, int k, bool all_equal,
     unsigned gt_before = run_gt + (ex & 0xffffu), eq_before = run_eq + (ex >> 16);
     if (gt || (eq && eq_before < kk)) {
       unsigned pos = gt_before + min(eq_before, kk);
-      out[pos] = remap ? remap[i] : i;
+      if (COVSPEC_IN_BOUNDS(pos, k, status)) out[pos] = remap ? remap[i] : i;
     }
     run_gt += tot & 0xffffu;
     run_eq += tot >> 16;
@@ -280,7 +281,7 @@ constexpr int kGatherWarps = 8;
 __global__ void __launch_bounds__(kGatherWarps * 32)
 gather_rows_kernel(const uint4* __restrict__ src, const int* __restrict__ idx,
                    const ReqPlan* __restrict__ plan, int batch, int use_presel, int row_vec16, int rows,
-                   uint4* __restrict__ dst, int* __restrict__ out_pos) {
+                   uint4* __restrict__ dst, int* __restrict__ out_pos, int* status) {
   const int lane = threadIdx.x & 31;
   const int row = blockIdx.x * kGatherWarps + (threadIdx.x >> 5);
   if (row >= rows) return;
@@ -291,10 +292,12 @@ gather_rows_kernel(const uint4* __restrict__ src, const int* __restrict__ idx,
       return use_presel ? plan[q].presel_off : plan[q].keep_off;
     });
     tok = idx[row];
-    first = (long long)plan[b].vis_off + tok;
+    // checked build: a token index outside its request is reported and the row is skipped
+    first = COVSPEC_IN_BOUNDS(tok, plan[b].n, status) ? (long long)plan[b].vis_off + tok : -1;
     if (out_pos != nullptr) out_pos[row] = tok;
   }
   first = __shfl_sync(0xffffffffu, first, 0);
+  if (first < 0) return;
   const uint4* s = src + (size_t)first * row_vec16;
   uint4* d = dst + (size_t)row * row_vec16;
   int v = lane;

@@ -116,8 +116,8 @@ def test_host_side_rejections(lib):
 
 
 def test_strerror(lib):
-    texts = {lib.covspec_strerror(s).decode() for s in range(0, -10, -1)}
-    assert len(texts) == 10 and "unknown status" not in texts
+    texts = {lib.covspec_strerror(s).decode() for s in range(0, -11, -1)}
+    assert len(texts) == 11 and "unknown status" not in texts
     assert lib.covspec_strerror(-99).decode() == "unknown status"
 
 
@@ -126,3 +126,15 @@ def test_binding_fails_loudly_without_library(monkeypatch):
     monkeypatch.setattr(api, "_LIB_PATH", "/nonexistent/libcovspec.so")
     with pytest.raises(RuntimeError, match="no fallback"):
         api.load_library()
+
+
+def test_checked_build_exports_the_same_interface(lib):
+    # libcovspec_debug.so: the same sources with the index tests compiled in
+    path = build.build(debug_bounds=True)
+    dbg = C.CDLL(path)
+    for name in api.EXPORTS:
+        assert getattr(dbg, name) is not None
+    assert dbg.covspec_build_has_bounds_checks() == 1
+    assert lib.covspec_build_has_bounds_checks() == 0
+    dbg.covspec_strerror.restype = C.c_char_p
+    assert b"out of range" in dbg.covspec_strerror(-10)
