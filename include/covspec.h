@@ -76,8 +76,10 @@ typedef struct {
   int max_vis_per_req;           /* max N_b */
   int max_presel_per_req;        /* max M_b   (0: derive from max_vis_per_req) */
   long long max_total_presel;    /* sum of M_b (0: derive from max_total_vis)  */
-  int relevance_path;  /* 0: Eq. 10 on the tensor cores (tcgen05) whenever the configuration allows
-                          (bf16, 128-wide heads, max over heads, d >= 64), else the CUDA-core path;
+  int relevance_path;  /* 0: Eq. 10 and the Gram matrix of Eq. 13 on the tensor cores (tcgen05) whenever
+                          the configuration allows (128-wide heads, max over heads, d >= 64; float32
+                          inputs are first split into three bf16 terms, about 2^-17 relative, which
+                          takes workspace for 1.5 times the inputs), else the CUDA-core path;
                           1: always the CUDA-core path; 2: the two-SM form of the tensor-core kernel
                           (tcgen05.mma.cta_group::2 on pairs of token tiles; measured no faster than
                           the one-SM form, kept selectable)                                        */

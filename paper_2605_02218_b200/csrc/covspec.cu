@@ -105,6 +105,12 @@ struct covspec_ctx {
   float* Cg = nullptr;                   // factor columns of the greedy low-rank mode
   long long cg_cap = 0;
   CUtensorMap map_zg, map_zgw, map_gh, map_gl, map_y[2][2];
+  // float32 inputs on the tensor cores: operands split into bf16 rows three times as wide
+  // (split3_kernel); nullptr / 0 when the configuration does not take that route
+  bool split_tc = false;
+  int dp = 0, d3 = 0;                    // d rounded up to 64; 3 * dp
+  __nv_bfloat16 *X3 = nullptr, *Q3 = nullptr, *Wq3 = nullptr, *Wk3 = nullptr, *Za3 = nullptr, *Zb3 = nullptr;
+  CUtensorMap map_za3, map_zb3w;
   // pinned staging for the plan upload
   char* h_stage = nullptr;
   long long stage_bytes = 0, stage_sched_off = 0;
@@ -424,7 +430,7 @@ int make_map_bf16(CUtensorMap* map, const void* base, long long rows, long long 
 
 bool tc_supported(const covspec_ctx* ctx) {
   const covspec_config& c = ctx->cfg;
-  return ctx->tc_ready && c.relevance_path != 1 && c.dtype == COVSPEC_BF16 && c.n_heads > 0 &&
+  return ctx->tc_ready && c.relevance_path != 1 && (c.dtype == COVSPEC_BF16 || ctx->split_tc) && c.n_heads > 0 &&
          c.head_dim == tc::kHeadDim && c.head_reduce == 0 && c.d >= tc::kBK;
 }
 
@@ -434,14 +440,16 @@ int relevance_pair(covspec_ctx* ctx, const covspec_problem* p, float* s_query, c
   const covspec_config& cfg = ctx->cfg;
   const Plan& pl = ctx->plan;
   int P = ctx->P, d = cfg.d;
+  const void *X = p->X, *Q = p->Q, *Wk = p->Wk, *Wq = p->Wq;
+  if (ctx->split_tc) { X = ctx->X3; Q = ctx->Q3; Wk = ctx->Wk3; Wq = ctx->Wq3; d = ctx->d3; }
   __nv_bfloat16* qn = reinterpret_cast<__nv_bfloat16*>(ctx->Qn);
   CUtensorMap map_x, map_wk, map_q, map_wq, map_qn, map_qnl;
   long long lo_off = (long long)cfg.max_total_txt * P;   // lo parts follow the hi parts
   int st;
-  if ((st = make_map_bf16(&map_x, p->X, pl.total_vis, d, tc::kTileM))) return st;
-  if ((st = make_map_bf16(&map_wk, p->Wk, P, d, tc::kTileN / 2))) return st;
-  if ((st = make_map_bf16(&map_q, p->Q, pl.total_txt, d, tc::kTileM))) return st;
-  if ((st = make_map_bf16(&map_wq, p->Wq, P, d, tc::kTileN / 2))) return st;
+  if ((st = make_map_bf16(&map_x, X, pl.total_vis, d, tc::kTileM))) return st;
+  if ((st = make_map_bf16(&map_wk, Wk, P, d, tc::kTileN / 2))) return st;
+  if ((st = make_map_bf16(&map_q, Q, pl.total_txt, d, tc::kTileM))) return st;
+  if ((st = make_map_bf16(&map_wq, Wq, P, d, tc::kTileN / 2))) return st;
   if ((st = make_map_bf16(&map_qn, qn, pl.total_txt, P, tc::kTT / 2))) return st;
   if ((st = make_map_bf16(&map_qnl, qn + lo_off, pl.total_txt, P, tc::kTT / 2))) return st;
   int n_hp = (cfg.n_heads + 1) / 2;
@@ -478,14 +486,16 @@ int relevance_tc(covspec_ctx* ctx, const covspec_problem* p, float* s_query, cud
   const covspec_config& cfg = ctx->cfg;
   const Plan& pl = ctx->plan;
   int P = ctx->P, d = cfg.d;
+  const void *X = p->X, *Q = p->Q, *Wk = p->Wk, *Wq = p->Wq;
+  if (ctx->split_tc) { X = ctx->X3; Q = ctx->Q3; Wk = ctx->Wk3; Wq = ctx->Wq3; d = ctx->d3; }
   __nv_bfloat16* qn = reinterpret_cast<__nv_bfloat16*>(ctx->Qn);
   CUtensorMap map_x, map_wk, map_q, map_wq, map_qn, map_qnl;
   long long lo_off = (long long)cfg.max_total_txt * P;   // lo parts follow the hi parts
   int st;
-  if ((st = make_map_bf16(&map_x, p->X, pl.total_vis, d, tc::kTileM))) return st;
-  if ((st = make_map_bf16(&map_wk, p->Wk, P, d, tc::kTileN))) return st;
-  if ((st = make_map_bf16(&map_q, p->Q, pl.total_txt, d, tc::kTileM))) return st;
-  if ((st = make_map_bf16(&map_wq, p->Wq, P, d, tc::kTileN))) return st;
+  if ((st = make_map_bf16(&map_x, X, pl.total_vis, d, tc::kTileM))) return st;
+  if ((st = make_map_bf16(&map_wk, Wk, P, d, tc::kTileN))) return st;
+  if ((st = make_map_bf16(&map_q, Q, pl.total_txt, d, tc::kTileM))) return st;
+  if ((st = make_map_bf16(&map_wq, Wq, P, d, tc::kTileN))) return st;
   if ((st = make_map_bf16(&map_qn, qn, pl.total_txt, P, tc::kTT))) return st;
   if ((st = make_map_bf16(&map_qnl, qn + lo_off, pl.total_txt, P, tc::kTT))) return st;
   int n_hp = (cfg.n_heads + 1) / 2;
@@ -577,6 +587,18 @@ int score_impl(covspec_ctx* ctx, const covspec_problem* p, float* s_query, float
     CUDA_TRY(cudaEventRecord(ctx->ev_join, ctx->side));
   }
   if (use_tc) {
+    if (ctx->split_tc) {
+      // float32 inputs: tokens and queries in the "a" form, the two weight matrices in the "b" form
+      SplitJobs jobs{};
+      jobs.j[0] = SplitJob{reinterpret_cast<const float*>(p->X), nullptr, ctx->X3, nullptr, rowsX};
+      jobs.j[1] = SplitJob{reinterpret_cast<const float*>(p->Q), nullptr, ctx->Q3, nullptr, (long long)rowsQ};
+      jobs.j[2] = SplitJob{reinterpret_cast<const float*>(p->Wk), nullptr, nullptr, ctx->Wk3, (long long)P};
+      jobs.j[3] = SplitJob{reinterpret_cast<const float*>(p->Wq), nullptr, nullptr, ctx->Wq3, (long long)P};
+      long long most = std::max<long long>(std::max<long long>(rowsX, rowsQ), P);
+      dim3 grid((unsigned)std::min<long long>(most, 8ll * ctx->num_sms), 4);
+      split3_kernel<<<grid, 256, 0, s>>>(jobs, ctx->d_plan, B, cfg.d, ctx->dp);
+      LAUNCH_CHECK(ctx);
+    }
     int st = cfg.relevance_path == 2 ? relevance_pair(ctx, p, s_query, s) : relevance_tc(ctx, p, s_query, s);
     if (st) return st;
   } else {
@@ -650,13 +672,29 @@ int select_impl(covspec_ctx* ctx, const covspec_problem* p, const float* s_fused
   }
   if (pl.n_stage2 > 0) {
     prof_mark(ctx, ST_GRAM, 0, s);
+    int st;
+    dim3 gb(std::min(64, (pl.p_max * pl.m_max + 255) / 256 + 1), B);
+    if (ctx->split_tc) {
+      // float32 inputs on the tensor cores: the preselected rows are gathered and split in one pass
+      SplitJobs jobs{};
+      jobs.j[0] = SplitJob{reinterpret_cast<const float*>(p->X), presel, ctx->Za3, ctx->Zb3, pl.total_presel};
+      dim3 grid((unsigned)std::min<long long>(pl.total_presel, 8ll * ctx->num_sms), 1);
+      split3_kernel<<<grid, 256, 0, s>>>(jobs, ctx->d_plan, B, cfg.d, ctx->dp);
+      LAUNCH_CHECK(ctx);
+      sub::GramParams gp{};
+      gp.plan = ctx->d_plan; gp.batch = B; gp.n_items = pl.n_gram_tiles;
+      gp.k_chunks = ctx->d3 / sub::kBK;
+      gp.g_hi = ctx->Ghi; gp.g_lo = ctx->Glo; gp.ld = ctx->ld; gp.status = ctx->status;
+      int grid_g = std::min(pl.n_gram_tiles, ctx->num_sms);
+      sub::gram_tc_kernel<<<grid_g, 192, sub::kGramSmem, s>>>(ctx->map_za3, ctx->map_zb3w, gp);
+      LAUNCH_CHECK(ctx);
+      prof_mark(ctx, ST_GRAM, 1, s);
+    } else {
     int vec16 = cfg.d * ctx->esize / 16;
     gather_rows_kernel<<<gather_grid(pl.total_presel), kGatherWarps * 32, 0, s>>>(
         reinterpret_cast<const uint4*>(p->X), presel, ctx->d_plan, B, 1, vec16, (int)pl.total_presel,
         reinterpret_cast<uint4*>(ctx->Zg), nullptr, ctx->status);
     LAUNCH_CHECK(ctx);
-    int st;
-    dim3 gb(std::min(64, (pl.p_max * pl.m_max + 255) / 256 + 1), B);
     if (cfg.dtype == COVSPEC_BF16) {
       sub::GramParams gp{};
       gp.plan = ctx->d_plan; gp.batch = B; gp.n_items = pl.n_gram_tiles;
@@ -672,6 +710,7 @@ int select_impl(covspec_ctx* ctx, const covspec_problem* p, const float* s_fused
       LAUNCH_CHECK(ctx);
     }
     prof_mark(ctx, ST_GRAM, 1, s);
+    }
     prof_mark(ctx, ST_EIG, 0, s);
     if (cfg.lowrank_mode == 1) {
       // greedy pivoted selection instead of the subspace energies; it writes its own `energy`
@@ -847,6 +886,19 @@ int covspec_prune_init(const covspec_config* cfg, covspec_ctx** out) {
   long long o_sync = carve(4ll * (c.max_batch * sub::kSyncStride + 4));
   ctx->cg_cap = c.lowrank_mode == 1 ? (long long)c.max_total_presel * c.max_presel_per_req : 0;
   long long o_cg = carve(4ll * ctx->cg_cap);
+  ctx->split_tc = f32 && c.relevance_path != 1 && c.n_heads > 0 && c.head_dim == tc::kHeadDim &&
+                  c.head_reduce == 0 && c.d >= tc::kBK && c.d % 4 == 0;
+  ctx->dp = (int)round_up(c.d, 64);
+  ctx->d3 = 3 * ctx->dp;
+  long long o_x3 = 0, o_q3 = 0, o_wq3 = 0, o_wk3 = 0, o_za3 = 0, o_zb3 = 0;
+  if (ctx->split_tc) {
+    o_x3 = carve(2ll * c.max_total_vis * ctx->d3);
+    o_q3 = carve(2ll * c.max_total_txt * ctx->d3);
+    o_wq3 = carve(2ll * ctx->P * ctx->d3);
+    o_wk3 = carve(2ll * ctx->P * ctx->d3);
+    o_za3 = carve(2ll * c.max_total_presel * ctx->d3);
+    o_zb3 = carve(2ll * c.max_total_presel * ctx->d3);
+  }
   ctx->ws_bytes = off;
   cudaError_t e = cudaMalloc(&ctx->ws, (size_t)off);
   if (e != cudaSuccess) {
@@ -878,6 +930,14 @@ int covspec_prune_init(const covspec_config* cfg, covspec_ctx** out) {
   ctx->Lbuf = reinterpret_cast<float*>(w + o_lbuf);
   ctx->Ub = reinterpret_cast<float*>(w + o_ub);
   ctx->sync = reinterpret_cast<unsigned*>(w + o_sync);
+  if (ctx->split_tc) {
+    ctx->X3 = reinterpret_cast<__nv_bfloat16*>(w + o_x3);
+    ctx->Q3 = reinterpret_cast<__nv_bfloat16*>(w + o_q3);
+    ctx->Wq3 = reinterpret_cast<__nv_bfloat16*>(w + o_wq3);
+    ctx->Wk3 = reinterpret_cast<__nv_bfloat16*>(w + o_wk3);
+    ctx->Za3 = reinterpret_cast<__nv_bfloat16*>(w + o_za3);
+    ctx->Zb3 = reinterpret_cast<__nv_bfloat16*>(w + o_zb3);
+  }
   ctx->Cg = reinterpret_cast<float*>(w + o_cg);
   ctx->stage_bytes = round_up(sizeof(ReqPlan) * c.max_batch, 256) +
                      sizeof(GemmProb) * (long long)T_COUNT * c.max_batch;
@@ -932,6 +992,8 @@ int covspec_prune_init(const covspec_config* cfg, covspec_ctx** out) {
     int st = COVSPEC_OK;
     if (!f32) st = make_map_bf16(&ctx->map_zg, ctx->Zg, c.max_total_presel, c.d, sub::kTile);
     if (!f32 && !st) st = make_map_bf16(&ctx->map_zgw, ctx->Zg, c.max_total_presel, c.d, sub::kGramN);
+    if (ctx->split_tc && !st) st = make_map_bf16(&ctx->map_za3, ctx->Za3, c.max_total_presel, ctx->d3, sub::kTile);
+    if (ctx->split_tc && !st) st = make_map_bf16(&ctx->map_zb3w, ctx->Zb3, c.max_total_presel, ctx->d3, sub::kGramN);
     if (!st) st = make_map_bf16(&ctx->map_gh, ctx->Ghi, ctx->cap_rows, ctx->ld, sub::kTile);
     if (!st) st = make_map_bf16(&ctx->map_gl, ctx->Glo, ctx->cap_rows, ctx->ld, sub::kTile);
     for (int i = 0; i < 2 && !st; ++i)

@@ -170,6 +170,53 @@ activity_stream_kernel(LayerPtrs hs, int n_layers /* = act_layers */, long long 
   }
 }
 
+// float32 operands for the bf16 tensor-core kernels.  A float32 row x of width d becomes two bf16
+// rows of width 3 dp (dp = d rounded up to 64, padding zero): the "a" form [hi | lo | hi] and the "b"
+// form [hi | hi | lo] with hi = bf16(x), lo = bf16(x - hi).  The K-major product of an "a" row and a
+// "b" row is hi.hi + lo.hi + hi.lo, the three-term bf16 product (about 2^-17 relative), so the
+// kernels written for bf16 inputs run unchanged on a three times longer inner dimension.
+struct SplitJob {
+  const float* src;            // [rows or more, d] float32
+  const int* idx;              // nullptr: row r of src; else row plan[request of r].vis_off + idx[r]
+  __nv_bfloat16* out_a;        // [rows, 3 dp] or nullptr
+  __nv_bfloat16* out_b;        // [rows, 3 dp] or nullptr
+  long long rows;
+};
+struct SplitJobs { SplitJob j[4]; };
+
+__global__ void __launch_bounds__(256)
+split3_kernel(SplitJobs jobs, const ReqPlan* __restrict__ plan, int batch, int d, int dp) {
+  const SplitJob job = jobs.j[blockIdx.y];
+  for (long long row = blockIdx.x; row < job.rows; row += gridDim.x) {
+    long long src_row = row;
+    if (job.idx != nullptr) {
+      int b = find_request((int)row, batch, [&](int q) { return plan[q].presel_off; });
+      src_row = (long long)plan[b].vis_off + job.idx[row];
+    }
+    const float* x = job.src + (size_t)src_row * d;
+    for (int c = threadIdx.x * 4; c < dp; c += blockDim.x * 4) {       // d and dp are multiples of 4
+      float4 v = c < d ? *reinterpret_cast<const float4*>(x + c) : make_float4(0.f, 0.f, 0.f, 0.f);
+      __nv_bfloat162 h0 = __floats2bfloat162_rn(v.x, v.y), h1 = __floats2bfloat162_rn(v.z, v.w);
+      __nv_bfloat162 l0 = __floats2bfloat162_rn(v.x - __low2float(h0), v.y - __high2float(h0));
+      __nv_bfloat162 l1 = __floats2bfloat162_rn(v.z - __low2float(h1), v.w - __high2float(h1));
+      uint2 hi = make_uint2(*reinterpret_cast<uint32_t*>(&h0), *reinterpret_cast<uint32_t*>(&h1));
+      uint2 lo = make_uint2(*reinterpret_cast<uint32_t*>(&l0), *reinterpret_cast<uint32_t*>(&l1));
+      if (job.out_a != nullptr) {
+        __nv_bfloat16* o = job.out_a + (size_t)row * 3 * dp + c;
+        *reinterpret_cast<uint2*>(o) = hi;
+        *reinterpret_cast<uint2*>(o + dp) = lo;
+        *reinterpret_cast<uint2*>(o + 2 * dp) = hi;
+      }
+      if (job.out_b != nullptr) {
+        __nv_bfloat16* o = job.out_b + (size_t)row * 3 * dp + c;
+        *reinterpret_cast<uint2*>(o) = hi;
+        *reinterpret_cast<uint2*>(o + dp) = hi;
+        *reinterpret_cast<uint2*>(o + 2 * dp) = lo;
+      }
+    }
+  }
+}
+
 // ---- block-wide reductions used by the fuse kernel (blockDim.x multiple of 32, <= 1024) ----
 template <typename Op>
 __device__ __forceinline__ float block_reduce(float v, Op op, float identity, float* scratch) {
