@@ -43,7 +43,7 @@ from paper_2605_02218_b200 import workloads
 # launch of the full workload processes; see the summary named here.
 NCU_RELEVANCE_TRAFFIC = {"bytes_per_token": (148.589e6 - 25.69e6) / 16384, "fixed_bytes": 25.69e6, "config": "c5",
                          "source": "profiles/relevance_tc_kernel_c5_one_request.md"}
-NCU_CORRECT_BYTES_PER_ROW = 364.4e6 / 512          # profiles/correct_kernel_vocab152k.md
+NCU_CORRECT_BYTES_PER_ROW = 366.5e6 / 512          # profiles/correct_kernel_vocab152k.md
 
 METRIC = "visual_tokens_pruned_per_s"
 UNIT = "tokens/s"
