@@ -10,10 +10,14 @@
 //               factor[b] >= k
 //   ritz[b]     1 once the Rayleigh-Ritz vectors of the last block are published
 //   last[b]     index of the request's last step: eig_iters on entry; the tile that factors step k
-//               lowers it to k + 2 when the Ritz value estimates say that the energies will have
-//               settled by then (see team_cholesky).  It only ever decreases, and a change made after
-//               step k first matters two steps later, so every role of every CTA reads the same
-//               answer to "is step s skipped?" and "is step s the last?"
+//               lowers it to k + 1 when the Ritz value estimates say that the energies will have
+//               settled by then (see team_cholesky).  It only ever decreases and is written before
+//               factor[b] = k + 1 is published: the epilogue of step k + 1, which waits for that
+//               factor, reads "is this the last step?" with it, and the producer and MMA roles, which
+//               only ask "is step s skipped?", can first be affected at step k + 2, whose start
+//               every tile's arrival of step k + 1 precedes
+//   summed[b]   tiles of request b that have added up their slice of the partial Gram matrices of a
+//               step (only when every CTA holds exactly one tile, see spread_sum)
 // The tile that makes arrive[b] reach tiles(b) * (k + 1) (an atomic ticket; nobody waits for it to be
 // a particular CTA) sums the partial Gram matrices in tile order and factors the sum right there: a
 // Cholesky factorisation after the first steps, the Rayleigh-Ritz solve of the window next to the cut
@@ -21,8 +25,9 @@
 // every wait is bounded and a CTA that gives up raises a global abort word that ends the others'
 // waits too.  After the last step every CTA evaluates the energies (Eq. 15) of its own tiles.
 //
-// Data that crosses CTAs inside the kernel (partial sums, factors, Ritz vectors, the float32 blocks)
-// is read with L1-bypassing loads; the bf16 planes are read by TMA, behind a proxy fence.
+// Data that crosses CTAs inside the kernel (partial sums, factors, Ritz vectors, the float32 window
+// columns, the bf16 planes the last step re-reads) is read with L1-bypassing loads; the operand
+// tiles of the bf16 planes are read by TMA, behind a proxy fence.
 #pragma once
 #include "eig_kernels.cuh"
 
@@ -41,8 +46,8 @@ struct FusedParams {
   __nv_bfloat16* y_hi[2];   // plane buffers: step k reads [k & 1], writes [(k & 1) ^ 1]
   __nv_bfloat16* y_lo[2];
   int ld;
-  float* yf[2];             // [sum M_b, kPMax]: the block before the last multiplication (turned into
-                            // the orthonormal basis Q during the last step) and after it
+  float* yf[2];             // [sum M_b, kPMax], window columns only: the orthonormal basis Q of the block
+                            // before the last multiplication, and the block after it (Eq. 15)
   double* partial;          // [tiles][kTileDoubles], see tile_offset
   float* ub;                // [batch][kPMax * kPMax] Ritz vectors of the discarded pairs
   float* energy;            // [sum M_b] (out)
@@ -368,7 +373,7 @@ __device__ __forceinline__ bool extra_tile(int e, int nb8, int units, int& ta, i
 
 // Cholesky factor of the summed Gram matrix, written in the layout the triangular solve reads
 // (see lt_row_offset) followed by the reciprocal diagonal.  Tm: cholesky_smem_bytes(p) of scratch.
-// Returns (to every thread) whether the iteration may stop two steps from now: from the diagonal of
+// Returns (to every thread) whether the next step may be the last one: from the diagonal of
 // the summed Gram matrix B = Y'^T Y' (theta_i = sqrt(B_ii) estimates the i-th eigenvalue of G once the
 // basis has started to order itself) the energy error after q_final multiplications is predicted as
 // max_i 2 (theta_i / theta_1) (theta_min / theta_i)^q_final over the kept directions i < r that the
