@@ -53,6 +53,18 @@ def test_small_shapes(kw):
     _report(wl.name, parity.run_gpu(wl))
 
 
+@pytest.mark.parametrize("d,heads", [(200, 3), (64, 1), (328, 2)])
+def test_float32_on_the_tensor_cores_with_padded_width(d, heads):
+    # float32 inputs reach the tensor-core kernels as three bf16 terms laid side by side; every term
+    # is padded to a multiple of 64 columns (d = 200 -> 256, 328 -> 384), several requests, ragged sizes
+    wl = workloads.make_workload(f"f32-d{d}", seed=60 + heads, dtype=torch.float32, batch=3,
+                                 n_vis=(140, 700), n_txt=(3, 70), d=d, n_heads=heads, rank=12,
+                                 keep_ratio=0.25)
+    stats = parity.run_gpu(wl)
+    _report(wl.name, stats)
+    assert stats["launches"] == 12
+
+
 def test_zero_token_on_the_tensor_core_path():
     # an all-zero visual token has cosine 0 with every query element (zero-norm reading), also when
     # the query elements lean negative
