@@ -464,16 +464,15 @@ int relevance_pair(covspec_ctx* ctx, const covspec_problem* p, float* s_query, c
   prm.rows_total = pl.total_txt;
   prm.n_items = (int)((pl.total_txt + 2 * tc::kTileM - 1) / (2 * tc::kTileM)) * prm.n_groups;
   prm.qn_out = qn; prm.qn_lo_off = lo_off; prm.s_query = nullptr;
+  prm.fill = s_query; prm.fill_n = pl.total_vis;          // -inf for the visual-side launch below
   int grid = 2 * std::min(prm.n_items, max_clusters);
   tc2::relevance_pair_kernel<1><<<grid, tc2::kPairThreads, tc2::kSmemBytes2, s>>>(map_q, map_wq, map_qn, map_qnl, prm);
   LAUNCH_CHECK(ctx);
   prof_mark(ctx, ST_QEMBED, 1, s);
   // visual side
   prof_mark(ctx, ST_RELEVANCE, 0, s);
-  tc::fill_neg_inf_kernel<<<(unsigned)((pl.total_vis + 255) / 256), 256, 0, s>>>(s_query, pl.total_vis);
-  LAUNCH_CHECK(ctx);
   prm.n_items = pl.n_pairs * prm.n_groups;
-  prm.qn_out = nullptr; prm.s_query = s_query;
+  prm.qn_out = nullptr; prm.s_query = s_query; prm.fill = nullptr;
   grid = 2 * std::min(prm.n_items, max_clusters);
   tc2::relevance_pair_kernel<0><<<grid, tc2::kPairThreads, tc2::kSmemBytes2, s>>>(map_x, map_wk, map_qn, map_qnl, prm);
   LAUNCH_CHECK(ctx);
@@ -509,16 +508,15 @@ int relevance_tc(covspec_ctx* ctx, const covspec_problem* p, float* s_query, cud
   prm.rows_total = pl.total_txt;
   prm.n_items = (int)((pl.total_txt + tc::kTileM - 1) / tc::kTileM) * prm.n_groups;
   prm.qn_out = qn; prm.qn_lo_off = lo_off; prm.s_query = nullptr;
+  prm.fill = s_query; prm.fill_n = pl.total_vis;          // -inf for the visual-side launch below
   int grid = prm.n_items < ctx->num_sms ? prm.n_items : ctx->num_sms;
   tc::relevance_tc_kernel<1><<<grid, 192, tc::kSmemBytes, s>>>(map_q, map_wq, map_qn, map_qnl, prm);
   LAUNCH_CHECK(ctx);
   prof_mark(ctx, ST_QEMBED, 1, s);
   // visual side
   prof_mark(ctx, ST_RELEVANCE, 0, s);
-  tc::fill_neg_inf_kernel<<<(unsigned)((pl.total_vis + 255) / 256), 256, 0, s>>>(s_query, pl.total_vis);
-  LAUNCH_CHECK(ctx);
   prm.n_items = pl.n_tiles * prm.n_groups;
-  prm.qn_out = nullptr; prm.s_query = s_query;
+  prm.qn_out = nullptr; prm.s_query = s_query; prm.fill = nullptr;
   grid = prm.n_items < ctx->num_sms ? prm.n_items : ctx->num_sms;
   tc::relevance_tc_kernel<0><<<grid, 192, tc::kSmemBytes, s>>>(map_x, map_wk, map_qn, map_qnl, prm);
   LAUNCH_CHECK(ctx);

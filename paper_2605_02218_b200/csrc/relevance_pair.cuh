@@ -56,6 +56,8 @@ struct PairParams {
   float* s_query;       // MODE 0 out (pre-filled with -inf)
   __nv_bfloat16* qn_out;// MODE 1 out: hi [rows_total, P] followed by lo at qn_out + qn_lo_off
   long long qn_lo_off;
+  float* fill;          // MODE 1: score array to fill with -inf for the MODE 0 launch that follows
+  long long fill_n;     //         (nullptr: nothing to fill)
   int* status;
 };
 
@@ -157,6 +159,12 @@ relevance_pair_kernel(const __grid_constant__ CUtensorMap map_a,   // X (MODE 0)
   cluster_sync_all();                      // both CTAs' barriers exist before anything arrives on them
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  if (MODE == 1 && prm.fill != nullptr) {
+    // the visual-side launch combines head groups with an atomic max: its score array starts at -inf
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < prm.fill_n;
+         i += (long long)gridDim.x * blockDim.x)
+      prm.fill[i] = -INFINITY;
+  }
 
   const int n_hp = (prm.n_heads + 1) >> 1;
   const int n_clusters = gridDim.x >> 1, cluster_id = blockIdx.x >> 1;

@@ -61,6 +61,8 @@ struct Params {
   float* s_query;       // MODE 0 out (pre-filled with -inf)
   __nv_bfloat16* qn_out;// MODE 1 out: hi [rows_total, P] followed by lo at qn_out + qn_lo_off
   long long qn_lo_off;
+  float* fill;          // MODE 1: score array to fill with -inf for the MODE 0 launch that follows
+  long long fill_n;     //         (nullptr: nothing to fill)
   int* status;
 };
 
@@ -116,6 +118,12 @@ relevance_tc_kernel(const __grid_constant__ CUtensorMap map_a,   // X (MODE 0) o
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  if (MODE == 1 && prm.fill != nullptr) {
+    // the visual-side launch combines head groups with an atomic max: its score array starts at -inf
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < prm.fill_n;
+         i += (long long)gridDim.x * blockDim.x)
+      prm.fill[i] = -INFINITY;
+  }
 
   const int n_hp = (prm.n_heads + 1) >> 1;
 
@@ -382,13 +390,6 @@ relevance_tc_kernel(const __grid_constant__ CUtensorMap map_a,   // X (MODE 0) o
                  : "memory");
   }
   if (threadIdx.x == 0 && *abort_flag) atomicOr(prm.status, kStatusTimeout);
-}
-
-// Fills the score array with -inf so that the relevance kernel can combine head groups with an
-// atomic max.
-__global__ void fill_neg_inf_kernel(float* __restrict__ s, long long n) {
-  long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-  if (i < n) s[i] = -INFINITY;
 }
 
 }  // namespace tc
