@@ -64,7 +64,8 @@ struct Plan {
   int t_max = 0, p_max = 0, m_max = 0, win_max = 0, nbot_max = 0;
   int n_tiles = 0;                            // 128-token tiles over all requests
   int n_pairs = 0;                            // pairs of neighbouring tiles of one request
-  int n_gram_tiles = 0, n_ptiles = 0;         // lower-triangle Gram tiles / 128-row block tiles (stage 2)
+  int n_gram_tiles = 0, n_ptiles = 0;         // lower-triangle Gram items / row tiles of the subspace blocks (stage 2)
+  int tile_rows = 128;                        // rows of a subspace-block tile: 64 when that still gives every tile a CTA
   int pow_grid = 0;                           // CTAs of the power step
   std::vector<int> sched;                     // [pow_grid + 1] offsets + item lists (longest first)
   long long total_vis = 0, total_txt = 0, total_keep = 0, total_presel = 0;
@@ -228,7 +229,6 @@ int get_plan(covspec_ctx* ctx, const covspec_problem* p, cudaStream_t stream) {
     r.pair_off = pl.n_pairs;
     pl.n_pairs += ((r.n + tc::kTileM - 1) / tc::kTileM + 1) / 2;
     r.gram_tile_off = pl.n_gram_tiles;
-    r.ptile_off = pl.n_ptiles;
     r.g_off = g_off;
     r.c_off = c_off;
     if (r.stage2) {
@@ -237,7 +237,6 @@ int get_plan(covspec_ctx* ctx, const covspec_problem* p, cudaStream_t stream) {
       ++pl.n_stage2;
       int nt = (r.m + sub::kTile - 1) / sub::kTile;
       pl.n_gram_tiles += sub::gram_items(nt);
-      pl.n_ptiles += nt;
       if (f32) g_off += (long long)r.m * r.ldm;
       if (cfg.lowrank_mode == 1) {
         if (r.m > kGreedyMaxM || r.b_vis > kGreedyMaxB) return COVSPEC_ERR_UNSUPPORTED;
@@ -263,7 +262,22 @@ int get_plan(covspec_ctx* ctx, const covspec_problem* p, cudaStream_t stream) {
       pl.total_presel > ctx->cfg.max_total_presel || pl.n_ptiles > ctx->cap_ptiles)
     return COVSPEC_ERR_WORKSPACE;
 
-  // Schedule of the subspace kernel.  Its items (128-row tiles) differ in cost (basis size p, rows
+  // Row tiles of the subspace blocks: 128 rows, or 64 when every 64-row tile still gets a CTA of its
+  // own (the per-tile epilogue is the critical path of a step: half the rows, half the time).
+  {
+    long long n64 = 0;
+    for (int b = 0; b < B; ++b)
+      if (pl.req[b].stage2) n64 += (pl.req[b].m + 63) / 64;
+    pl.tile_rows = (n64 > 0 && n64 <= std::min<long long>(ctx->num_sms, ctx->cap_ptiles)) ? 64 : sub::kTile;
+    pl.n_ptiles = 0;
+    for (int b = 0; b < B; ++b) {
+      pl.req[b].ptile_off = pl.n_ptiles;
+      if (pl.req[b].stage2) pl.n_ptiles += (pl.req[b].m + pl.tile_rows - 1) / pl.tile_rows;
+    }
+    if (pl.n_ptiles > ctx->cap_ptiles) return COVSPEC_ERR_WORKSPACE;
+  }
+
+  // Schedule of the subspace kernel.  Its items (row tiles) differ in cost (basis size p, rows
   // in the tile), and every step of a request ends when its slowest tile does.  With more tiles
   // than CTAs, consecutive tiles of one request are therefore merged into groups and a group goes
   // to one CTA as a whole: a CTA that carries several tiles then delays one request instead of
@@ -272,7 +286,7 @@ int get_plan(covspec_ctx* ctx, const covspec_problem* p, cudaStream_t stream) {
   pl.sched.assign((size_t)pl.pow_grid + 1 + pl.n_ptiles, 0);
   if (pl.n_ptiles > 0) {
     auto tile_cost = [&](const ReqPlan& r, int t) {
-      int rows = std::min(sub::kTile, r.m - t * sub::kTile);
+      int rows = std::min(pl.tile_rows, r.m - t * pl.tile_rows);
       double pp = (double)r.p;
       return pp * pp * (1.0 + 1.5 * rows / sub::kTile) + 64.0 * r.m;
     };
@@ -283,7 +297,7 @@ int get_plan(covspec_ctx* ctx, const covspec_problem* p, cudaStream_t stream) {
     for (int b = 0; b < B; ++b) {
       const ReqPlan& r = pl.req[b];
       if (!r.stage2) continue;
-      int nt = (r.m + sub::kTile - 1) / sub::kTile;
+      int nt = (r.m + pl.tile_rows - 1) / pl.tile_rows;
       for (int t = 0; t < nt; ++t) groups.push_back(Group{tile_cost(r, t), r.ptile_off + t, 1, b});
     }
     while ((int)groups.size() > pl.pow_grid) {
@@ -727,6 +741,7 @@ int select_impl(covspec_ctx* ctx, const covspec_problem* p, const float* s_fused
     // energies: one cooperative launch (its CTAs wait on one another through global counters)
     sub::FusedParams fp{};
     fp.plan = ctx->d_plan; fp.batch = B; fp.n_items = pl.n_ptiles; fp.sched = ctx->d_sched;
+    fp.tile_rows = pl.tile_rows;
     fp.spread_sum = pl.n_ptiles <= pl.pow_grid ? 1 : 0;      // one tile per CTA (see the schedule above)
     fp.steps = cfg.eig_iters + 1;
     fp.lbuf = ctx->Lbuf;
@@ -856,7 +871,7 @@ int covspec_prune_init(const covspec_config* cfg, covspec_ctx** out) {
   ctx->g_cap = f32 ? (c.max_total_presel + 4ll * c.max_batch) * ldm_max : 0;
   ctx->ld = (int)round_up(c.max_presel_per_req, 64);
   ctx->cap_rows = c.max_total_presel;
-  ctx->cap_ptiles = c.max_total_presel / sub::kTile + c.max_batch;
+  ctx->cap_ptiles = std::max<long long>(c.max_total_presel / sub::kTile + c.max_batch, 192);   // >= one per SM
 
   long long off = 0;
   auto carve = [&](long long bytes) { long long o = off; off += round_up(bytes, 1024); return o; };

@@ -39,7 +39,8 @@ constexpr int kSyncStride = 8;           // unsigned words per request: arrive, 
 struct FusedParams {
   const ReqPlan* plan;
   int batch;
-  int n_items;              // 128-row tiles over all stage-2 requests
+  int n_items;              // row tiles over all stage-2 requests
+  int tile_rows;            // rows of a tile: 128, or 64 (the MMA still computes 128 rows; the upper half is dropped)
   const int* sched;         // [gridDim.x + 1] offsets, then the item lists of every CTA
   int steps;                // multiplications by G (eig_iters + 1, >= 2)
   float* lbuf;              // [batch][kLbufStride] triangular factor + reciprocal diagonal
@@ -577,6 +578,7 @@ subspace_kernel(const __grid_constant__ CUtensorMap map_gh, const __grid_constan
   const int s_begin = prm.sched[blockIdx.x], s_end = prm.sched[blockIdx.x + 1];
   const int* s_items = prm.sched + gridDim.x + 1;
   const int last_step = prm.steps - 1;
+  const int R = prm.tile_rows;
   auto decode = [&](int item, int& b, ReqPlan& rp, int& tile) {
     b = find_request(item, prm.batch, [&](int q) { return prm.plan[q].ptile_off; });
     rp = prm.plan[b];
@@ -598,7 +600,7 @@ subspace_kernel(const __grid_constant__ CUtensorMap map_gh, const __grid_constan
           if (step > 0) {
             // every tile of the request has written its slab of the block this step multiplies,
             // unless the request has already had its last step
-            const unsigned nt = (unsigned)((rp.m + kTile - 1) / kTile);
+            const unsigned nt = (unsigned)((rp.m + R - 1) / R);
             int last_b;
             const int go = step_decide(prm.sync + (size_t)b * kSyncStride, nt, step, gabort, abort_flag, &last_b);
             if (go < 0) { ok = false; break; }
@@ -614,7 +616,7 @@ subspace_kernel(const __grid_constant__ CUtensorMap map_gh, const __grid_constan
             if (!(ok = mbar_wait(&empty[s], ((it / kPowStages) & 1u) ^ 1u, abort_flag))) break;
             mbar_expect_tx(&full[s], kPowStageBytes);
             uint32_t dst = smem_u32(smem + s * kPowStageBytes);
-            int grow = rp.presel_off + tile * kTile;
+            int grow = rp.presel_off + tile * R;
             tma_load_2d(dst, &map_gh, kc * kBK, grow, &full[s]);
             tma_load_2d(dst + kPowBytesA, &map_gl, kc * kBK, grow, &full[s]);
             tma_load_2d(dst + 2 * kPowBytesA, myh, kc * kBK, b * kPMax, &full[s]);
@@ -636,7 +638,7 @@ subspace_kernel(const __grid_constant__ CUtensorMap map_gh, const __grid_constan
           decode(item, b, rp, tile);
           const uint32_t idesc = umma_idesc(kTile, (rp.p + 15) & ~15);
           if (step > 0) {
-            const unsigned nt = (unsigned)((rp.m + kTile - 1) / kTile);
+            const unsigned nt = (unsigned)((rp.m + R - 1) / R);
             int last_b;
             const int go = step_decide(prm.sync + (size_t)b * kSyncStride, nt, step, gabort, abort_flag, &last_b);
             if (go < 0) { ok = false; break; }
@@ -693,7 +695,7 @@ subspace_kernel(const __grid_constant__ CUtensorMap map_gh, const __grid_constan
         decode(item, b, rp, tile);
         const int p = rp.p, P = (p + 7) & ~7;
         unsigned* sync_b = prm.sync + (size_t)b * kSyncStride;
-        const unsigned nt = (unsigned)((rp.m + kTile - 1) / kTile);
+        const unsigned nt = (unsigned)((rp.m + R - 1) / R);
         // does the request still run this step, and is it its last one?  (one answer for the team)
         int last_b = last_step;
         if (!identity) {
@@ -734,7 +736,7 @@ subspace_kernel(const __grid_constant__ CUtensorMap map_gh, const __grid_constan
         const bool is_last = step == last_b;
         float* yf = is_last ? prm.yf[1] : nullptr;
         float* qprev = is_last ? prm.yf[0] : nullptr;
-        const int nrows = min(kTile, rp.m - tile * kTile);
+        const int nrows = min(R, rp.m - tile * R);
         // ---- Y_next row = T row * L^-T (forward substitution per row), staged as xs[c][r] ----
         // Between the first and the last step two threads share a row: warps 0-3 own the 32-column
         // super-block S being solved (contributions of the previous super-block and of its own
@@ -748,9 +750,13 @@ subspace_kernel(const __grid_constant__ CUtensorMap map_gh, const __grid_constan
           tc_fence_after();
         }
         const bool row_ok = r < nrows;
+        // with 64-row tiles the warps that own rows 64-127 (and their helpers) have nothing to solve;
+        // they keep taking part in the barriers
+        const bool active = (warp & 3) * 32 < R;
 #pragma unroll 1
         for (int S = 0; S < nS; ++S) {
           if (warp < 4) {
+            if (active) {
             float v[32];
             tmem_ld32(t_lane + S * 32, v);
             const float* hcur = hs + (S & 1) * 32 * kXsLd;
@@ -775,7 +781,8 @@ subspace_kernel(const __grid_constant__ CUtensorMap map_gh, const __grid_constan
                 for (int e = 0; e < 8; ++e) xs[(jb + e) * kXsLd + r] = (row_ok && ok) ? acc[e] : 0.f;
               }
             }
-          } else if (split && S >= 1 && S + 1 < nS) {
+            }
+          } else if (active && split && S >= 1 && S + 1 < nS) {
             // minus the contributions of the columns before 32 S to super-block S + 1
             float* hnext = hs + ((S + 1) & 1) * 32 * kXsLd;
 #pragma unroll 1
@@ -800,11 +807,11 @@ subspace_kernel(const __grid_constant__ CUtensorMap map_gh, const __grid_constan
           // ---- last step, warps 4-7: rows of Q = Y L^-T for the previous block Y, in place ----
           ok = ok && mbar_wait(acc_full, n & 1u, abort_flag);      // the ring is no longer read
           const int t4 = et - 128;
-          float* qrows = qprev + ((size_t)rp.presel_off + tile * kTile) * kPMax;
+          float* qrows = qprev + ((size_t)rp.presel_off + tile * R) * kPMax;
           {
             // the block this step multiplied, row t4 of the tile, from its two bf16 planes
-            const __nv_bfloat16* ph = prm.y_hi[step & 1] + (size_t)b * kPMax * prm.ld + tile * kTile + t4;
-            const __nv_bfloat16* pl = prm.y_lo[step & 1] + (size_t)b * kPMax * prm.ld + tile * kTile + t4;
+            const __nv_bfloat16* ph = prm.y_hi[step & 1] + (size_t)b * kPMax * prm.ld + tile * R + t4;
+            const __nv_bfloat16* pl = prm.y_lo[step & 1] + (size_t)b * kPMax * prm.ld + tile * R + t4;
             const unsigned short* uh = reinterpret_cast<const unsigned short*>(ph);
             const unsigned short* ul = reinterpret_cast<const unsigned short*>(pl);
             const bool have_row = t4 < nrows;
@@ -823,7 +830,7 @@ subspace_kernel(const __grid_constant__ CUtensorMap map_gh, const __grid_constan
             }
           }
           named_barrier(2, 128);
-          for (int jb = 0; jb < P; jb += 8) {
+          for (int jb = 0; jb < P && active; jb += 8) {
             float acc[8];
 #pragma unroll
             for (int e = 0; e < 8; ++e) acc[e] = xq[(jb + e) * kXsLd + t4];
@@ -843,14 +850,15 @@ subspace_kernel(const __grid_constant__ CUtensorMap map_gh, const __grid_constan
           // energy array until the Ritz vectors of the request are known
           float total = 0.f;
           for (int c = 0; c < p; ++c) total += xs[c * kXsLd + et] * xq[c * kXsLd + et];
-          prm.energy[(size_t)rp.presel_off + tile * kTile + et] = total;
+          prm.energy[(size_t)rp.presel_off + tile * R + et] = total;
         }
         // ---- bf16 planes of the new block (K-major operand of the next step): 8 positions per thread
         if (!is_last) {
           const int cols = (rp.m + kBK - 1) / kBK * kBK;
-          for (int wi = et; wi < p * 16; wi += kEpiThreads) {
-            int c = wi >> 4, ch = wi & 15;
-            int pos = tile * kTile + ch * 8;
+          const int cshift = R == 64 ? 3 : 4;          // 8-position chunks per row of the tile: 2^cshift
+          for (int wi = et; wi < (p << cshift); wi += kEpiThreads) {
+            int c = wi >> cshift, ch = wi & ((1 << cshift) - 1);
+            int pos = tile * R + ch * 8;
             if (pos >= cols) continue;
             const float4* xp = reinterpret_cast<const float4*>(xs + c * kXsLd + ch * 8);
             float4 a = xp[0], d = xp[1];
@@ -869,7 +877,7 @@ subspace_kernel(const __grid_constant__ CUtensorMap map_gh, const __grid_constan
         }
         if (yf != nullptr) {
           // float32 window columns of the final block, one token per row (second half of Eq. 15)
-          float* yrows = yf + ((size_t)rp.presel_off + tile * kTile) * kPMax;
+          float* yrows = yf + ((size_t)rp.presel_off + tile * R) * kPMax;
           for (int c = (p - rp.win) + (et & 31); c < p; c += 32)
             for (int rr = et >> 5; rr < nrows; rr += 8) yrows[(size_t)rr * kPMax + c] = xs[c * kXsLd + rr];
         }
@@ -1038,11 +1046,11 @@ subspace_kernel(const __grid_constant__ CUtensorMap map_gh, const __grid_constan
           epi_sync();
           cached_u = b;
         }
-        const int nrows = min(kTile, rp.m - tile * kTile);
+        const int nrows = min(R, rp.m - tile * R);
         // the discarded Ritz pairs take only the window columns of the two blocks: one thread per
         // row, window slices read straight from the float32 blocks
         for (int rr = et; rr < nrows; rr += kEpiThreads) {
-          const size_t grow = (size_t)rp.presel_off + tile * kTile + rr;
+          const size_t grow = (size_t)rp.presel_off + tile * R + rr;
           const float* yrow = prm.yf[1] + grow * kPMax + w0;
           const float* qrow = prm.yf[0] + grow * kPMax + w0;
           // projections of the two window slices on every discarded Ritz vector, accumulated over
