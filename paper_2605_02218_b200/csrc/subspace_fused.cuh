@@ -750,9 +750,10 @@ subspace_kernel(const __grid_constant__ CUtensorMap map_gh, const __grid_constan
           tc_fence_after();
         }
         const bool row_ok = r < nrows;
-        // with 64-row tiles the warps that own rows 64-127 (and their helpers) have nothing to solve;
-        // they keep taking part in the barriers
-        const bool active = (warp & 3) * 32 < R;
+        // warps whose 32 rows all lie beyond the tile's rows (64-row tiles, ragged last tiles), and
+        // their helpers, have nothing to solve; they keep taking part in the barriers.  Their rows
+        // of the staged block stay unwritten and are not read below.
+        const bool active = (warp & 3) * 32 < nrows;
 #pragma unroll 1
         for (int S = 0; S < nS; ++S) {
           if (warp < 4) {
@@ -863,6 +864,11 @@ subspace_kernel(const __grid_constant__ CUtensorMap map_gh, const __grid_constan
             const float4* xp = reinterpret_cast<const float4*>(xs + c * kXsLd + ch * 8);
             float4 a = xp[0], d = xp[1];
             float f[8] = {a.x, a.y, a.z, a.w, d.x, d.y, d.z, d.w};
+            if (ch * 8 + 8 > nrows) {                  // padding positions up to the k-chunk boundary are zero
+#pragma unroll
+              for (int e = 0; e < 8; ++e)
+                if (ch * 8 + e >= nrows) f[e] = 0.f;
+            }
             uint32_t ph[4], pl[4];
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
