@@ -66,6 +66,7 @@ struct Plan {
   int n_pairs = 0;                            // pairs of neighbouring tiles of one request
   int n_gram_tiles = 0, n_ptiles = 0;         // lower-triangle Gram items / row tiles of the subspace blocks (stage 2)
   int tile_rows = 128;                        // rows of a subspace-block tile: 64 when that still gives every tile a CTA
+  int tile_ctas = 0, servers = 0;             // CTAs of the subspace kernel that carry tiles / that only factor
   int pow_grid = 0;                           // CTAs of the power step
   std::vector<int> sched;                     // [pow_grid + 1] offsets + item lists (longest first)
   long long total_vis = 0, total_txt = 0, total_keep = 0, total_presel = 0;
@@ -282,7 +283,11 @@ int get_plan(covspec_ctx* ctx, const covspec_problem* p, cudaStream_t stream) {
   // than CTAs, consecutive tiles of one request are therefore merged into groups and a group goes
   // to one CTA as a whole: a CTA that carries several tiles then delays one request instead of
   // several.  Groups are handed out longest first, each to the least loaded CTA.
-  pl.pow_grid = std::min(pl.n_ptiles, ctx->num_sms);
+  // When SMs are left over, one more CTA per stage-2 request does nothing but factor for it (see the
+  // kernel): their item lists are empty.
+  pl.tile_ctas = std::min(pl.n_ptiles, ctx->num_sms);
+  pl.servers = (pl.n_ptiles > 0 && pl.n_ptiles + pl.n_stage2 <= ctx->num_sms) ? pl.n_stage2 : 0;
+  pl.pow_grid = pl.tile_ctas + pl.servers;
   pl.sched.assign((size_t)pl.pow_grid + 1 + pl.n_ptiles, 0);
   if (pl.n_ptiles > 0) {
     auto tile_cost = [&](const ReqPlan& r, int t) {
@@ -300,7 +305,7 @@ int get_plan(covspec_ctx* ctx, const covspec_problem* p, cudaStream_t stream) {
       int nt = (r.m + pl.tile_rows - 1) / pl.tile_rows;
       for (int t = 0; t < nt; ++t) groups.push_back(Group{tile_cost(r, t), r.ptile_off + t, 1, b});
     }
-    while ((int)groups.size() > pl.pow_grid) {
+    while ((int)groups.size() > pl.tile_ctas) {
       int best = -1;
       double best_cost = 0.0;
       for (int g = 0; g + 1 < (int)groups.size(); ++g) {
@@ -314,11 +319,11 @@ int get_plan(covspec_ctx* ctx, const covspec_problem* p, cudaStream_t stream) {
       groups.erase(groups.begin() + best + 1);
     }
     std::stable_sort(groups.begin(), groups.end(), [](const Group& a, const Group& b2) { return a.cost > b2.cost; });
-    std::vector<double> load(pl.pow_grid, 0.0);
-    std::vector<std::vector<int>> lists(pl.pow_grid);
+    std::vector<double> load(pl.tile_ctas, 0.0);
+    std::vector<std::vector<int>> lists(pl.tile_ctas);
     for (const Group& g : groups) {
       int best = 0;
-      for (int c = 1; c < pl.pow_grid; ++c) if (load[c] < load[best]) best = c;
+      for (int c = 1; c < pl.tile_ctas; ++c) if (load[c] < load[best]) best = c;
       load[best] += g.cost;
       for (int t = 0; t < g.count; ++t) lists[best].push_back(g.first + t);
     }
@@ -327,7 +332,8 @@ int get_plan(covspec_ctx* ctx, const covspec_problem* p, cudaStream_t stream) {
     int* items_out = pl.sched.data() + pl.pow_grid + 1;
     for (int g = 0; g < pl.pow_grid; ++g) {
       pl.sched[g] = off;
-      for (int v : lists[g]) items_out[off++] = v;
+      if (g < pl.tile_ctas)
+        for (int v : lists[g]) items_out[off++] = v;
     }
     pl.sched[pl.pow_grid] = off;
   }
@@ -742,7 +748,8 @@ int select_impl(covspec_ctx* ctx, const covspec_problem* p, const float* s_fused
     sub::FusedParams fp{};
     fp.plan = ctx->d_plan; fp.batch = B; fp.n_items = pl.n_ptiles; fp.sched = ctx->d_sched;
     fp.tile_rows = pl.tile_rows;
-    fp.spread_sum = pl.n_ptiles <= pl.pow_grid ? 1 : 0;      // one tile per CTA (see the schedule above)
+    fp.spread_sum = pl.n_ptiles <= pl.tile_ctas ? 1 : 0;     // one tile per CTA (see the schedule above)
+    fp.n_tile_ctas = pl.tile_ctas; fp.n_servers = pl.servers;
     fp.steps = cfg.eig_iters + 1;
     fp.lbuf = ctx->Lbuf;
     for (int i = 0; i < 2; ++i) { fp.y_hi[i] = ctx->Yp[i][0]; fp.y_lo[i] = ctx->Yp[i][1]; fp.yf[i] = ctx->Yf[i]; }

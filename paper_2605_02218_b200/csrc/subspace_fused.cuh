@@ -18,7 +18,9 @@
 //               every tile's arrival of step k + 1 precedes
 //   summed[b]   tiles of request b that have added up their slice of the partial Gram matrices of a
 //               step (only when every CTA holds exactly one tile, see spread_sum)
-// The tile that makes arrive[b] reach tiles(b) * (k + 1) (an atomic ticket; nobody waits for it to be
+// With SMs to spare the grid carries one more CTA per request that holds no tile and only factors for
+// that request (n_servers); otherwise
+// the tile that makes arrive[b] reach tiles(b) * (k + 1) (an atomic ticket; nobody waits for it to be
 // a particular CTA) sums the partial Gram matrices in tile order and factors the sum right there: a
 // Cholesky factorisation after the first steps, the Rayleigh-Ritz solve of the window next to the cut
 // after the last one.  All CTAs are resident at the same time (cooperative launch, one CTA per SM),
@@ -54,6 +56,9 @@ struct FusedParams {
   float* energy;            // [sum M_b] (out)
   unsigned* sync;           // [batch][kSyncStride] counters (zero on entry), then the abort word
   int spread_sum;           // every CTA holds exactly one tile: the tiles of a request sum the partial matrices together
+  int n_tile_ctas;          // CTAs that carry tiles: blockIdx.x < n_tile_ctas
+  int n_servers;            // CTAs after those, one per stage-2 request, that only factor (0: the last tile to
+                            // finish a step factors)
   int max_sweeps;
   float conv_tol;           // bound on the estimated energy error before NOCONVERGE is raised
   int early_stop;           // 1: requests whose estimate is far below conv_tol stop before `steps`
@@ -685,6 +690,60 @@ subspace_kernel(const __grid_constant__ CUtensorMap map_gh, const __grid_constan
     uint32_t n = 0;
     int cached_b = -1, cached_step = -1;
     bool ok = true;
+    // Factors the summed Gram matrix of request b after step `step` (Cholesky, or the Rayleigh-Ritz
+    // solve after the last step) and publishes the result; returns whether the next step was
+    // declared the last one.  Uses the operand ring as scratch.
+    auto factor_request = [&](int b, const ReqPlan& rp, unsigned* sync_b, int step, bool is_last, int last_b,
+                              int nt_sum) -> bool {
+      __threadfence();
+      const int p = rp.p;
+      const double* pbase = prm.partial + (size_t)rp.ptile_off * kTileDoubles;
+      double* Tm = reinterpret_cast<double*>(smem);        // the region is free: every thread passed the barrier
+      bool stop = false;
+      if (!is_last) {
+        // after the second multiplication and later: may the next step be the last one?  (asked with a
+        // margin of 8 under the tolerance, 64 at the first opportunity: the estimate is rough while
+        // the basis is still mixing)
+        const bool may_stop = prm.early_stop && step >= 1 && step + 1 < last_b && p < rp.m;
+        const float margin = step == 1 ? 0.015625f : 0.125f;
+        stop = team_cholesky(pbase, nt_sum, p, rp.r, prm.lbuf + (size_t)b * kLbufStride, Tm, dinv,
+                             s_word, step + 2, may_stop ? margin * prm.conv_tol : 0.f);
+        __threadfence();
+        epi_sync();
+        if (et == 0) {
+          if (stop) st_release_u32(sync_b + 3, (unsigned)(step + 1));
+          st_release_u32(sync_b + 1, (unsigned)(step + 1));
+        }
+      } else {
+        team_ritz(pbase, nt_sum, p, rp.win, rp.r, rp.m, prm.ub + (size_t)b * kPMax * kPMax, reinterpret_cast<float*>(smem), lt,
+                  s_scale, s_flag, prm.max_sweeps, prm.conv_tol, step + 1, prm.status);
+        __threadfence();
+        epi_sync();
+        if (et == 0) st_release_u32(sync_b + 2, 1u);
+      }
+      return stop;
+    };
+    if (prm.n_servers > 0 && (int)blockIdx.x >= prm.n_tile_ctas) {
+      // ------------------------------------------------------------ factor server
+      // This CTA carries no tile.  It factors for one request: on a CTA that also carries a tile the
+      // factorisation, which needs the operand ring as scratch, would delay that tile's next
+      // multiplication, and with it the request's next step.
+      const int mine = (int)blockIdx.x - prm.n_tile_ctas;
+      int b = -1, seen = 0;
+      for (int q = 0; q < prm.batch && b < 0; ++q)
+        if (prm.plan[q].stage2) { if (seen == mine) b = q; ++seen; }
+      if (b >= 0) {
+        const ReqPlan rp = prm.plan[b];
+        unsigned* sync_b = prm.sync + (size_t)b * kSyncStride;
+        const unsigned nt = (unsigned)((rp.m + R - 1) / R);
+        const bool summed = prm.spread_sum && nt >= 4;      // the tiles have added up the partial matrices
+        int last_b = last_step;
+        for (int step = 0; step <= last_b; ++step) {
+          if (!team_wait(summed ? sync_b + 4 : sync_b, nt * (unsigned)(step + 1))) break;
+          if (factor_request(b, rp, sync_b, step, step == last_b, last_b, summed ? 1 : (int)nt)) last_b = step + 1;
+        }
+      }
+    }
     for (int step = 0; step <= last_step; ++step) {
       const bool identity = step == 0;
       __nv_bfloat16* y_hi = prm.y_hi[(step & 1) ^ 1];
@@ -1004,32 +1063,9 @@ subspace_kernel(const __grid_constant__ CUtensorMap map_gh, const __grid_constan
           *s_word = (old + 1u == nt * (unsigned)(step + 1) && !*abort_flag) ? 1 : 0;
         }
         epi_sync();
-        if (*s_word) {
+        if (*s_word && prm.n_servers == 0) {
           // ---- the last tile of the request to finish this step factors the summed Gram matrix ----
-          __threadfence();
-          const double* pbase = prm.partial + (size_t)rp.ptile_off * kTileDoubles;
-          double* Tm = reinterpret_cast<double*>(smem);        // the region is free: every thread passed the barrier
-          if (!is_last) {
-            // after the second multiplication and later: may the next step be the last one?  (asked with a
-            // margin of 8 under the tolerance, 64 at the first opportunity: the estimate is rough while
-            // the basis is still mixing)
-            const bool may_stop = prm.early_stop && step >= 1 && step + 1 < last_b && p < rp.m;
-            const float margin = step == 1 ? 0.015625f : 0.125f;
-            const bool stop = team_cholesky(pbase, nt_sum, p, rp.r, prm.lbuf + (size_t)b * kLbufStride, Tm, dinv,
-                                            s_word, step + 2, may_stop ? margin * prm.conv_tol : 0.f);
-            __threadfence();
-            epi_sync();
-            if (et == 0) {
-              if (stop) st_release_u32(sync_b + 3, (unsigned)(step + 1));
-              st_release_u32(sync_b + 1, (unsigned)(step + 1));
-            }
-          } else {
-            team_ritz(pbase, nt_sum, p, rp.win, rp.r, rp.m, prm.ub + (size_t)b * kPMax * kPMax, reinterpret_cast<float*>(smem), lt,
-                      s_scale, s_flag, prm.max_sweeps, prm.conv_tol, step + 1, prm.status);
-            __threadfence();
-            epi_sync();
-            if (et == 0) st_release_u32(sync_b + 2, 1u);
-          }
+          factor_request(b, rp, sync_b, step, is_last, last_b, nt_sum);
         }
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         mbar_arrive(epi_done);
