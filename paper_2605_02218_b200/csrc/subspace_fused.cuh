@@ -912,6 +912,9 @@ subspace_kernel(const __grid_constant__ CUtensorMap map_gh, const __grid_constan
           for (int c = 0; c < p; ++c) total += xs[c * kXsLd + et] * xq[c * kXsLd + et];
           prm.energy[(size_t)rp.presel_off + tile * R + et] = total;
         }
+        // the partial Gram below stages its slabs where the previous block (xq) lives: nobody may
+        // start on them while a row still reads xq
+        if (is_last) epi_sync();
         // ---- bf16 planes of the new block (K-major operand of the next step): 8 positions per thread
         if (!is_last) {
           const int cols = (rp.m + kBK - 1) / kBK * kBK;

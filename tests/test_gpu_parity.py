@@ -407,3 +407,22 @@ def test_iteration_counts_reflect_the_adaptive_stop():
         assert any(c > 0 for c in counts)
         if not stop:
             assert all(c in (0, iters + 1) for c in counts)
+
+
+def test_repeated_calls_on_ragged_batch_agree():
+    # 150 fused calls on the ragged workload (last tiles of a few rows, several tiles per CTA, requests
+    # that stop at different steps) must give the same keep-set every time: a missing barrier between
+    # two users of one shared-memory region showed up as a rare garbage energy in a ragged last tile
+    from paper_2605_02218_b200 import api
+    wl = workloads.make_config("c4", device="cuda:0")
+    pr = api.Pruner.for_workload(wl)
+    m = pr.marshal(wl)
+    _, first, _ = pr.prune(m)
+    first = first.clone()
+    different = 0
+    for _ in range(150):
+        _, keep, _ = pr.prune(m)
+        different += int(not torch.equal(keep, first))
+    assert pr.device_status() == 0
+    pr.close()
+    assert different == 0
