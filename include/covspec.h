@@ -293,6 +293,13 @@ int covspec_query_score_static(int dtype, int d, int batch, const void* X, const
 /* Number of kernels the last call on this context launched. */
 int covspec_last_launch_count(const covspec_ctx* ctx);
 
+/* Test aid: fills the context's scratch (scores, Gram planes, subspace blocks, partial sums, factors,
+ * Ritz vectors, synchronisation words; not the per-call plan) with `byte` (0..255) on `stream`.  The
+ * next call must give the same results whatever the byte (0xFF makes every float and bf16 a NaN):
+ * every kernel has to write what it later reads.  Returns COVSPEC_OK, COVSPEC_ERR_ARG or
+ * COVSPEC_ERR_CUDA. */
+int covspec_selftest_fill_workspace(covspec_ctx* ctx, int byte, void* stream);
+
 /* 1 when the library was built with -DCOVSPEC_DEBUG_BOUNDS (libcovspec_debug.so): the kernels whose
  * global accesses are driven by computed indices (row gathers of Eq. 13 and of the compaction, the
  * ordered emission of the top-k selections) test every such index, raise COVSPEC_ERR_BOUNDS in the

@@ -31,6 +31,7 @@ EXPORTS = [
     "covspec_correct", "covspec_fanout", "covspec_branch_candidates",
     "covspec_uplink_bits", "covspec_downlink_bits", "covspec_comm_latency", "covspec_ema_update",
     "covspec_draft_length", "covspec_get_iteration_counts", "covspec_build_has_bounds_checks",
+    "covspec_selftest_fill_workspace",
 ]
 STATIC_MAX_BATCH = 256
 STATIC_MAX_QUERY_ELEMS = 1 << 20
@@ -98,6 +99,7 @@ def load_library():
     lib.covspec_compact_rows.argtypes = [vp, C.POINTER(Problem), vp, ip, vp, C.c_longlong, vp, vp]
     lib.covspec_get_device_status.argtypes = [vp, vp]
     lib.covspec_selftest_wait_timeout.argtypes = [vp, vp]
+    lib.covspec_selftest_fill_workspace.argtypes = [vp, C.c_int, vp]
     lib.covspec_get_iteration_counts.argtypes = [vp, C.c_int, ip, vp]
     lib.covspec_fanout.argtypes = [C.c_int, C.c_double, C.c_int]
     lib.covspec_uplink_bits.argtypes = [C.c_longlong, C.c_int, C.c_longlong, C.c_int]
@@ -361,6 +363,12 @@ class Pruner:
         if st:
             raise CovspecError(st, "covspec_get_iteration_counts")
         return out
+
+    def fill_workspace(self, byte: int):
+        """covspec_selftest_fill_workspace: poisons the context's scratch before the next call."""
+        st = self.lib.covspec_selftest_fill_workspace(self._ctx, int(byte), _stream())
+        if st:
+            raise CovspecError(st, "covspec_selftest_fill_workspace")
 
     def device_status(self) -> int:
         return int(self.lib.covspec_get_device_status(self._ctx, _stream()))

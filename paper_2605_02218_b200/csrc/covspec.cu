@@ -1317,6 +1317,15 @@ const char* covspec_strerror(int status) {
 
 const char* covspec_last_cuda_error(void) { return g_cuda_error.c_str(); }
 
+int covspec_selftest_fill_workspace(covspec_ctx* ctx, int byte, void* stream) {
+  if (!ctx || byte < 0 || byte > 255) return COVSPEC_ERR_ARG;
+  // everything behind the per-call plan, schedule and tables: scores, Gram planes, subspace blocks,
+  // partial sums, factors, Ritz vectors, synchronisation words
+  char* from = reinterpret_cast<char*>(ctx->Qn);
+  CUDA_TRY(cudaMemsetAsync(from, byte, (size_t)(ctx->ws + ctx->ws_bytes - from), reinterpret_cast<cudaStream_t>(stream)));
+  return COVSPEC_OK;
+}
+
 int covspec_build_has_bounds_checks(void) {
 #ifdef COVSPEC_DEBUG_BOUNDS
   return 1;

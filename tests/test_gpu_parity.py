@@ -426,3 +426,20 @@ def test_repeated_calls_on_ragged_batch_agree():
     assert pr.device_status() == 0
     pr.close()
     assert different == 0
+
+
+@pytest.mark.parametrize("name", ["c2", "c4"])
+def test_poisoned_scratch_changes_nothing_at_full_size(name):
+    # the whole scratch of the context filled with NaN patterns, huge values and zeros between calls
+    from paper_2605_02218_b200 import api
+    wl = workloads.make_config(name, device="cuda:0")
+    pr = api.Pruner.for_workload(wl)
+    m = pr.marshal(wl)
+    out, keep, _ = pr.prune(m)
+    out, keep = out.clone(), keep.clone()
+    for byte in (0xFF, 0x7F, 0x00):
+        pr.fill_workspace(byte)
+        out2, keep2, _ = pr.prune(m)
+        assert pr.device_status() == 0
+        assert torch.equal(keep2, keep) and torch.equal(out2, out), hex(byte)
+    pr.close()
