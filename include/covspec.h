@@ -82,7 +82,7 @@ typedef struct {
                           takes workspace for 1.5 times the inputs), else the CUDA-core path;
                           1: always the CUDA-core path; 2: the two-SM form of the tensor-core kernel
                           (tcgen05.mma.cta_group::2 on pairs of token tiles; measured no faster than
-                          the one-SM form, kept selectable)                                        */
+                          the one-SM form, kept selectable); other values: COVSPEC_ERR_ARG         */
   int lowrank_mode;    /* 0: energy in the top-r singular subspace (Eq. 14-15, the paper's criterion);
                           1: greedy pivoted selection (not in the paper): pick B_vis times the token with
                              the largest residual energy after projecting out the picked ones; needs

@@ -168,6 +168,7 @@ int validate_cfg(const covspec_config* c) {
   if (c->eig_iters < 1 || c->eig_oversample < 0) return COVSPEC_ERR_ARG;
   if (c->rank_cap + c->eig_oversample > kPMax) return COVSPEC_ERR_UNSUPPORTED;
   if (c->lowrank_mode < 0 || c->lowrank_mode > 1) return COVSPEC_ERR_ARG;
+  if (c->relevance_path < 0 || c->relevance_path > 2) return COVSPEC_ERR_ARG;
   if (c->ritz_window < 0) return COVSPEC_ERR_ARG;
   if (c->activity_overlap < 0 || c->activity_overlap > 2) return COVSPEC_ERR_ARG;
   if (c->eig_iters > 1000 || !(c->conv_tol >= 0.f)) return COVSPEC_ERR_ARG;

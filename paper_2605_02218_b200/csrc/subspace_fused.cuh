@@ -138,6 +138,19 @@ __device__ __forceinline__ double gram_entry_cg(int ntile, const double* src) {
 __device__ __forceinline__ void team_sum_partials(double* T, const double* pbase, int ntile, int count,
                                                   int tid, int nthreads) {
   const int pairs = count >> 1;
+  if (ntile == 1) {
+    // one matrix (already summed, or a one-tile request): a plain copy, eight loads in flight per thread
+    const double2* src = reinterpret_cast<const double2*>(pbase);
+    for (int e0 = tid; e0 < pairs; e0 += 8 * nthreads) {
+      double2 v[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) v[u] = __ldcg(src + min(e0 + u * nthreads, pairs - 1));
+#pragma unroll
+      for (int u = 0; u < 8; ++u)
+        if (e0 + u * nthreads < pairs) reinterpret_cast<double2*>(T)[e0 + u * nthreads] = v[u];
+    }
+    return;
+  }
   for (int e0 = tid; e0 < pairs; e0 += 4 * nthreads) {
     int e[4];
     double2 s[4];
@@ -232,7 +245,10 @@ __device__ __forceinline__ void factor_diag_thread(double* D, const double* d0, 
 // tiles are replaced by the identity here.
 //   store(I, J, tile, rd)   receives the factor tile (I, J) (64 doubles, row-major) and the array of
 //                           reciprocal diagonal entries; called by a whole warp
-template <typename Store, typename Sync>
+// kEarlyStore: warp 4 (idle in the panel loop) hands panel J - 1 to store() during iteration J (the
+// panel is final since the last barrier) instead of leaving all tiles to the end; the team then has
+// at least five warps.
+template <bool kEarlyStore = false, typename Store, typename Sync>
 __device__ __forceinline__ void cholesky_blocked_team(int n, double* T, double* aux, int tid, int nthreads,
                                                       Store store, Sync sync) {
   const int lane = tid & 31, warp = tid >> 5, nw = nthreads >> 5;
@@ -328,13 +344,23 @@ __device__ __forceinline__ void cholesky_blocked_team(int n, double* T, double* 
           update_tile(J, I1, K1);
         }
       }
+    } else if (kEarlyStore && warp == 4 && J >= 1) {
+      for (int I = J - 1; I < nb; ++I) store(I, J - 1, T + tri_index(I, J - 1) * 64, rd);
     }
     sync();
   }
-  for (int t = warp; t < ntile; t += nw) {
-    int I, J;
-    tri_decode(t, I, J);
-    store(I, J, T + t * 64, rd);
+  if constexpr (kEarlyStore) {
+    // the last two panels (or the only one)
+    int t = 0;
+    for (int J = nb >= 2 ? nb - 2 : 0; J < nb; ++J)
+      for (int I = J; I < nb; ++I, ++t)
+        if (t % nw == warp) store(I, J, T + tri_index(I, J) * 64, rd);
+  } else {
+    for (int t = warp; t < ntile; t += nw) {
+      int I, J;
+      tri_decode(t, I, J);
+      store(I, J, T + t * 64, rd);
+    }
   }
 }
 
@@ -385,19 +411,22 @@ __device__ __forceinline__ bool extra_tile(int e, int nb8, int units, int& ta, i
 // max_i 2 (theta_i / theta_1) (theta_min / theta_i)^q_final over the kept directions i < r that the
 // cut can tell apart from the discarded ones (theta_i - theta_min > 1e-3 theta_1), the estimate
 // team_ritz reports at the end; stop_below is the bound it has to stay under (0: never stop early).
+// pad: also write the entries of the layout that no factor touches (the first factorisation of a
+// launch does; they stay as they are for the later ones).
 __device__ __noinline__ bool team_cholesky(const double* pbase, int nt, int p, int r, float* out, double* Tm,
-                                           float* dg, volatile int* s_word, int q_final, float stop_below) {
+                                           float* dg, volatile int* s_word, int q_final, float stop_below,
+                                           bool pad) {
   const int et = threadIdx.x, warp = et >> 5, lane = et & 31;
   const int P = (p + 7) & ~7, nb = (p + 7) >> 3;
   auto epi_sync = [&]() { named_barrier(1, kEpiThreads); };
   // identity padding of the layout rows / columns p .. P-1 and the entries left of the diagonal
-  for (int i = warp; i < P; i += 8) {
+  for (int i = warp; pad && i < P; i += 8) {
     int j0 = i & ~3;
     float* row = out + lt_row_offset(i, P) - j0;
     for (int j = j0 + lane; j < P; j += 32)
       if (j < i || i >= p || j >= p) row[j] = (i == j) ? 1.f : 0.f;
   }
-  for (int j = p + et; j < P; j += kEpiThreads) out[kLtFloats + j] = 1.f;
+  for (int j = p + et; pad && j < P; j += kEpiThreads) out[kLtFloats + j] = 1.f;
   team_sum_partials(Tm, pbase, nt, nb * (nb + 1) / 2 * 64, et, kEpiThreads);
   epi_sync();
   if (stop_below > 0.f) {
@@ -434,7 +463,7 @@ __device__ __noinline__ bool team_cholesky(const double* pbase, int nt, int p, i
       if (I == J && (lane & 3) == 0) out[kLtFloats + j] = (float)rd[j];
     }
   };
-  cholesky_blocked_team(p, Tm, Tm + (size_t)nb * (nb + 1) / 2 * 64, et, kEpiThreads, store, epi_sync);
+  cholesky_blocked_team<true>(p, Tm, Tm + (size_t)nb * (nb + 1) / 2 * 64, et, kEpiThreads, store, epi_sync);
   return stop;
 }
 
@@ -707,7 +736,7 @@ subspace_kernel(const __grid_constant__ CUtensorMap map_gh, const __grid_constan
         const bool may_stop = prm.early_stop && step >= 1 && step + 1 < last_b && p < rp.m;
         const float margin = step == 1 ? 0.015625f : 0.125f;
         stop = team_cholesky(pbase, nt_sum, p, rp.r, prm.lbuf + (size_t)b * kLbufStride, Tm, dinv,
-                             s_word, step + 2, may_stop ? margin * prm.conv_tol : 0.f);
+                             s_word, step + 2, may_stop ? margin * prm.conv_tol : 0.f, step == 0);
         __threadfence();
         epi_sync();
         if (et == 0) {

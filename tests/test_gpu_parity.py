@@ -85,6 +85,16 @@ def test_two_sm_relevance_kernel(kw):
     _report(wl.name, parity.run_gpu(wl, pruner_kw=dict(relevance_path=2)))
 
 
+@pytest.mark.parametrize("d", [136, 1104])
+def test_relevance_kernel_several_items_per_block(d):
+    # more (token tile, head pair) items than SMs, so that every block of the relevance kernel walks
+    # through several of them (its ring and accumulator phases wrap); three and eighteen k-chunks; an
+    # odd number of heads leaves a single head in the last pair
+    wl = workloads.make_workload(f"items-d{d}", seed=23, dtype=torch.bfloat16, batch=3, n_vis=(3000, 9000),
+                                 n_txt=(5, 64), d=d, n_heads=5, rank=8, keep_ratio=0.02)
+    _report(wl.name, parity.run_gpu(wl))
+
+
 def test_degenerate_requests():
     # N = 1; B_vis >= N (keep everything); B_vis = N - 1; B_vis = 1; T = 1
     wl = workloads.make_workload("degenerate", seed=21, dtype=torch.bfloat16, batch=6,

@@ -107,7 +107,7 @@ def test_host_side_rejections(lib):
     for kw, code in [(dict(d=12), -3), (dict(d=64, n_heads=2, head_dim=64), -3),
                      (dict(d=64, lam=1.5), -1), (dict(d=64, rank_cap=150, eig_oversample=32), -3),
                      (dict(d=64, act_layers=40), -3), (dict(d=64, presel_factor=0.5), -1),
-                     (dict(d=64, dtype=7), -1)]:
+                     (dict(d=64, dtype=7), -1), (dict(d=64, relevance_path=3), -1)]:
         c = api.default_config(**kw)
         c.max_batch, c.max_total_vis, c.max_total_txt, c.max_vis_per_req = 1, 8, 8, 8
         assert lib.covspec_prune_init(C.byref(c), C.byref(out)) == code and not out.value
