@@ -173,7 +173,12 @@ int covspec_compact_rows(covspec_ctx* ctx, const covspec_problem* p, const int* 
                          void* stream);
 
 /* The whole path, Eq. 10 through the compacted buffer, in one call.  out_hidden device
- * [sum B_vis, d]; keep_idx device [sum B_vis]; keep_offsets host [batch+1] (may be NULL). */
+ * [sum B_vis, d]; keep_idx device [sum B_vis]; keep_offsets host [batch+1] (may be NULL).
+ * The call only enqueues work: on `stream` and on a second stream of the context that forks from it
+ * and joins it again; it never waits for the device.  The plan of a batch shape (offsets, budgets)
+ * is uploaded by the first call that sees it; later calls with the same offsets copy nothing from
+ * the host, so they may be recorded by stream capture and replayed as a CUDA graph (the graph keeps
+ * the device pointers of `p` and of the outputs; new contents in the same buffers are fine). */
 int covspec_prune(covspec_ctx* ctx, const covspec_problem* p, void* out_hidden, int* keep_idx,
                   int* keep_offsets, void* stream);
 
