@@ -281,9 +281,10 @@ int get_plan(covspec_ctx* ctx, const covspec_problem* p, cudaStream_t stream) {
 
   // Schedule of the subspace kernel.  Its items (row tiles) differ in cost (basis size p, rows
   // in the tile), and every step of a request ends when its slowest tile does.  With more tiles
-  // than CTAs, consecutive tiles of one request are therefore merged into groups and a group goes
-  // to one CTA as a whole: a CTA that carries several tiles then delays one request instead of
-  // several.  Groups are handed out longest first, each to the least loaded CTA.
+  // than CTAs, consecutive tiles of one request therefore form groups and a group goes to one CTA
+  // as a whole: a CTA that carries several tiles then delays one request instead of several.
+  // Groups are handed out longest first, each to the least loaded CTA (with more requests than CTAs
+  // every request is one group and the hand-out stacks them).
   // When SMs are left over, one more CTA per stage-2 request does nothing but factor for it (see the
   // kernel): their item lists are empty.
   pl.tile_ctas = std::min(pl.n_ptiles, ctx->num_sms);
@@ -294,31 +295,79 @@ int get_plan(covspec_ctx* ctx, const covspec_problem* p, cudaStream_t stream) {
     auto tile_cost = [&](const ReqPlan& r, int t) {
       int rows = std::min(pl.tile_rows, r.m - t * pl.tile_rows);
       double pp = (double)r.p;
-      return pp * pp * (1.0 + 1.5 * rows / sub::kTile) + 64.0 * r.m;
+      return pp * pp * (1.75 + 0.75 * rows / sub::kTile) + 10.0 * r.m;
     };
-    // start with one group per tile; while there are more groups than CTAs, merge the cheapest pair
-    // of neighbouring groups of one request (requests are never mixed inside a group)
+    // Every stage-2 request gets CTAs of its own and runs its steps independently of the others, so the
+    // call ends with the request whose steps take longest.  A request's tiles are split into g
+    // consecutive groups whose sizes differ by at most one, the larger ones last (the last tile may
+    // be ragged, hence cheaper); its step time is the cost of its most expensive group.  The number of
+    // groups per request (sum = CTAs) minimises the largest step time: the smallest feasible bound
+    // is found among the step times every request can have; CTAs that are left then go, one at a
+    // time, to the request that is slowest at that moment.  Requests are never mixed inside a group.
     struct Group { double cost; int first, count, req; };
+    struct Share { int req, nt, g; };
     std::vector<Group> groups;
-    for (int b = 0; b < B; ++b) {
-      const ReqPlan& r = pl.req[b];
-      if (!r.stage2) continue;
-      int nt = (r.m + pl.tile_rows - 1) / pl.tile_rows;
-      for (int t = 0; t < nt; ++t) groups.push_back(Group{tile_cost(r, t), r.ptile_off + t, 1, b});
-    }
-    while ((int)groups.size() > pl.tile_ctas) {
-      int best = -1;
-      double best_cost = 0.0;
-      for (int g = 0; g + 1 < (int)groups.size(); ++g) {
-        if (groups[g].req != groups[g + 1].req) continue;
-        double c = groups[g].cost + groups[g + 1].cost;
-        if (best < 0 || c < best_cost) { best = g; best_cost = c; }
+    std::vector<Share> shares;
+    for (int b = 0; b < B; ++b)
+      if (pl.req[b].stage2) shares.push_back(Share{b, (pl.req[b].m + pl.tile_rows - 1) / pl.tile_rows, 1});
+    // calls fn(first tile, tile count, cost) for every group of the split into g groups
+    auto split = [&](const Share& sh, int g, auto&& fn) {
+      const ReqPlan& r = pl.req[sh.req];
+      const int small = sh.nt / g, n_large = sh.nt % g;
+      for (int i = 0, t = 0; i < g; ++i) {
+        const int count = small + (i >= g - n_large ? 1 : 0);
+        double cost = 0.0;
+        for (int q = 0; q < count; ++q) cost += tile_cost(r, t + q);
+        fn(t, count, cost);
+        t += count;
       }
-      if (best < 0) break;                         // more requests than CTAs: the hand-out below stacks them
-      groups[best].cost = best_cost;
-      groups[best].count += groups[best + 1].count;
-      groups.erase(groups.begin() + best + 1);
+    };
+    auto step_time = [&](const Share& sh, int g) {
+      double worst = 0.0;
+      split(sh, g, [&](int, int, double cost) { worst = std::max(worst, cost); });
+      return worst;
+    };
+    if ((int)shares.size() < pl.tile_ctas) {
+      // times[i][g - 1]: step time of request i on g groups
+      std::vector<std::vector<double>> times(shares.size());
+      std::vector<double> cand;
+      for (size_t i = 0; i < shares.size(); ++i)
+        for (int g = 1; g <= shares[i].nt; ++g) {
+          times[i].push_back(step_time(shares[i], g));
+          cand.push_back(times[i].back());
+        }
+      std::sort(cand.begin(), cand.end());
+      auto fewest_groups = [&](size_t i, double bound) {       // nt: one tile per group always fits
+        for (int g = 1; g < shares[i].nt; ++g)
+          if (times[i][g - 1] <= bound) return g;
+        return shares[i].nt;
+      };
+      auto groups_needed = [&](double bound) {
+        long long n = 0;
+        for (size_t i = 0; i < shares.size(); ++i)
+          n += times[i].back() <= bound ? fewest_groups(i, bound) : (long long)1 << 40;
+        return n;
+      };
+      size_t lo = 0, hi = cand.size() - 1;           // the largest candidate needs one group per request
+      while (lo < hi) {
+        size_t mid = (lo + hi) / 2;
+        if (groups_needed(cand[mid]) <= pl.tile_ctas) hi = mid; else lo = mid + 1;
+      }
+      int used = 0;
+      for (size_t i = 0; i < shares.size(); ++i) used += shares[i].g = fewest_groups(i, cand[lo]);
+      for (; used < pl.tile_ctas; ++used) {
+        int worst = -1;
+        for (size_t i = 0; i < shares.size(); ++i)
+          if (shares[i].g < shares[i].nt &&
+              (worst < 0 || times[i][shares[i].g - 1] > times[worst][shares[worst].g - 1])) worst = (int)i;
+        if (worst < 0) break;
+        ++shares[worst].g;
+      }
     }
+    for (const Share& sh : shares)
+      split(sh, sh.g, [&](int t, int count, double cost) {
+        groups.push_back(Group{cost, pl.req[sh.req].ptile_off + t, count, sh.req});
+      });
     std::stable_sort(groups.begin(), groups.end(), [](const Group& a, const Group& b2) { return a.cost > b2.cost; });
     std::vector<double> load(pl.tile_ctas, 0.0);
     std::vector<std::vector<int>> lists(pl.tile_ctas);
