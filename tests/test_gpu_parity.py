@@ -95,6 +95,18 @@ def test_relevance_kernel_several_items_per_block(d):
     _report(wl.name, parity.run_gpu(wl))
 
 
+def test_more_requests_than_sms_and_more_tiles_than_sms():
+    # 170 stage-2 requests of two to six row tiles: every request is one group of the subspace kernel's
+    # schedule and the CTAs carry more than one request; then 24 requests with up to twelve tiles, whose
+    # tiles are split into groups so that the slowest request's step is as short as the CTAs allow
+    many = workloads.make_workload("many-requests", seed=104, dtype=torch.bfloat16, batch=170, n_vis=(260, 700),
+                                   n_txt=(2, 20), d=128, n_heads=1, rank=8, keep_ratio=0.3)
+    _report(many.name, parity.run_gpu(many))
+    ragged = workloads.make_workload("many-tiles", seed=101, dtype=torch.bfloat16, batch=24, n_vis=(500, 3000),
+                                     n_txt=(4, 60), d=256, n_heads=2, rank=24, keep_ratio=0.25)
+    _report(ragged.name, parity.run_gpu(ragged))
+
+
 def test_degenerate_requests():
     # N = 1; B_vis >= N (keep everything); B_vis = N - 1; B_vis = 1; T = 1
     wl = workloads.make_workload("degenerate", seed=21, dtype=torch.bfloat16, batch=6,
